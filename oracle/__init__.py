@@ -1,0 +1,185 @@
+"""ctypes front-end of the CPU oracle (``sparkattn_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by the smoke check and by
+the benchmark's CPU-baseline leg.  The CUDA package never imports this module
+and this module never imports the CUDA package.
+
+All tensors are CPU torch tensors; bf16 data is passed as its raw 16-bit
+pattern, FP8 data as raw E4M3 codes plus fp32 block scales.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sparkattn_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-shared", "-fPIC", "-Wall",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_LIB)
+        L.oracle_e4m3_decode.restype = ctypes.c_double
+        L.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        L.oracle_e4m3_encode.restype = ctypes.c_uint8
+        L.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+        L.oracle_attention.restype = ctypes.c_int
+        L.oracle_select.restype = ctypes.c_int
+        L.oracle_select_f64_diff.restype = ctypes.c_int64
+        L.oracle_quant_fp8.restype = None
+        L.oracle_pool.restype = None
+        L.oracle_num_threads.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.device.type == "cpu" and t.is_contiguous()
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _raw16(x: torch.Tensor) -> torch.Tensor:
+    assert x.dtype == torch.bfloat16
+    return x.contiguous().view(torch.int16)
+
+
+def e4m3_decode(code: int) -> float:
+    return float(_load().oracle_e4m3_decode(ctypes.c_uint8(code)))
+
+
+def e4m3_encode(y: float) -> int:
+    return int(_load().oracle_e4m3_encode(ctypes.c_float(y)))
+
+
+def e4m3_encode_array(y: np.ndarray) -> np.ndarray:
+    L = _load()
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    out = np.empty(y.shape, dtype=np.uint8)
+    yf, of = y.reshape(-1), out.reshape(-1)
+    for i in range(yf.size):
+        of[i] = L.oracle_e4m3_encode(ctypes.c_float(float(yf[i])))
+    return out
+
+
+def attention(
+    q: torch.Tensor,
+    k: torch.Tensor,
+    v: torch.Tensor,
+    kept_idx: torch.Tensor,
+    kept_cnt: torch.Tensor,
+    block: int,
+    items: Optional[Sequence[Tuple[int, int]]] = None,
+    scales: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
+    softmax_scale: float = 0.0,
+):
+    """ATT-0.  q, k, v: [H, N, d] bf16, or uint8 E4M3 codes with
+    ``scales = (q_scale, k_scale, v_scale)`` each fp32 [H, nb].
+    kept_idx int32 [H, nb, kmax], kept_cnt int32 [H, nb].
+    Returns (out fp64 [n_items, block, d], lse fp64 [n_items, block]) for the
+    (head, query-block) pairs in ``items`` (default: all, head-major)."""
+    L = _load()
+    H, N, d = q.shape
+    nb = (N + block - 1) // block
+    kmax = kept_idx.shape[-1]
+    assert kept_idx.shape == (H, nb, kmax) and kept_cnt.shape == (H, nb)
+    if items is None:
+        items = [(h, i) for h in range(H) for i in range(nb)]
+    it = torch.tensor(list(items), dtype=torch.int32).reshape(-1, 2).contiguous()
+    n_items = it.shape[0]
+    out = torch.zeros((n_items, block, d), dtype=torch.float64)
+    lse = torch.zeros((n_items, block), dtype=torch.float64)
+    if scales is None:
+        dtype = 0
+        qq, kk, vv = _raw16(q), _raw16(k), _raw16(v)
+        sq = sk = sv = None
+    else:
+        dtype = 1
+        assert q.dtype == torch.uint8
+        qq, kk, vv = q.contiguous(), k.contiguous(), v.contiguous()
+        sq, sk, sv = (s.contiguous().float() for s in scales)
+    ki = kept_idx.contiguous().to(torch.int32)
+    kc = kept_cnt.contiguous().to(torch.int32)
+    rc = L.oracle_attention(
+        ctypes.c_int(dtype), _ptr(qq), _ptr(kk), _ptr(vv), _ptr(sq), _ptr(sk), _ptr(sv),
+        ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d), ctypes.c_int(block),
+        _ptr(ki), _ptr(kc), ctypes.c_int(kmax), ctypes.c_double(softmax_scale),
+        _ptr(it), ctypes.c_int(n_items), _ptr(out), _ptr(lse))
+    if rc != 0:
+        raise ValueError("kept_idx holds a block index outside [0, nb)")
+    return out, lse
+
+
+def pool(x: torch.Tensor, block: int) -> torch.Tensor:
+    """SEL-1 steps 1-2: pooled fp32 block means [H, nb, d] of a bf16 [H, N, d] tensor."""
+    L = _load()
+    H, N, d = x.shape
+    nb = (N + block - 1) // block
+    out = torch.empty((H, nb, d), dtype=torch.float32)
+    L.oracle_pool(_ptr(_raw16(x)), ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d),
+                  ctypes.c_int(block), _ptr(out))
+    return out
+
+
+def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, return_scores: bool = False):
+    """SEL-1.  q, k: [H, N, d] bf16.  Returns kept_idx int32 [H, nb, topk]
+    (ascending), kept_cnt int32 [H, nb] (and the fp32 scores [H, nb, nb])."""
+    L = _load()
+    H, N, d = q.shape
+    nb = (N + block - 1) // block
+    idx = torch.empty((H, nb, topk), dtype=torch.int32)
+    cnt = torch.empty((H, nb), dtype=torch.int32)
+    scores = torch.empty((H, nb, nb), dtype=torch.float32) if return_scores else None
+    rc = L.oracle_select(_ptr(_raw16(q)), _ptr(_raw16(k)), ctypes.c_int(H), ctypes.c_int(N),
+                         ctypes.c_int(d), ctypes.c_int(block), ctypes.c_int(topk),
+                         _ptr(idx), _ptr(cnt), _ptr(scores))
+    if rc != 0:
+        raise ValueError("topk must be in [1, nb]")
+    return (idx, cnt, scores) if return_scores else (idx, cnt)
+
+
+def select_f64_diff(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, kept_idx: torch.Tensor):
+    """Diagnostic: rows whose fp64 top-k set differs from ``kept_idx`` and the
+    smallest relative gap between the k-th and (k+1)-th fp64 score."""
+    L = _load()
+    H, N, d = q.shape
+    gap = ctypes.c_double(0.0)
+    n = L.oracle_select_f64_diff(_ptr(_raw16(q)), _ptr(_raw16(k)), ctypes.c_int(H), ctypes.c_int(N),
+                                 ctypes.c_int(d), ctypes.c_int(block), ctypes.c_int(topk),
+                                 _ptr(kept_idx.contiguous().to(torch.int32)), ctypes.byref(gap))
+    return int(n), float(gap.value)
+
+
+def quant_fp8(x: torch.Tensor, block: int):
+    """QNT-1.  x: [H, N, d] bf16.  Returns (codes uint8 [H, N, d], scales fp32 [H, nb])."""
+    L = _load()
+    H, N, d = x.shape
+    nb = (N + block - 1) // block
+    codes = torch.zeros((H, N, d), dtype=torch.uint8)
+    scales = torch.zeros((H, nb), dtype=torch.float32)
+    L.oracle_quant_fp8(_ptr(_raw16(x)), ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d),
+                       ctypes.c_int(block), _ptr(codes), _ptr(scales))
+    return codes, scales
