@@ -1,0 +1,159 @@
+/*
+ * sparkattn -- block-sparse attention for long video-DiT token sequences on
+ * NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no framework types.
+ *
+ * The library implements the sparse branch O_s = A_M(Q, K, V) of the paper's
+ * compensated sparse attention (Sec. 2, "Block sparsity" and "Compensated
+ * sparse attention"; Sec. 4.1): the attention matrix is cut into contiguous
+ * query-block x key-block tiles, a selector keeps a fraction 1 - s of the key
+ * blocks for every query block, and exact softmax attention
+ * softmax(Q K^T / sqrt(d)) V is evaluated over the kept tiles only.
+ *
+ * Three device entry points make up the path:
+ *   sparkattn_select     pooled block scores + top-k -> kept-block index lists
+ *   sparkattn_quant_fp8  per-(head, token-block) absmax scale + E4M3 encode
+ *   sparkattn_fwd        block-sparse flash-attention forward (bf16 or FP8)
+ * plus one host-buffer convenience call that chains them with the copies.
+ *
+ * Conventions shared by all calls
+ *   - Every data pointer is DEVICE memory owned by the caller unless a
+ *     parameter name ends in `_host`.  The library allocates nothing, keeps
+ *     no pointer after the call returns and keeps no per-call global state.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream) and return without synchronising,
+ *     except sparkattn_read_status and sparkattn_attention_host.
+ *   - Tensors are [B, H, N, d] with d contiguous; strides are in elements.
+ *   - Tokens are cut into nb = ceil(N / block) contiguous blocks; the last
+ *     block may be ragged.  Rows >= N are never read as data or written.
+ *   - Return value: SPARKATTN_OK (0) or a negative sparkattn_status code.
+ *     Argument errors are detected on the host before anything is enqueued.
+ *     Errors found on the device (a kept index outside [0, nb), a wait that
+ *     ran out) are recorded in the first word of the caller's workspace and
+ *     read back with sparkattn_read_status; the kernel skips the offending
+ *     tile and still terminates.
+ *   - Same inputs give bitwise identical outputs (no atomics on data, fixed
+ *     reduction order).
+ */
+#ifndef SPARKATTN_H_
+#define SPARKATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPARKATTN_VERSION 1
+
+typedef enum {
+  SPARKATTN_OK = 0,
+  SPARKATTN_E_INVALID_ARG = -1,       /* NULL pointer, non-positive size, topk/kmax out of range      */
+  SPARKATTN_E_UNSUPPORTED_SHAPE = -2, /* (d, block) not one of (64,64), (128,128); nb too large        */
+  SPARKATTN_E_MISALIGNED = -3,        /* pointer not 16-byte aligned or stride * elem not 16-byte mult. */
+  SPARKATTN_E_WORKSPACE_TOO_SMALL = -4,
+  SPARKATTN_E_CUDA = -5,              /* launch or driver error; cudaGetLastError has the detail       */
+  SPARKATTN_E_DEVICE_TIMEOUT = -6,    /* a bounded device-side wait expired (device status word)       */
+  SPARKATTN_E_BAD_INDEX = -7,         /* a kept block index outside [0, nb) (device status word)       */
+  SPARKATTN_E_NO_DEVICE = -8          /* no CUDA device / driver entry point unavailable               */
+} sparkattn_status;
+
+typedef enum { SPARKATTN_BF16 = 0, SPARKATTN_FP8_E4M3 = 1 } sparkattn_dtype;
+
+/* Problem shape.  Caller fills it; the library reads it during the call only. */
+typedef struct {
+  uint32_t struct_size; /* sizeof(sparkattn_shape_t)                                   */
+  uint32_t version;     /* SPARKATTN_VERSION                                           */
+  int32_t B, H, N, d;   /* batch, heads (queries and keys share them), tokens, head dim */
+  int32_t block;        /* tokens per query block = tokens per key block               */
+  int32_t reserved;     /* must be 0                                                   */
+  int64_t stride_b, stride_h, stride_n; /* element strides of [B,H,N,d]; d has stride 1 */
+  float softmax_scale;  /* 0 selects 1/sqrt(d) (the paper's dense attention formula)   */
+  uint32_t pad;         /* must be 0                                                   */
+} sparkattn_shape_t;
+
+int sparkattn_version(void);
+const char* sparkattn_status_string(int status);
+
+/* Bytes of device workspace a call needs.  which: 0 = sparkattn_select,
+ * 1 = sparkattn_fwd.  Returns 0 for an invalid shape. */
+size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t topk_or_kmax);
+
+/*
+ * Block selection (the selector M_phi of Sec. 2 / Sec. 4.1; the paper names
+ * "top-k selection, blockwise scores" without fixing a rule, so the rule is:)
+ *   1. pooled sum over the valid tokens of a block, fp32, ascending token order
+ *   2. pooled mean = sum / n_valid (IEEE fp32 divide)
+ *   3. score(i, j) = fmaf chain over channels c ascending of pq[i,c] * pk[j,c]
+ *   4. keep the `topk` key blocks first under (score descending, index ascending)
+ *   5. write them in ascending index order.
+ * Selection always reads the bf16 Q and K (Sec. 4.3 keeps mask selection in BF16).
+ *
+ * q_bf16, k_bf16 : in,  bf16 [B,H,N,d] with the strides of `shape`
+ * topk           : in,  1 .. nb
+ * kept_idx       : out, int32 [B,H,nb,topk] contiguous
+ * kept_cnt       : out, int32 [B,H,nb] (every entry = topk); may be NULL
+ * workspace      : scratch of >= sparkattn_workspace_bytes(shape, 0, topk) bytes,
+ *                  256-byte aligned; its first word is the device status.
+ */
+int sparkattn_select(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                     int32_t* kept_idx, int32_t* kept_cnt, void* workspace, size_t workspace_bytes,
+                     void* cuda_stream);
+
+/*
+ * Fused FP8 quantisation (Sec. 4.3: FP8 E4M3, scale and cast in one pass over
+ * memory; the granularity here is one scale per (batch, head, token block)).
+ *   amax = max |x| over the block's valid tokens x d ; amax = max(amax, 1e-12)
+ *   scale = amax / 448 ; code = e4m3_rne_satfinite(x * (448 / amax))
+ * x_bf16 : in,  bf16 [B,H,N,d] (strides of `shape`)
+ * codes  : out, uint8 E4M3 codes, same element strides as x
+ * scales : out, fp32 [B,H,nb] contiguous dequantisation scales (value = decode(code) * scale)
+ * flags  : must be 0
+ */
+int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes, float* scales,
+                        uint32_t flags, void* cuda_stream);
+
+/*
+ * Block-sparse attention forward (Sec. 2 dense attention formula restricted
+ * to the kept tiles; Sec. 4.1 sparse branch).  For query token i in query
+ * block qb, over the keys j of the kept key blocks kept_idx[b,h,qb,0..cnt):
+ *   out[i,:] = sum_j softmax_j(scale * q_i . k_j) v_j ,  lse[i] = ln sum_j exp(scale * q_i . k_j)
+ * Keys >= N in a ragged last block are masked.  cnt = 0 gives out = 0, lse = -inf.
+ *
+ * dtype      : SPARKATTN_BF16: q,k,v bf16.  SPARKATTN_FP8_E4M3: q,k,v are E4M3
+ *              codes from sparkattn_quant_fp8 with q_scale/k_scale/v_scale fp32
+ *              [B,H,nb]; requires d = block = 128.  Scales are NULL for bf16.
+ * kept_idx   : in, int32 [B,H,nb,kmax]; entries distinct, each in [0, nb)
+ * kept_cnt   : in, int32 [B,H,nb] with 0 <= cnt <= kmax; NULL means cnt = kmax everywhere
+ * out_bf16   : out, bf16 [B,H,N,d], same strides as q
+ * lse        : out, fp32 [B,H,N] contiguous (natural log); may be NULL
+ * workspace  : >= sparkattn_workspace_bytes(shape, 1, kmax) bytes, 256-byte aligned
+ * Accumulation, row maximum and row sum are fp32; P is rounded to the input
+ * dtype for the second product.
+ */
+int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+                  const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                  const int32_t* kept_cnt, int32_t kmax, void* out_bf16, float* lse, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises the stream and returns the device status word of a workspace
+ * (SPARKATTN_OK, SPARKATTN_E_BAD_INDEX or SPARKATTN_E_DEVICE_TIMEOUT). */
+int sparkattn_read_status(void* workspace, void* cuda_stream);
+
+/*
+ * Whole path on HOST buffers: copies Q, K, V to the device arena, runs
+ * select (+ quant for FP8) + fwd, copies the output back and synchronises.
+ * q_host, k_host, v_host, out_host: contiguous bf16 [B,H,N,d] in (preferably
+ * pinned) host memory; kept_idx_host may be NULL or int32 [B,H,nb,topk] to
+ * receive the selected lists.  arena: device scratch of at least
+ * sparkattn_arena_bytes(shape, dtype, topk) bytes, 256-byte aligned.
+ */
+size_t sparkattn_arena_bytes(const sparkattn_shape_t* shape, int32_t dtype, int32_t topk);
+int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, const void* q_host,
+                             const void* k_host, const void* v_host, int32_t topk, void* out_host,
+                             int32_t* kept_idx_host, void* arena, size_t arena_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARKATTN_H_ */

@@ -1,0 +1,228 @@
+"""Python binding of the sparkattn C-ABI library (``libsparkattn.so``).
+
+Argument marshalling only: every step of the path (block selection, FP8
+quantisation, block-sparse attention) runs in the CUDA kernels behind the
+``extern "C"`` entry points declared in ``include/sparkattn.h``.  PyTorch is
+used for device memory and streams.  There is no CPU fallback: if the shared
+library is missing or cannot be loaded, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsparkattn.so")
+VERSION = 1
+
+OK = 0
+E_INVALID_ARG = -1
+E_UNSUPPORTED_SHAPE = -2
+E_MISALIGNED = -3
+E_WORKSPACE_TOO_SMALL = -4
+E_CUDA = -5
+E_DEVICE_TIMEOUT = -6
+E_BAD_INDEX = -7
+E_NO_DEVICE = -8
+
+BF16 = 0
+FP8_E4M3 = 1
+
+EXPORTS = (
+    "sparkattn_version", "sparkattn_status_string", "sparkattn_workspace_bytes", "sparkattn_select",
+    "sparkattn_quant_fp8", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
+    "sparkattn_attention_host",
+)
+
+
+class Shape(ctypes.Structure):
+    """Mirror of ``sparkattn_shape_t``."""
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("version", ctypes.c_uint32),
+        ("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32), ("d", ctypes.c_int32),
+        ("block", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64),
+        ("softmax_scale", ctypes.c_float), ("pad", ctypes.c_uint32),
+    ]
+
+
+class SparkAttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2609_23153_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        sp = ctypes.POINTER(Shape)
+        L.sparkattn_version.restype = ctypes.c_int
+        L.sparkattn_status_string.restype = ctypes.c_char_p
+        L.sparkattn_status_string.argtypes = [ctypes.c_int]
+        L.sparkattn_workspace_bytes.restype = sz
+        L.sparkattn_workspace_bytes.argtypes = [sp, i32, i32]
+        L.sparkattn_select.restype = ctypes.c_int
+        L.sparkattn_select.argtypes = [sp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.sparkattn_quant_fp8.restype = ctypes.c_int
+        L.sparkattn_quant_fp8.argtypes = [sp, vp, vp, vp, ctypes.c_uint32, vp]
+        L.sparkattn_fwd.restype = ctypes.c_int
+        L.sparkattn_fwd.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.sparkattn_read_status.restype = ctypes.c_int
+        L.sparkattn_read_status.argtypes = [vp, vp]
+        L.sparkattn_arena_bytes.restype = sz
+        L.sparkattn_arena_bytes.argtypes = [sp, i32, i32]
+        L.sparkattn_attention_host.restype = ctypes.c_int
+        L.sparkattn_attention_host.argtypes = [sp, i32, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().sparkattn_status_string(int(status)).decode()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise SparkAttnError(rc, where)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> ctypes.c_void_p:
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def make_shape(x: torch.Tensor, block: int, softmax_scale: float = 0.0) -> Shape:
+    """Shape descriptor for a [B, H, N, d] tensor (d contiguous, arbitrary outer strides)."""
+    if x.dim() != 4 or x.stride(3) != 1:
+        raise ValueError("expected a [B, H, N, d] tensor with a contiguous last dimension")
+    B, H, N, d = x.shape
+    return Shape(ctypes.sizeof(Shape), VERSION, B, H, N, d, block, 0,
+                 x.stride(0), x.stride(1), x.stride(2), float(softmax_scale), 0)
+
+
+def _same_layout(ref: torch.Tensor, *others: torch.Tensor) -> None:
+    for o in others:
+        if o.shape != ref.shape or o.stride() != ref.stride():
+            raise ValueError("tensors of one call must share shape and strides")
+
+
+def workspace_bytes(shape: Shape, which: int, topk_or_kmax: int) -> int:
+    return int(lib().sparkattn_workspace_bytes(ctypes.byref(shape), which, topk_or_kmax))
+
+
+def alloc_workspace(shape: Shape, which: int, topk_or_kmax: int, device) -> torch.Tensor:
+    n = workspace_bytes(shape, which, topk_or_kmax)
+    if n == 0:
+        raise SparkAttnError(E_UNSUPPORTED_SHAPE, "sparkattn_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def read_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> int:
+    return int(lib().sparkattn_read_status(_ptr(workspace), _stream_ptr(stream)))
+
+
+def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, *,
+           kept_idx: Optional[torch.Tensor] = None, kept_cnt: Optional[torch.Tensor] = None,
+           workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+           ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_select``: q, k bf16 [B,H,N,d] on the device -> (kept_idx int32
+    [B,H,nb,topk] ascending, kept_cnt int32 [B,H,nb])."""
+    _same_layout(q, k)
+    shape = make_shape(q, block)
+    B, H, N, _ = q.shape
+    nb = (N + block - 1) // block
+    if kept_idx is None:
+        kept_idx = torch.empty((B, H, nb, max(topk, 1)), dtype=torch.int32, device=q.device)
+    if kept_cnt is None:
+        kept_cnt = torch.empty((B, H, nb), dtype=torch.int32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(shape, 0, topk, q.device)
+    rc = lib().sparkattn_select(ctypes.byref(shape), _ptr(q), _ptr(k), topk, _ptr(kept_idx), _ptr(kept_cnt),
+                                _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_select")
+    return kept_idx, kept_cnt
+
+
+def quant_fp8(x: torch.Tensor, block: int, *, codes: Optional[torch.Tensor] = None,
+              scales: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+              ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_quant_fp8``: x bf16 [B,H,N,d] -> (codes uint8, same strides; scales fp32 [B,H,nb])."""
+    shape = make_shape(x, block)
+    B, H, N, _ = x.shape
+    nb = (N + block - 1) // block
+    if codes is None:
+        codes = torch.empty_strided(x.shape, x.stride(), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty((B, H, nb), dtype=torch.float32, device=x.device)
+    rc = lib().sparkattn_quant_fp8(ctypes.byref(shape), _ptr(x), _ptr(codes), _ptr(scales), 0, _stream_ptr(stream))
+    _check(rc, "sparkattn_quant_fp8")
+    return codes, scales
+
+
+def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tensor,
+        kept_cnt: Optional[torch.Tensor], block: int, *,
+        scales: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
+        softmax_scale: float = 0.0, out: Optional[torch.Tensor] = None, return_lse: bool = False,
+        workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+        check_status: bool = False):
+    """``sparkattn_fwd``.  bf16 q,k,v, or uint8 E4M3 codes with ``scales=(q_scale,
+    k_scale, v_scale)``.  Returns out bf16 [B,H,N,d] (and lse fp32 [B,H,N])."""
+    _same_layout(q, k, v)
+    shape = make_shape(q, block, softmax_scale)
+    B, H, N, _ = q.shape
+    dtype = BF16 if scales is None else FP8_E4M3
+    kmax = kept_idx.shape[-1]
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    if workspace is None:
+        workspace = alloc_workspace(shape, 1, kmax, q.device)
+    sq, sk, sv = scales if scales is not None else (None, None, None)
+    rc = lib().sparkattn_fwd(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(sq), _ptr(sk), _ptr(sv),
+                             _ptr(kept_idx), _ptr(kept_cnt), kmax, _ptr(out), _ptr(lse), _ptr(workspace),
+                             workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_fwd")
+    if check_status:
+        _check(read_status(workspace, stream), "sparkattn_fwd (device status)")
+    return (out, lse) if return_lse else out
+
+
+def arena_bytes(shape: Shape, dtype: int, topk: int) -> int:
+    return int(lib().sparkattn_arena_bytes(ctypes.byref(shape), dtype, topk))
+
+
+def attention_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, block: int, topk: int, *,
+                   dtype: int = BF16, out: Optional[torch.Tensor] = None,
+                   kept_idx: Optional[torch.Tensor] = None, arena: Optional[torch.Tensor] = None,
+                   device="cuda:0", stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """``sparkattn_attention_host``: q, k, v contiguous bf16 HOST tensors (pinned for
+    speed); runs copy-in, select, (quant,) fwd, copy-out and returns the host output."""
+    for t in (q, k, v):
+        if t.device.type != "cpu" or not t.is_contiguous() or t.dtype != torch.bfloat16:
+            raise ValueError("attention_host expects contiguous bf16 CPU tensors")
+    shape = make_shape(q, block)
+    if out is None:
+        out = torch.empty_like(q).pin_memory()
+    if arena is None:
+        arena = torch.empty(arena_bytes(shape, dtype, topk), dtype=torch.uint8, device=device)
+    rc = lib().sparkattn_attention_host(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), topk, _ptr(out),
+                                        _ptr(kept_idx), _ptr(arena), arena.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_attention_host")
+    return out

@@ -1,0 +1,208 @@
+// C-ABI layer of sparkattn: argument validation, workspace sizing and the
+// host-buffer convenience path.  All device work is in select.cu, quant.cu and
+// fwd.cu; nothing here touches tensor data on the CPU.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+using namespace sparkattn;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_shape(const sparkattn_shape_t* s) {
+  if (s == nullptr) return SPARKATTN_E_INVALID_ARG;
+  if (s->struct_size != sizeof(sparkattn_shape_t) || s->version != SPARKATTN_VERSION) return SPARKATTN_E_INVALID_ARG;
+  if (s->B < 1 || s->H < 1 || s->N < 1 || s->reserved != 0 || s->pad != 0) return SPARKATTN_E_INVALID_ARG;
+  if (!(s->softmax_scale >= 0.0f) || isinf(s->softmax_scale)) return SPARKATTN_E_INVALID_ARG;
+  if (!((s->d == 64 && s->block == 64) || (s->d == 128 && s->block == 128))) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (s->stride_n < s->d || s->stride_h < 1 || s->stride_b < 1) return SPARKATTN_E_INVALID_ARG;
+  // 16-byte rule for vector loads and TMA, for 2-byte and for 1-byte elements
+  if (s->stride_n % 16 || s->stride_h % 16 || s->stride_b % 16) return SPARKATTN_E_MISALIGNED;
+  if ((long long)s->B * s->H > 65535LL * 32768LL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  return SPARKATTN_OK;
+}
+
+inline int num_blocks(const sparkattn_shape_t* s) { return (s->N + s->block - 1) / s->block; }
+
+}  // namespace
+
+extern "C" {
+
+int sparkattn_version(void) { return SPARKATTN_VERSION; }
+
+const char* sparkattn_status_string(int status) {
+  switch (status) {
+    case SPARKATTN_OK: return "ok";
+    case SPARKATTN_E_INVALID_ARG: return "invalid argument";
+    case SPARKATTN_E_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case SPARKATTN_E_MISALIGNED: return "misaligned pointer or stride";
+    case SPARKATTN_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case SPARKATTN_E_CUDA: return "CUDA error";
+    case SPARKATTN_E_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case SPARKATTN_E_BAD_INDEX: return "kept block index out of range";
+    case SPARKATTN_E_NO_DEVICE: return "no CUDA device or driver entry point";
+    default: return "unknown status";
+  }
+}
+
+size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t /*topk_or_kmax*/) {
+  if (check_shape(shape) != SPARKATTN_OK) return 0;
+  if (which == 0) return select_workspace_bytes(*shape);
+  if (which == 1) return fwd_workspace_bytes(*shape);
+  return 0;
+}
+
+int sparkattn_select(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                     int32_t* kept_idx, int32_t* kept_cnt, void* workspace, size_t workspace_bytes,
+                     void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!q_bf16 || !k_bf16 || !kept_idx || !workspace) return SPARKATTN_E_INVALID_ARG;
+  const int nb = num_blocks(shape);
+  if (topk < 1 || topk > nb) return SPARKATTN_E_INVALID_ARG;
+  if (nb > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (!aligned16(q_bf16) || !aligned16(k_bf16) || !aligned256(workspace)) return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < select_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  return launch_select(*shape, q_bf16, k_bf16, topk, kept_idx, kept_cnt, workspace, stream);
+}
+
+int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes, float* scales,
+                        uint32_t flags, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!x_bf16 || !codes || !scales || flags != 0) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned16(x_bf16) || !aligned16(codes)) return SPARKATTN_E_MISALIGNED;
+  return launch_quant_fp8(*shape, x_bf16, codes, scales, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+                  const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                  const int32_t* kept_cnt, int32_t kmax, void* out_bf16, float* lse, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (dtype != SPARKATTN_BF16 && dtype != SPARKATTN_FP8_E4M3) return SPARKATTN_E_INVALID_ARG;
+  if (!q || !k || !v || !kept_idx || !out_bf16 || !workspace) return SPARKATTN_E_INVALID_ARG;
+  if (kmax < 1 || kmax > num_blocks(shape)) return SPARKATTN_E_INVALID_ARG;
+  if (dtype == SPARKATTN_FP8_E4M3) {
+    if (!q_scale || !k_scale || !v_scale) return SPARKATTN_E_INVALID_ARG;
+    if (!(shape->d == 128 && shape->block == 128)) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  }
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out_bf16) || !aligned256(workspace))
+    return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < fwd_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  return launch_fwd(*shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, out_bf16, lse,
+                    workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sparkattn_read_status(void* workspace, void* cuda_stream) {
+  if (!workspace) return SPARKATTN_E_INVALID_ARG;
+  int32_t word = 0;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  return word;
+}
+
+// Arena layout of the host-buffer path (every region 256-byte aligned):
+//   q, k, v, out (bf16) | kept_idx | kept_cnt | select workspace | fwd workspace |
+//   FP8 only: q/k/v codes, q/k/v scales
+namespace {
+struct Arena {
+  size_t q, k, v, out, idx, cnt, ws_sel, ws_fwd, cq, ck, cv, sq, sk, sv, total;
+};
+Arena plan_arena(const sparkattn_shape_t& s, int dtype, int topk) {
+  Arena a;
+  const size_t nb = (size_t)num_blocks(&s);
+  const size_t elems = (size_t)s.B * s.H * s.N * s.d;
+  const size_t bhn = (size_t)s.B * s.H * nb;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+  a.q = take(elems * 2); a.k = take(elems * 2); a.v = take(elems * 2); a.out = take(elems * 2);
+  a.idx = take(bhn * topk * 4); a.cnt = take(bhn * 4);
+  sparkattn_shape_t c = s;
+  c.stride_n = s.d; c.stride_h = (int64_t)s.N * s.d; c.stride_b = (int64_t)s.H * s.N * s.d;
+  a.ws_sel = take(select_workspace_bytes(c));
+  a.ws_fwd = take(fwd_workspace_bytes(c));
+  a.cq = a.ck = a.cv = a.sq = a.sk = a.sv = 0;
+  if (dtype == SPARKATTN_FP8_E4M3) {
+    a.cq = take(elems); a.ck = take(elems); a.cv = take(elems);
+    a.sq = take(bhn * 4); a.sk = take(bhn * 4); a.sv = take(bhn * 4);
+  }
+  a.total = off;
+  return a;
+}
+}  // namespace
+
+size_t sparkattn_arena_bytes(const sparkattn_shape_t* shape, int32_t dtype, int32_t topk) {
+  if (check_shape(shape) != SPARKATTN_OK || topk < 1 || topk > num_blocks(shape)) return 0;
+  return plan_arena(*shape, dtype, topk).total;
+}
+
+int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, const void* q_host,
+                             const void* k_host, const void* v_host, int32_t topk, void* out_host,
+                             int32_t* kept_idx_host, void* arena, size_t arena_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!q_host || !k_host || !v_host || !out_host || !arena) return SPARKATTN_E_INVALID_ARG;
+  if (dtype != SPARKATTN_BF16 && dtype != SPARKATTN_FP8_E4M3) return SPARKATTN_E_INVALID_ARG;
+  const int nb = num_blocks(shape);
+  if (topk < 1 || topk > nb) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned256(arena)) return SPARKATTN_E_MISALIGNED;
+  sparkattn_shape_t s = *shape;  // host tensors are contiguous
+  s.stride_n = s.d; s.stride_h = (int64_t)s.N * s.d; s.stride_b = (int64_t)s.H * s.N * s.d;
+  const Arena a = plan_arena(s, dtype, topk);
+  if (arena_bytes < a.total) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(arena);
+  const size_t bytes = (size_t)s.B * s.H * s.N * s.d * 2;
+  if (cudaMemcpyAsync(base + a.q, q_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(base + a.k, k_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(base + a.v, v_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  int32_t* idx = reinterpret_cast<int32_t*>(base + a.idx);
+  int32_t* cnt = reinterpret_cast<int32_t*>(base + a.cnt);
+  rc = sparkattn_select(&s, base + a.q, base + a.k, topk, idx, cnt, base + a.ws_sel, select_workspace_bytes(s),
+                        cuda_stream);
+  if (rc != SPARKATTN_OK) return rc;
+  const void *fq = base + a.q, *fk = base + a.k, *fv = base + a.v;
+  const float *sq = nullptr, *sk = nullptr, *sv = nullptr;
+  if (dtype == SPARKATTN_FP8_E4M3) {
+    const size_t tensor_off[3] = {a.q, a.k, a.v}, code_off[3] = {a.cq, a.ck, a.cv}, scale_off[3] = {a.sq, a.sk, a.sv};
+    for (int i = 0; i < 3; ++i) {
+      rc = sparkattn_quant_fp8(&s, base + tensor_off[i], reinterpret_cast<uint8_t*>(base + code_off[i]),
+                               reinterpret_cast<float*>(base + scale_off[i]), 0, cuda_stream);
+      if (rc != SPARKATTN_OK) return rc;
+    }
+    fq = base + a.cq; fk = base + a.ck; fv = base + a.cv;
+    sq = reinterpret_cast<const float*>(base + a.sq);
+    sk = reinterpret_cast<const float*>(base + a.sk);
+    sv = reinterpret_cast<const float*>(base + a.sv);
+  }
+  rc = sparkattn_fwd(&s, dtype, fq, fk, fv, sq, sk, sv, idx, cnt, topk, base + a.out, nullptr, base + a.ws_fwd,
+                     fwd_workspace_bytes(s), cuda_stream);
+  if (rc != SPARKATTN_OK) return rc;
+  if (cudaMemcpyAsync(out_host, base + a.out, bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  if (kept_idx_host != nullptr &&
+      cudaMemcpyAsync(kept_idx_host, idx, (size_t)s.B * s.H * nb * topk * 4, cudaMemcpyDeviceToHost, stream) !=
+          cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  int32_t st[2] = {0, 0};
+  if (cudaMemcpyAsync(&st[0], base + a.ws_sel, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(&st[1], base + a.ws_fwd, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  return st[0] != 0 ? st[0] : st[1];
+}
+
+}  // extern "C"

@@ -1,0 +1,454 @@
+// sparkattn_fwd: block-sparse flash-attention forward for sm_100a.
+//
+// Computes the paper's sparse branch O_s = A_M(Q, K, V) (Sec. 4.1): exact
+// softmax attention (Sec. 2, softmax(Q K^T / sqrt(d)) V) restricted, for every
+// query block, to the key blocks of its kept list.
+//
+// One CTA owns one (batch, head, query block) work item; two CTAs share an SM
+// so that one item's softmax overlaps the other's tensor-core work.
+//   warps 0-3  softmax: thread r owns query row r.  tcgen05.ld S from TMEM,
+//              fp32 online softmax (row max / row sum need no shuffles: a row
+//              lives in one thread), P written back to TMEM over S in the
+//              input precision, conditional rescale of O, final normalise and
+//              store.
+//   warp 4     TMA producer: Q tile once, then K_j / V_j tiles of each kept
+//              block into one K slot and one V slot (128-byte swizzle).
+//   warp 5     MMA issuer: S = Q K_j^T (operands in shared memory) and
+//              O += P V_j (P from TMEM, V MN-major from shared memory) as
+//              tcgen05.mma with fp32 accumulators in TMEM.
+// TMEM columns: [0, BLK) S (P overlays its first BLK*elt/4 columns), [BLK, BLK+D) O.
+//
+// Every wait on an mbarrier is bounded (common.cuh); a kept index outside
+// [0, nb) is reported in the status word and its tile skipped by all roles.
+#include <cuda.h>
+#include <cuda_fp8.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace sparkattn {
+
+constexpr int kFwdThreads = 192;
+constexpr int kSoftmaxThreads = 128;
+// In log2 units: O and l are only rescaled when the running row maximum grows
+// by more than this; until then P may exceed 1 by at most 2^threshold, which
+// bf16 holds without loss.  Exact: the final division by l uses the same
+// reference maximum.  The FP8 path rescales on every increase (threshold 0)
+// because its P is pre-scaled close to the E4M3 maximum.
+constexpr float kLazyRescaleLog2 = 8.0f;
+constexpr float kFp8PScaleLog2 = 8.0f;  // P * 2^8 <= 256 < 448
+
+template <int D, int BLK, bool FP8>
+struct FwdCfg {
+  static constexpr int kElt = FP8 ? 1 : 2;
+  static constexpr int kSlabs = D * kElt / 128;          // 128-byte-wide column slabs per tile
+  static constexpr int kSlabElems = 128 / kElt;          // elements per slab row
+  static constexpr int kQSlabBytes = 128 * 128;          // MMA M = 128 rows
+  static constexpr int kKVSlabBytes = BLK * 128;
+  static constexpr int kQBytes = kSlabs * kQSlabBytes;
+  static constexpr int kKVBytes = kSlabs * kKVSlabBytes;
+  static constexpr int kTileTxBytes = kSlabs * BLK * 128;  // bytes one Q / K / V load delivers
+  static constexpr int kUmmaK = 32 / kElt;               // elements per MMA along K
+  static constexpr int kQKSteps = 128 / 32;              // MMAs per slab for S
+  static constexpr int kPVSteps = BLK / kUmmaK;          // MMAs for O
+  static constexpr int kPCols = BLK * kElt / 4;
+  static constexpr int kTmemCols = (BLK + D) <= 128 ? 128 : 256;
+  static constexpr int kSmemBytes = 1024 /*align slack*/ + kQBytes + 2 * kKVBytes + 256 /*barriers*/;
+  static_assert(D * kElt % 128 == 0 && BLK % 32 == 0 && D % 32 == 0, "tile shape");
+};
+
+struct FwdParams {
+  const int32_t* kept_idx;
+  const int32_t* kept_cnt;
+  const float* q_scale;
+  const float* k_scale;
+  const float* v_scale;
+  __nv_bfloat16* out;
+  float* lse;
+  int32_t* status;
+  int H, N, nb, kmax;
+  int64_t stride_b, stride_h, stride_n;
+  float scale_log2;  // softmax_scale * log2(e)
+};
+
+template <int D, int BLK, bool FP8>
+__global__ void __launch_bounds__(kFwdThreads, 2)
+fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+           const __grid_constant__ CUtensorMap tmap_v, const FwdParams p) {
+  using Cfg = FwdCfg<D, BLK, FP8>;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* sQ = smem;
+  unsigned char* sK = sQ + Cfg::kQBytes;
+  unsigned char* sV = sK + Cfg::kKVBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + Cfg::kKVBytes);
+  uint64_t* bar_q_full = bars + 0;
+  uint64_t* bar_k_full = bars + 1;
+  uint64_t* bar_v_full = bars + 2;
+  uint64_t* bar_s_full = bars + 3;   // S_n complete (also: K slot free)
+  uint64_t* bar_p_full = bars + 4;   // P_n written by all softmax threads
+  uint64_t* bar_o_done = bars + 5;   // O += P_n V_n complete (also: V slot and S/P columns free)
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(bars + 8);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 9);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int qb = blockIdx.x % p.nb;
+  const int bh = blockIdx.x / p.nb;
+  const int h = bh % p.H, b = bh / p.H;
+  const int cnt = p.kept_cnt ? min(max(p.kept_cnt[(int64_t)bh * p.nb + qb], 0), p.kmax) : p.kmax;
+  const int32_t* list = p.kept_idx + ((int64_t)bh * p.nb + qb) * p.kmax;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q_full, 1);
+    mbar_init(bar_k_full, 1);
+    mbar_init(bar_v_full, 1);
+    mbar_init(bar_s_full, 1);
+    mbar_init(bar_p_full, kSoftmaxThreads);
+    mbar_init(bar_o_done, 1);
+    // a timeout recorded by an earlier CTA of this launch makes the rest of the grid drain at once
+    *s_abort = (*reinterpret_cast<volatile int32_t*>(p.status) == SPARKATTN_E_DEVICE_TIMEOUT) ? 1 : 0;
+    mbar_fence_init();
+  }
+  if (warp == 4) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_q);
+      tma_prefetch_desc(&tmap_k);
+      tma_prefetch_desc(&tmap_v);
+    }
+    __syncwarp();
+    tmem_alloc(s_tmem_base, Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem_base;
+  const uint32_t tmem_S = tmem;
+  const uint32_t tmem_P = tmem;
+  const uint32_t tmem_O = tmem + BLK;
+  const bool dead = *s_abort != 0;
+
+  if (dead) {
+    // nothing to do: fall through to the teardown
+  } else if (warp == 4) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int n = 0;
+      for (int t = 0; t < cnt; ++t) {
+        const int kb = __ldg(list + t);
+        if (kb < 0 || kb >= p.nb) continue;
+        if (n == 0) {
+          mbar_expect_tx(bar_q_full, Cfg::kTileTxBytes);
+#pragma unroll
+          for (int s = 0; s < Cfg::kSlabs; ++s)
+            tma_load_4d(sQ + s * Cfg::kQSlabBytes, &tmap_q, bar_q_full, s * Cfg::kSlabElems, qb * BLK, h, b);
+        } else {
+          if (!mbar_wait(bar_s_full, (n - 1) & 1, s_abort, p.status, 1)) break;  // K slot free
+        }
+        mbar_expect_tx(bar_k_full, Cfg::kTileTxBytes);
+#pragma unroll
+        for (int s = 0; s < Cfg::kSlabs; ++s)
+          tma_load_4d(sK + s * Cfg::kKVSlabBytes, &tmap_k, bar_k_full, s * Cfg::kSlabElems, kb * BLK, h, b);
+        if (n > 0) {
+          if (!mbar_wait(bar_o_done, (n - 1) & 1, s_abort, p.status, 2)) break;  // V slot free
+        }
+        mbar_expect_tx(bar_v_full, Cfg::kTileTxBytes);
+#pragma unroll
+        for (int s = 0; s < Cfg::kSlabs; ++s)
+          tma_load_4d(sV + s * Cfg::kKVSlabBytes, &tmap_v, bar_v_full, s * Cfg::kSlabElems, kb * BLK, h, b);
+        ++n;
+      }
+    }
+  } else if (warp == 5) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t kFmt = FP8 ? 0u : 1u;
+      constexpr uint32_t idesc_qk = make_idesc(kFmt, 128, BLK, false);
+      constexpr uint32_t idesc_pv = make_idesc(kFmt, 128, D, true);
+      const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
+      int n = 0;
+      for (int t = 0; t < cnt; ++t) {
+        const int kb = __ldg(list + t);
+        if (kb < 0 || kb >= p.nb) continue;
+        if (n == 0) {
+          if (!mbar_wait(bar_q_full, 0, s_abort, p.status, 3)) break;
+        } else {
+          if (!mbar_wait(bar_o_done, (n - 1) & 1, s_abort, p.status, 4)) break;  // P_{n-1} consumed
+        }
+        if (!mbar_wait(bar_k_full, n & 1, s_abort, p.status, 5)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < Cfg::kSlabs; ++s) {
+#pragma unroll
+          for (int kk = 0; kk < Cfg::kQKSteps; ++kk) {
+            const uint64_t da = make_smem_desc_sw128(aQ + s * Cfg::kQSlabBytes + kk * 32, 16);
+            const uint64_t db = make_smem_desc_sw128(aK + s * Cfg::kKVSlabBytes + kk * 32, 16);
+            mma_ss<FP8>(tmem_S, da, db, idesc_qk, (s | kk) != 0);
+          }
+        }
+        tc_commit(bar_s_full);
+        if (!mbar_wait(bar_v_full, n & 1, s_abort, p.status, 6)) break;
+        if (!mbar_wait(bar_p_full, n & 1, s_abort, p.status, 7)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < Cfg::kPVSteps; ++kk) {
+          const uint64_t db = make_smem_desc_sw128(aV + kk * Cfg::kUmmaK * 128, Cfg::kKVSlabBytes);
+          mma_ts<FP8>(tmem_O, tmem_P + kk * 8, db, idesc_pv, (n | kk) != 0);
+        }
+        tc_commit(bar_o_done);
+        ++n;
+      }
+    }
+  } else {
+    // ----------------------------------------------------------------- softmax
+    const int row = threadIdx.x;                      // query row inside the block = TMEM lane
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    const int q_row = qb * BLK + row;
+    const bool row_valid = row < BLK && q_row < p.N;
+    float m_used = 0.0f, l = 0.0f;
+    float q_sc = 1.0f, v_max = 1.0f;
+    if constexpr (FP8) {
+      q_sc = __ldg(p.q_scale + (int64_t)bh * p.nb + qb);
+      float vm = 0.0f;
+      for (int j = 0; j < p.nb; ++j) vm = fmaxf(vm, __ldg(p.v_scale + (int64_t)bh * p.nb + j));
+      v_max = vm;
+    }
+    int n = 0;
+    bool ok = true;
+    for (int t = 0; t < cnt; ++t) {
+      const int kb = __ldg(list + t);
+      if (kb < 0 || kb >= p.nb) {
+        if (threadIdx.x == 0) report_status(p.status, SPARKATTN_E_BAD_INDEX, kb);
+        continue;
+      }
+      const int ncols = min(BLK, p.N - kb * BLK);    // valid keys in this block
+      float c = p.scale_log2;                        // logit -> log2 units
+      float p_off = 0.0f;                            // log2 of the factor folded into P
+      if constexpr (FP8) {
+        c *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb);
+        p_off = kFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb) / v_max);
+      }
+      ok = mbar_wait(bar_s_full, n & 1, s_abort, p.status, 8);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+
+      // pass 1: row maximum of the raw accumulators
+      float mx = -INFINITY;
+#pragma unroll
+      for (int ch = 0; ch < BLK / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_S + lane_off + ch * 32, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float s = __uint_as_float(r[i]);
+          if (ch * 32 + i < ncols) mx = fmaxf(mx, s);
+        }
+      }
+      const float m_new = mx * c;
+      float alpha = 1.0f;
+      bool need = false;
+      if (n == 0) {
+        m_used = m_new;
+      } else if (m_new > m_used + (FP8 ? 0.0f : kLazyRescaleLog2)) {
+        alpha = fast_exp2(m_used - m_new);
+        m_used = m_new;
+        need = true;
+      }
+      if (__any_sync(0xffffffffu, need)) {
+        // S_n complete implies O += P_{n-1} V_{n-1} complete: O is quiescent here.
+        l *= alpha;
+#pragma unroll
+        for (int ch = 0; ch < D / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tmem_O + lane_off + ch * 32, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+          tmem_st32(tmem_O + lane_off + ch * 32, r);
+        }
+      }
+
+      // pass 2: P = exp2(S*c - m) in the input precision, written over S
+      const float neg_m = p_off - m_used;
+      float l_tile = 0.0f;
+#pragma unroll
+      for (int ch = 0; ch < BLK / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_S + lane_off + ch * 32, r);
+        tc_wait_ld();
+        float pv[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float e = fast_exp2(fmaf(__uint_as_float(r[i]), c, neg_m));
+          pv[i] = (ch * 32 + i < ncols) ? e : 0.0f;
+          l_tile += pv[i];
+        }
+        if constexpr (FP8) {
+          uint32_t w[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(pv[4 * i], pv[4 * i + 1]), __NV_SATFINITE, __NV_E4M3);
+            const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(pv[4 * i + 2], pv[4 * i + 3]), __NV_SATFINITE, __NV_E4M3);
+            w[i] = lo | (hi << 16);
+          }
+          tmem_st8(tmem_P + lane_off + ch * 8, w);
+        } else {
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[2 * i], pv[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          tmem_st16(tmem_P + lane_off + ch * 16, w);
+        }
+      }
+      if constexpr (FP8) l += l_tile * fast_exp2(-p_off);
+      else l += l_tile;
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p_full);
+      ++n;
+    }
+
+    // ---------------------------------------------------------------- epilogue
+    __nv_bfloat16* orow = p.out + b * p.stride_b + h * p.stride_h + (int64_t)q_row * p.stride_n;
+    if (n == 0 || !ok) {
+      if (row_valid && ok) {
+#pragma unroll
+        for (int ch = 0; ch < D / 8; ++ch) reinterpret_cast<uint4*>(orow)[ch] = make_uint4(0u, 0u, 0u, 0u);
+        if (p.lse) p.lse[(int64_t)bh * p.N + q_row] = -INFINITY;
+      }
+    } else {
+      ok = mbar_wait(bar_o_done, (n - 1) & 1, s_abort, p.status, 9);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after();
+        float inv = 1.0f / l;
+        if constexpr (FP8) inv *= v_max * fast_exp2(-kFp8PScaleLog2);
+#pragma unroll
+        for (int ch = 0; ch < D / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tmem_O + lane_off + ch * 32, r);
+          tc_wait_ld();
+          if (row_valid) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[8 * i + 2 * j]) * inv,
+                                                                __uint_as_float(r[8 * i + 2 * j + 1]) * inv);
+                w[j] = *reinterpret_cast<const uint32_t*>(&h2);
+              }
+              reinterpret_cast<uint4*>(orow + ch * 32)[i] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        if (row_valid && p.lse) p.lse[(int64_t)bh * p.N + q_row] = (m_used + log2f(l)) * 0.6931471805599453f;
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    if (*s_abort) __nanosleep(200000);  // let copies / MMAs in flight land before the CTA's resources go
+    tc_fence_after();
+    tmem_dealloc(tmem, Cfg::kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  return fn;
+}
+
+// [B,H,N,d] tensor, box = one 128-byte-wide slab of `box_rows` token rows, 128-byte swizzle.
+static int make_tile_map(CUtensorMap* map, const void* base, int elt_bytes, const sparkattn_shape_t& s,
+                         int box_rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return SPARKATTN_E_NO_DEVICE;
+  const cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.H, (cuuint64_t)s.B};
+  const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * elt_bytes, (cuuint64_t)s.stride_h * elt_bytes,
+                                 (cuuint64_t)s.stride_b * elt_bytes};
+  const cuuint32_t box[4] = {(cuuint32_t)(128 / elt_bytes), (cuuint32_t)box_rows, 1u, 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r = enc(map, elt_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
+                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+size_t fwd_workspace_bytes(const sparkattn_shape_t&) { return kWorkspaceHeaderBytes; }
+
+template <int D, int BLK, bool FP8>
+static int launch_fwd_t(const sparkattn_shape_t& s, const CUtensorMap& mq, const CUtensorMap& mk,
+                        const CUtensorMap& mv, const FwdParams& prm, cudaStream_t stream) {
+  using Cfg = FwdCfg<D, BLK, FP8>;
+  // at least 100 KB so that no more than two CTAs (2 x <=256 TMEM columns) share an SM
+  const int smem = Cfg::kSmemBytes < 100 * 1024 ? 100 * 1024 : Cfg::kSmemBytes;
+  auto kern = fwd_kernel<D, BLK, FP8>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  const long long ctas = (long long)s.B * s.H * prm.nb;
+  if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  kern<<<(unsigned)ctas, kFwdThreads, smem, stream>>>(mq, mk, mv, prm);
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void* k, const void* v,
+               const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+               const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream) {
+  const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
+  const int elt = fp8 ? 1 : 2;
+  CUtensorMap mq, mk, mv;
+  int rc;
+  if ((rc = make_tile_map(&mq, q, elt, s, s.block)) != SPARKATTN_OK) return rc;
+  if ((rc = make_tile_map(&mk, k, elt, s, s.block)) != SPARKATTN_OK) return rc;
+  if ((rc = make_tile_map(&mv, v, elt, s, s.block)) != SPARKATTN_OK) return rc;
+  FwdParams prm;
+  prm.kept_idx = kept_idx;
+  prm.kept_cnt = kept_cnt;
+  prm.q_scale = q_scale;
+  prm.k_scale = k_scale;
+  prm.v_scale = v_scale;
+  prm.out = static_cast<__nv_bfloat16*>(out);
+  prm.lse = lse;
+  prm.status = static_cast<int32_t*>(workspace);
+  prm.H = s.H;
+  prm.N = s.N;
+  prm.nb = (s.N + s.block - 1) / s.block;
+  prm.kmax = kmax;
+  prm.stride_b = s.stride_b;
+  prm.stride_h = s.stride_h;
+  prm.stride_n = s.stride_n;
+  const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
+  prm.scale_log2 = sc * 1.4426950408889634f;
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  if (s.d == 128 && s.block == 128) {
+    return fp8 ? launch_fwd_t<128, 128, true>(s, mq, mk, mv, prm, stream)
+               : launch_fwd_t<128, 128, false>(s, mq, mk, mv, prm, stream);
+  }
+  if (s.d == 64 && s.block == 64 && !fp8) return launch_fwd_t<64, 64, false>(s, mq, mk, mv, prm, stream);
+  return SPARKATTN_E_UNSUPPORTED_SHAPE;
+}
+
+}  // namespace sparkattn

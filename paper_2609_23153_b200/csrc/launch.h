@@ -1,0 +1,29 @@
+// Internal host-side launch interface between the C-ABI layer (api.cu) and the
+// kernel translation units.  Every launcher validates nothing: api.cu has
+// already checked the arguments.  Each returns a sparkattn_status.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sparkattn.h"
+
+namespace sparkattn {
+
+// quant.cu
+int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
+                     cudaStream_t stream);
+
+// select.cu
+constexpr int kSelectMaxBlocks = 4096;  // largest nb the selection kernel holds in shared memory
+size_t select_workspace_bytes(const sparkattn_shape_t& s);
+int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int32_t* kept_idx,
+                  int32_t* kept_cnt, void* workspace, cudaStream_t stream);
+
+// fwd.cu
+size_t fwd_workspace_bytes(const sparkattn_shape_t& s);
+int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void* k, const void* v,
+               const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+               const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream);
+
+}  // namespace sparkattn

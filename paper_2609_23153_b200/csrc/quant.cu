@@ -1,0 +1,107 @@
+// sparkattn_quant_fp8: per-(batch, head, token block) absmax scale + E4M3
+// encode in one pass over memory (paper Sec. 4.3: FP8 E4M3, scaling and
+// casting fused in a single kernel).
+//
+// One CTA owns one token block: it loads the block's bf16 elements into
+// registers once (16-byte loads, rows contiguous), reduces |x| to the block
+// maximum, then scales, encodes (cvt.rn.satfinite.e4m3x2.f32) and stores from
+// the same registers, so HBM sees one read of x and one write of the codes:
+// 3 bytes per element.
+#include <cuda_fp8.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace sparkattn {
+
+constexpr int kQuantThreads = 256;
+
+template <int D, int BLK>
+__global__ void __launch_bounds__(kQuantThreads)
+quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ scales,
+                 int H, int N, int nb, int64_t stride_b, int64_t stride_h, int64_t stride_n) {
+  constexpr int kChunksPerRow = D / 8;                      // 16-byte chunks per token row
+  constexpr int kChunks = BLK * kChunksPerRow;              // chunks per token block
+  constexpr int kPerThread = kChunks / kQuantThreads;       // 8 for (128,128), 2 for (64,64)
+  static_assert(kChunks % kQuantThreads == 0, "block must split evenly over the CTA");
+
+  const int blk = blockIdx.x % nb;
+  const int bh = blockIdx.x / nb;
+  const int h = bh % H, b = bh / H;
+  const int row0 = blk * BLK;
+  const int nvalid = min(BLK, N - row0);
+  const int64_t base = b * stride_b + h * stride_h;
+
+  uint4 v[kPerThread];
+  float amax = 0.0f;
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int ci = threadIdx.x + i * kQuantThreads;
+    const int r = ci / kChunksPerRow, cc = ci % kChunksPerRow;
+    if (r < nvalid) {
+      v[i] = __ldg(reinterpret_cast<const uint4*>(x + base + (int64_t)(row0 + r) * stride_n + cc * 8));
+    } else {
+      v[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v[i]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(p[j]);
+      amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+    }
+  }
+  __shared__ float s_red[kQuantThreads / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = s_red[0];
+#pragma unroll
+  for (int w = 1; w < kQuantThreads / 32; ++w) amax = fmaxf(amax, s_red[w]);
+  amax = fmaxf(amax, 1e-12f);
+  const float inv = __fdiv_rn(448.0f, amax);
+  if (threadIdx.x == 0) scales[(int64_t)bh * nb + blk] = __fdiv_rn(amax, 448.0f);
+
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int ci = threadIdx.x + i * kQuantThreads;
+    const int r = ci / kChunksPerRow, cc = ci % kChunksPerRow;
+    if (r >= nvalid) continue;
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v[i]);
+    uint32_t w[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const float2 f0 = __bfloat1622float2(p[2 * j]);
+      const float2 f1 = __bfloat1622float2(p[2 * j + 1]);
+      const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f0.x, inv), __fmul_rn(f0.y, inv)),
+                                                    __NV_SATFINITE, __NV_E4M3);
+      const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f1.x, inv), __fmul_rn(f1.y, inv)),
+                                                    __NV_SATFINITE, __NV_E4M3);
+      w[j] = lo | (hi << 16);
+    }
+    *reinterpret_cast<uint2*>(codes + base + (int64_t)(row0 + r) * stride_n + cc * 8) = make_uint2(w[0], w[1]);
+  }
+}
+
+int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
+                     cudaStream_t stream) {
+  const int nb = (s.N + s.block - 1) / s.block;
+  const long long ctas = (long long)s.B * s.H * nb;
+  if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+  if (s.d == 128 && s.block == 128) {
+    quant_fp8_kernel<128, 128><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
+  } else if (s.d == 64 && s.block == 64) {
+    quant_fp8_kernel<64, 64><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
+  } else {
+    return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  }
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+}  // namespace sparkattn

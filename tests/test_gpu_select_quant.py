@@ -1,0 +1,107 @@
+"""GPU parity: sparkattn_select and sparkattn_quant_fp8 against the CPU oracle, bit for bit."""
+import pytest
+import torch
+
+import oracle
+import paper_2609_23153_b200 as sa
+import workloads
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _small_cases():
+    return [
+        workloads.small_structured(H=3, d=128, grid=(5, 12, 20), block=128, sparsity=0.8, cfg_id=11),   # N=1200: 9 full + tail 48
+        workloads.small_structured(H=2, d=128, grid=(3, 16, 16), block=128, sparsity=0.5, cfg_id=12),   # N=768: no tail
+        workloads.small_structured(H=2, d=64, grid=(3, 10, 21), block=64, sparsity=0.9, cfg_id=13),     # N=630: tail 54
+        workloads.small_structured(H=1, d=64, grid=(1, 1, 37), block=64, sparsity=0.0, cfg_id=14),      # one ragged block
+        workloads.small_structured(H=2, d=128, grid=(1, 1, 1), block=128, sparsity=0.0, cfg_id=15),     # N=1
+    ]
+
+
+@pytest.mark.parametrize("w", _small_cases(), ids=lambda w: f"{w.name}-N{w.N}-d{w.d}")
+def test_select_matches_oracle(w):
+    q, k, _ = workloads.structured_qkv(w)
+    for topk in sorted({1, w.topk, w.nb}):
+        ref_idx, ref_cnt = oracle.select(q[0], k[0], w.block, topk)
+        idx, cnt = sa.select(q.to(DEV), k.to(DEV), w.block, topk)
+        torch.cuda.synchronize()
+        assert torch.equal(idx[0].cpu(), ref_idx)
+        assert torch.equal(cnt[0].cpu(), ref_cnt)
+
+
+def test_select_tiny_workload_and_ties():
+    w = workloads.TINY
+    q, k, _ = workloads.tiny_inputs(w)
+    ref_idx, _ = oracle.select(q[0], k[0], w.block, 16)
+    idx, _ = sa.select(q.to(DEV), k.to(DEV), w.block, 16)
+    assert torch.equal(idx[0].cpu(), ref_idx)
+    # exact ties: every key block identical -> lowest indices win
+    kc = k.clone(); kc[:] = k[0, 0, 5]
+    ref_idx, _ = oracle.select(q[0], kc[0], w.block, 7)
+    idx, _ = sa.select(q.to(DEV), kc.to(DEV), w.block, 7)
+    assert torch.equal(idx[0].cpu(), ref_idx)
+    assert ref_idx[0, 0].tolist() == list(range(7))
+    # zero queries: all scores +0/-0 -> still the lowest indices
+    ref_idx, _ = oracle.select(torch.zeros_like(q[0]), -k[0], w.block, 5)
+    idx, _ = sa.select(torch.zeros_like(q).to(DEV), (-k).to(DEV), w.block, 5)
+    assert torch.equal(idx[0].cpu(), ref_idx)
+
+
+def test_select_strided_layout_and_batch():
+    # [B, N, H, d] storage viewed as [B, H, N, d]; two batches
+    w = workloads.small_structured(H=2, d=128, grid=(2, 10, 26), block=128, sparsity=0.75, cfg_id=16)
+    qs, ks = [], []
+    for b in range(2):
+        q, k, _ = workloads.structured_qkv(workloads.small_structured(2, 128, (2, 10, 26), 128, 0.75, cfg_id=16 + b))
+        qs.append(q[0]); ks.append(k[0])
+    q = torch.stack(qs); k = torch.stack(ks)
+    qd = q.permute(0, 2, 1, 3).contiguous().to(DEV).permute(0, 2, 1, 3)
+    kd = k.permute(0, 2, 1, 3).contiguous().to(DEV).permute(0, 2, 1, 3)
+    idx, cnt = sa.select(qd, kd, w.block, w.topk)
+    for b in range(2):
+        ref_idx, _ = oracle.select(q[b], k[b], w.block, w.topk)
+        assert torch.equal(idx[b].cpu(), ref_idx)
+
+
+@pytest.mark.parametrize("w", _small_cases(), ids=lambda w: f"{w.name}-N{w.N}-d{w.d}")
+def test_quant_matches_oracle(w):
+    q, _, v = workloads.structured_qkv(w)
+    for x in (q, v):
+        ref_codes, ref_scales = oracle.quant_fp8(x[0], w.block)
+        codes, scales = sa.quant_fp8(x.to(DEV), w.block)
+        torch.cuda.synchronize()
+        assert torch.equal(scales[0].cpu().view(torch.int32), ref_scales.view(torch.int32))
+        assert torch.equal(codes[0].cpu(), ref_codes)
+
+
+def test_quant_edge_values():
+    H, N, d, block = 2, 300, 128, 128
+    g = torch.Generator().manual_seed(21)
+    x = (torch.randn((1, H, N, d), generator=g) * 4).to(torch.bfloat16)
+    x[0, 0, :128] = 0                       # all-zero block
+    x[0, 1, 130, 7] = -1000.0               # one huge negative element: the rest underflows towards zero
+    x[0, 1, 131, 9] = 3.0e-3
+    x[0, 0, 256:] *= 1e-20                  # tiny magnitudes in the tail block
+    ref_codes, ref_scales = oracle.quant_fp8(x[0], block)
+    # canary: rows past N of a padded buffer must stay untouched
+    buf = torch.full((1, H, N + 20, d), 0xAB, dtype=torch.uint8, device=DEV)
+    xd = torch.zeros((1, H, N + 20, d), dtype=torch.bfloat16, device=DEV)
+    xd[:, :, :N] = x.to(DEV)
+    codes, scales = sa.quant_fp8(xd[:, :, :N], block, codes=buf[:, :, :N])
+    torch.cuda.synchronize()
+    assert torch.equal(codes[0].cpu(), ref_codes)
+    assert torch.equal(scales[0].cpu().view(torch.int32), ref_scales.view(torch.int32))
+    assert torch.all(buf[:, :, N:] == 0xAB)
+
+
+def test_select_and_quant_are_deterministic():
+    w = workloads.small_structured(H=4, d=128, grid=(4, 12, 20), block=128, sparsity=0.8, cfg_id=19)
+    q, k, v = (t.to(DEV) for t in workloads.structured_qkv(w))
+    a = sa.select(q, k, w.block, w.topk)[0].clone()
+    b = sa.select(q, k, w.block, w.topk)[0].clone()
+    assert torch.equal(a, b)
+    c1 = sa.quant_fp8(v, w.block)[0].clone()
+    c2 = sa.quant_fp8(v, w.block)[0].clone()
+    assert torch.equal(c1, c2)

@@ -1,0 +1,126 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every
+symbol the public header declares, and rejects bad arguments before touching
+the device."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+import paper_2609_23153_b200 as sa
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_23153_b200 import build
+    build.build()
+    return sa.lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "sparkattn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sparkattn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert set(sa.EXPORTS) <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in sparkattn.h but not exported"
+
+
+def test_version_and_status_strings(lib):
+    assert lib.sparkattn_version() == sa.VERSION
+    seen = set()
+    for code in range(0, -9, -1):
+        s = sa.status_string(code)
+        assert s and s != "unknown status" and s not in seen
+        seen.add(s)
+    assert sa.status_string(-99) == "unknown status"
+
+
+def _shape(B=1, H=2, N=2048, d=64, block=64):
+    return sa.Shape(ctypes.sizeof(sa.Shape), sa.VERSION, B, H, N, d, block, 0, H * N * d, N * d, d, 0.0, 0)
+
+
+def test_shape_struct_matches_header_size():
+    # 2*u32 + 6*i32 + 3*i64 + f32 + u32 = 64 bytes, no implicit padding
+    assert ctypes.sizeof(sa.Shape) == 64
+
+
+def test_workspace_sizes(lib):
+    s = _shape()
+    nb = 32
+    assert sa.workspace_bytes(s, 1, 16) == 256
+    assert sa.workspace_bytes(s, 0, 16) == 256 + 2 * nb * 64 * 4 + 2 * 64 * 32 * 4
+    assert sa.workspace_bytes(s, 2, 16) == 0
+    bad = _shape(d=96)
+    assert sa.workspace_bytes(bad, 0, 16) == 0
+    assert sa.arena_bytes(s, sa.BF16, 16) > 4 * 2 * 2048 * 64 * 2
+    assert sa.arena_bytes(s, sa.BF16, 0) == 0
+
+
+def test_argument_errors_are_caught_on_the_host(lib):
+    s = _shape()
+    fake = ctypes.c_void_p(0x1000)  # never dereferenced: validation fails first
+    null = ctypes.c_void_p(0)
+    st = ctypes.c_void_p(0)
+    r = lib.sparkattn_select(ctypes.byref(s), null, fake, 4, fake, null, fake, 1 << 20, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_select(ctypes.byref(s), fake, fake, 0, fake, null, fake, 1 << 20, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_select(ctypes.byref(s), fake, fake, 33, fake, null, fake, 1 << 20, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_select(ctypes.byref(s), fake, fake, 4, fake, null, fake, 16, st)
+    assert r == sa.E_WORKSPACE_TOO_SMALL
+    r = lib.sparkattn_select(ctypes.byref(s), ctypes.c_void_p(0x1008), fake, 4, fake, null, fake, 1 << 20, st)
+    assert r == sa.E_MISALIGNED
+    bad = _shape(d=96)
+    assert lib.sparkattn_quant_fp8(ctypes.byref(bad), fake, fake, fake, 0, st) == sa.E_UNSUPPORTED_SHAPE
+    assert lib.sparkattn_quant_fp8(ctypes.byref(s), fake, fake, fake, 1, st) == sa.E_INVALID_ARG
+    odd = _shape()
+    odd.stride_n = 72
+    assert lib.sparkattn_quant_fp8(ctypes.byref(odd), fake, fake, fake, 0, st) == sa.E_MISALIGNED
+    wrong = _shape()
+    wrong.version = 7
+    assert lib.sparkattn_quant_fp8(ctypes.byref(wrong), fake, fake, fake, 0, st) == sa.E_INVALID_ARG
+    # fwd: FP8 needs scales and the 128/128 shape; kmax in range
+    r = lib.sparkattn_fwd(ctypes.byref(s), sa.FP8_E4M3, fake, fake, fake, null, null, null, fake, null, 4, fake,
+                          null, fake, 256, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_fwd(ctypes.byref(s), sa.FP8_E4M3, fake, fake, fake, fake, fake, fake, fake, null, 4, fake,
+                          null, fake, 256, st)
+    assert r == sa.E_UNSUPPORTED_SHAPE
+    r = lib.sparkattn_fwd(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 40, fake,
+                          null, fake, 256, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_fwd(ctypes.byref(s), 5, fake, fake, fake, null, null, null, fake, null, 4, fake,
+                          null, fake, 256, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_fwd(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 4, fake,
+                          null, fake, 8, st)
+    assert r == sa.E_WORKSPACE_TOO_SMALL
+
+
+def test_binding_checks_layout():
+    q = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16)
+    with pytest.raises(ValueError):
+        sa.make_shape(q.transpose(2, 3), 64)
+    s = sa.make_shape(q, 64)
+    assert (s.B, s.H, s.N, s.d, s.block) == (1, 2, 128, 64, 64)
+    assert (s.stride_b, s.stride_h, s.stride_n) == (2 * 128 * 64, 128 * 64, 64)
+    # a [B, N, H, d] buffer viewed as [B, H, N, d]
+    x = torch.zeros((1, 128, 2, 64), dtype=torch.bfloat16).permute(0, 2, 1, 3)
+    s = sa.make_shape(x, 64)
+    assert (s.stride_h, s.stride_n) == (64, 128)
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(sa, "_lib", None)
+    monkeypatch.setattr(sa, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(ImportError):
+        sa.lib()
