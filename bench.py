@@ -1,0 +1,421 @@
+#!/usr/bin/env python
+"""Benchmark of the block-sparse attention path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload wan14b|wan1p3b] [--no-e2e] [--no-cpu] [--sweep]
+
+One "step" is one pass of the whole path over one batch of synthetic input
+resident in HBM: block selection (pool + top-k kernels) followed by the
+block-sparse attention forward, bf16, on the Wan2.1-14B-720P attention shape
+(B=1, H=40, N=75600, d=128, 128x128 blocks) at 97 % block sparsity.  The
+headline value is kept-block TFLOP/s = 4*d*sum(valid q rows * valid k rows
+over kept tiles) / step time.  The same JSON line also carries the FP8 leg
+(3 quantise launches + FP8 forward), per-kernel times, the roofline of the
+dominant kernel, the end-to-end number through the host-buffer C-ABI call and
+the CPU oracle timed on a bounded sample.
+
+With N > 1 (torchrun, one rank per GPU) every rank runs the same-shaped
+problem on its own seeded batch: batches are independent, so there is no
+data-path collective; the value is the aggregate over ranks ("weak" scaling).
+
+``--impl reference`` times the CPU oracle as it stands on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "block-sparse attn effective TFLOP/s (kept FLOPs), select+fwd, 97% sparse"
+UNIT = "TFLOP/s"
+# DRAM bytes (read + write) of one forward launch on the bench workload, from the
+# ncu capture summarised in profiles/fwd_bf16_wan14b_s97.md (null until captured).
+FWD_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16": float(p["bf16_tflops"]), "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "hbm": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16": 1590.0, "bf16_sustained": 1400.0, "hbm": 6650.0, "source": "fallback"}
+
+
+def kept_flops(w, kept_idx_cpu, kept_cnt_cpu, items=None):
+    """4*d*sum over kept (query block, key block) tiles of valid rows x valid keys."""
+    nb, blk, N = w.nb, w.block, w.N
+    valid = torch.full((nb,), blk, dtype=torch.int64)
+    valid[nb - 1] = w.tail
+    idx = kept_idx_cpu.reshape(-1, nb, kept_idx_cpu.shape[-1]).long()
+    cnt = kept_cnt_cpu.reshape(-1, nb).long()
+    mask = torch.arange(idx.shape[-1])[None, None, :] < cnt[..., None]
+    keys = (valid[idx.clamp(0, nb - 1)] * mask).sum(-1)           # [BH, nb] valid keys per query block
+    per_item = keys * valid[None, :]
+    if items is not None:
+        return 4 * w.d * int(sum(per_item[h, i] for h, i in items))
+    return 4 * w.d * int(per_item.sum())
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+
+def cpu_oracle_sample(w, target_seconds: float, head: int = 0):
+    """Times the CPU oracle (selection of one head in full + attention on a sample of
+    that head's query blocks) and returns kept-FLOP throughput of the sample."""
+    import oracle
+    cores = oracle.num_threads()
+    w1 = w.with_heads(1)
+    q, k, v = workloads.structured_qkv(w, heads=[head], device="cpu")
+    q, k, v = q[0], k[0], v[0]
+    t0 = time.perf_counter()
+    idx, cnt = oracle.select(q, k, w.block, w.topk)
+    t_sel = time.perf_counter() - t0
+    # calibrate on one batch of `cores` items, then size the sample for the time target
+    g = torch.Generator().manual_seed(1234)
+    order = torch.randperm(w.nb, generator=g).tolist()
+    first = [(0, i) for i in order[:cores]]
+    t0 = time.perf_counter()
+    oracle.attention(q, k, v, idx, cnt, w.block, items=first)
+    t_first = time.perf_counter() - t0
+    n_more = int(max(0, min(w.nb - cores, (target_seconds - t_first - t_sel) / max(t_first, 1e-6) * cores)))
+    rest = [(0, i) for i in order[cores:cores + n_more]]
+    t_rest = 0.0
+    if rest:
+        t0 = time.perf_counter()
+        oracle.attention(q, k, v, idx, cnt, w.block, items=rest)
+        t_rest = time.perf_counter() - t0
+    items = first + rest
+    flops = kept_flops(w1, idx, cnt, items)
+    t_total = t_first + t_rest + t_sel * len(items) / w.nb
+    return {"value": flops / t_total / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": (f"head {head} of {w.name}: oracle selection of the whole head ({t_sel:.2f} s, charged pro rata) + fp64 "
+                       f"oracle attention on {len(items)} of {w.nb} query blocks ({t_first + t_rest:.2f} s)"),
+            "seconds": t_total, "items": len(items)}
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle on the host cores, one bounded sample per step."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = oracle.num_threads()
+    q, k, v = workloads.structured_qkv(w, heads=[0], device="cpu")
+    q, k, v = q[0], k[0], v[0]
+    idx, cnt = oracle.select(q, k, w.block, w.topk)
+    w1 = w.with_heads(1)
+    g = torch.Generator().manual_seed(99)
+    per_step = 8 * max(1, cores)
+    times, flops = [], []
+    for step in range(args.warmup + args.steps):
+        items = [(0, int(i)) for i in torch.randint(0, w.nb, (per_step,), generator=g)]
+        t0 = time.perf_counter()
+        oracle.attention(q, k, v, idx, cnt, w.block, items=items)
+        dt = time.perf_counter() - t0
+        if step >= args.warmup:
+            times.append(dt); flops.append(kept_flops(w1, idx, cnt, items))
+    total_t, total_f = sum(times), sum(flops)
+    value = total_f / total_t / 1e12
+    sample = (f"each step: fp64 oracle attention on {per_step} random query blocks of head 0 of {w.name} "
+              f"(kept lists from the oracle's own selection); throughput = kept FLOPs / time")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(1, len(times)), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_dict(w, "bf16"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def config_dict(w, dtype):
+    return {"workload": f"{w.name}: B={w.B} H={w.H} N={w.N} d={w.d} grid={'x'.join(map(str, w.grid))} "
+                        f"block={w.block} sparsity={w.sparsity} (kept {w.topk} of {w.nb} key blocks per query block)",
+            "dtype_inputs": dtype, "selection": "pooled-score top-k (sparkattn_select)",
+            "l2": "inputs (3 x 774 MB) exceed the 126 MB L2; no explicit flush",
+            "parallelism": "independent batch per GPU, no collective"}
+
+
+# --------------------------------------------------------------------------- GPU leg
+
+def time_region(fn, steps, warmup, stream, dist_on):
+    """warmup untimed calls, then `steps` timed calls between barrier+sync; returns max-over-ranks ms."""
+    for _ in range(warmup):
+        fn(-1)
+    if dist_on:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if dist_on:
+        torch.distributed.barrier()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def run_ours(args, w):
+    import paper_2609_23153_b200 as sa
+    from paper_2609_23153_b200 import build as sa_build
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist_on = world > 1
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if dist_on:
+        torch.distributed.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        sa_build.build()
+    if dist_on:
+        torch.distributed.barrier()
+    sa.lib()
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+
+    # every rank owns an independent batch of the same shape (different seed)
+    wr = workloads.Workload(w.name, w.cfg_id + 1000 * rank, w.B, w.H, w.d, w.grid, w.block, w.sparsity)
+    q, k, v = workloads.structured_qkv(wr, device=dev)
+    topk, nb = w.topk, w.nb
+    shape = sa.make_shape(q, w.block)
+    ws_sel = sa.alloc_workspace(shape, 0, topk, dev)
+    ws_fwd = sa.alloc_workspace(shape, 1, topk, dev)
+    kept_idx = torch.empty((w.B, w.H, nb, topk), dtype=torch.int32, device=dev)
+    kept_cnt = torch.empty((w.B, w.H, nb), dtype=torch.int32, device=dev)
+    out = torch.empty_like(q)
+
+    K = args.steps
+    ev = {name: [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+          for name in ("select", "fwd")}
+
+    def step(i):
+        if i >= 0:
+            ev["select"][i][0].record(stream)
+        sa.select(q, k, w.block, topk, kept_idx=kept_idx, kept_cnt=kept_cnt, workspace=ws_sel)
+        if i >= 0:
+            ev["select"][i][1].record(stream); ev["fwd"][i][0].record(stream)
+        sa.fwd(q, k, v, kept_idx, kept_cnt, w.block, out=out, workspace=ws_fwd)
+        if i >= 0:
+            ev["fwd"][i][1].record(stream)
+
+    with ClockSampler(local) as clk:
+        ms_total = time_region(step, K, args.warmup, stream, dist_on)
+    clocks = clk.summary()
+    for wsb, name in ((ws_sel, "select"), (ws_fwd, "fwd")):
+        st = sa.read_status(wsb)
+        if st != sa.OK:
+            raise RuntimeError(f"device status after {name}: {sa.status_string(st)}")
+    ms_step = ms_total / K
+    ms_sel = statistics.mean(a.elapsed_time(b) for a, b in ev["select"])
+    ms_fwd = statistics.mean(a.elapsed_time(b) for a, b in ev["fwd"])
+    idx_cpu, cnt_cpu = kept_idx.cpu(), kept_cnt.cpu()
+    flops = kept_flops(w, idx_cpu, cnt_cpu)
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    fwd_tflops = flops / (ms_fwd * 1e-3) / 1e12
+    elems = w.B * w.H * w.N * w.d
+    sel_bytes = 2 * elems * 2 + kept_idx.numel() * 4 + kept_cnt.numel() * 4
+    kernels = {
+        "select": {"ms": ms_sel, "launches_per_step": 2, "algorithmic_bytes": sel_bytes,
+                   "GBps": sel_bytes / (ms_sel * 1e-3) / 1e9, "frac_of_hbm_peak": sel_bytes / (ms_sel * 1e-3) / 1e9 / peaks["hbm"]},
+        "fwd_bf16": {"ms": ms_fwd, "launches_per_step": 1, "TFLOPs": fwd_tflops},
+    }
+    roofline = {"kernel": "fwd_kernel<128,128,bf16>", "bound": "tensor", "achieved": fwd_tflops, "peak": peaks["bf16"],
+                "unit": "TFLOP/s", "frac": fwd_tflops / peaks["bf16"], "traffic": FWD_DRAM_TRAFFIC_BYTES,
+                "peak_source": f"{peaks['source']} bf16 burst (sustained {peaks['bf16_sustained']})",
+                "flops_per_launch": flops, "ms_per_launch": ms_fwd}
+
+    # ---- FP8 leg: 3 quantise launches + FP8 forward (selection reuses the bf16 lists)
+    fp8 = None
+    if not args.no_fp8:
+        codes = [torch.empty(q.shape, dtype=torch.uint8, device=dev) for _ in range(3)]
+        scales = [torch.empty((w.B, w.H, nb), dtype=torch.float32, device=dev) for _ in range(3)]
+        evq = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        evf = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+
+        def step8(i):
+            if i >= 0:
+                evq[i][0].record(stream)
+            for t, c, s in zip((q, k, v), codes, scales):
+                sa.quant_fp8(t, w.block, codes=c, scales=s)
+            if i >= 0:
+                evq[i][1].record(stream); evf[i][0].record(stream)
+            sa.fwd(codes[0], codes[1], codes[2], kept_idx, kept_cnt, w.block, scales=tuple(scales), out=out,
+                   workspace=ws_fwd)
+            if i >= 0:
+                evf[i][1].record(stream)
+
+        ms8 = time_region(step8, K, args.warmup, stream, dist_on) / K
+        if sa.read_status(ws_fwd) != sa.OK:
+            raise RuntimeError("device status after fp8 fwd")
+        ms_q = statistics.mean(a.elapsed_time(b) for a, b in evq)
+        ms_f8 = statistics.mean(a.elapsed_time(b) for a, b in evf)
+        qbytes = 3 * (elems * 3 + scales[0].numel() * 4)
+        fp8 = {"ms_per_step_quant_plus_fwd": ms8, "quant_ms_3_tensors": ms_q, "quant_GBps": qbytes / (ms_q * 1e-3) / 1e9,
+               "quant_frac_of_hbm_peak": qbytes / (ms_q * 1e-3) / 1e9 / peaks["hbm"],
+               "fwd_ms": ms_f8, "fwd_TFLOPs": flops / (ms_f8 * 1e-3) / 1e12,
+               "fwd_frac_of_nominal_fp8_peak_4500": flops / (ms_f8 * 1e-3) / 1e12 / 4500.0,
+               "fwd_frac_of_2x_measured_bf16_peak": flops / (ms_f8 * 1e-3) / 1e12 / (2 * peaks["bf16"])}
+        del codes
+
+    # ---- sparsity sweep (optional): fwd only, lists from sparkattn_select
+    sweep = None
+    if args.sweep:
+        sweep = []
+        for s in (0.0, 0.5, 0.75, 0.9, 0.97):
+            ws_ = w.with_sparsity(s)
+            ki, kc = sa.select(q, k, w.block, ws_.topk, workspace=ws_sel)
+            reps = 2 if s < 0.6 else 5
+            sa.fwd(q, k, v, ki, kc, w.block, out=out, workspace=ws_fwd)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                sa.fwd(q, k, v, ki, kc, w.block, out=out, workspace=ws_fwd)
+            b.record(stream); torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / reps
+            fl = kept_flops(w, ki.cpu(), kc.cpu())
+            sweep.append({"sparsity": s, "kept": ws_.topk, "dtype": "bf16", "ms": ms, "TFLOPs": fl / ms / 1e9,
+                          "frac_of_bf16_peak": fl / ms / 1e9 / peaks["bf16"]})
+            del ki, kc
+
+    # ---- end to end through the host-buffer C-ABI call (H2D of Q,K,V and D2H of O inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        del out
+        torch.cuda.empty_cache()
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+        ho = torch.empty_like(hq).pin_memory()
+        arena = torch.empty(sa.arena_bytes(shape, sa.BF16, topk), dtype=torch.uint8, device=dev)
+        ke = max(1, min(K, args.e2e_steps))
+
+        def step_e2e(i):
+            sa.attention_host(hq, hk, hv, w.block, topk, out=ho, arena=arena)
+
+        ms_e = time_region(step_e2e, ke, 1, stream, dist_on) / ke
+        e2e = {"value": world * flops / (ms_e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e, "steps": ke,
+               "h2d_bytes_per_step": 3 * hq.numel() * 2, "d2h_bytes_per_step": ho.numel() * 2 + 8,
+               "call": "sparkattn_attention_host (pinned host Q,K,V -> select -> fwd -> host O)"}
+        del arena, hq, hk, hv, ho
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_oracle_sample(w, target_seconds=args.cpu_seconds)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config_dict(w, "bf16"),
+            "kept_flops_per_step_per_gpu": flops, "clocks": clocks, "gpu_launches": 3 * K,
+            "kernels": kernels, "roofline": roofline, "fp8": fp8, "e2e": e2e, "cpu_baseline": cpu,
+        }
+        if sweep is not None:
+            line["sweep"] = sweep
+        print(json.dumps(line), flush=True)
+    if dist_on:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=["wan14b", "wan1p3b"], default="wan14b")
+    ap.add_argument("--sparsity", type=float, default=None)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-fp8", action="store_true")
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = workloads.WORKLOADS[args.workload]
+    if args.sparsity is not None:
+        w = w.with_sparsity(args.sparsity)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
