@@ -205,6 +205,20 @@ def config_dict(w, dtype):
 
 # --------------------------------------------------------------------------- GPU leg
 
+def max_over_ranks(value: float, device) -> float:
+    """Largest value over all ranks of the default process group (identity without one)."""
+    if not (torch.distributed.is_available() and torch.distributed.is_initialized()):
+        return value
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(flops_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job TFLOP/s when every rank did `flops_per_rank` in `ms` (the max over ranks)."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def time_region(fn, steps, warmup, stream, dist_on):
     """warmup untimed calls, then `steps` timed calls between barrier+sync; returns max-over-ranks ms."""
     for _ in range(warmup):
@@ -220,12 +234,7 @@ def time_region(fn, steps, warmup, stream, dist_on):
     torch.cuda.synchronize()
     if dist_on:
         torch.distributed.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist_on:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return max_over_ranks(e0.elapsed_time(e1), "cuda")
 
 
 def run_ours(args, w):
@@ -286,7 +295,7 @@ def run_ours(args, w):
     ms_fwd = statistics.mean(a.elapsed_time(b) for a, b in ev["fwd"])
     idx_cpu, cnt_cpu = kept_idx.cpu(), kept_cnt.cpu()
     flops = kept_flops(w, idx_cpu, cnt_cpu)
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = aggregate_throughput(flops, ms_step, world)
     fwd_tflops = flops / (ms_fwd * 1e-3) / 1e12
     elems = w.B * w.H * w.N * w.d
     sel_bytes = 2 * elems * 2 + kept_idx.numel() * 4 + kept_cnt.numel() * 4
