@@ -153,6 +153,39 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
                              const void* k_host, const void* v_host, int32_t topk, void* out_host,
                              int32_t* kept_idx_host, void* arena, size_t arena_bytes, void* cuda_stream);
 
+/*
+ * Block selection without any allocation (the paper has no counterpart: this
+ * is a packaging variant of sparkattn_select, same rule, same outputs).
+ *
+ * For callers that may not allocate device memory when they call: a serving
+ * loop whose memory budget was fixed at start-up, a host application whose
+ * allocator is frozen after initialisation, a plugin that only receives its
+ * input and output buffers.  The scratch that sparkattn_select takes as a
+ * workspace lives here in a fixed device array inside the library image, of
+ * sparkattn_select_noalloc_max_bytes() bytes (32 MiB), which every GPU that
+ * loads the library holds until the process exits.  The call itself performs
+ * no cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ *   - Arguments as for sparkattn_select, minus the workspace.  q_bf16, k_bf16,
+ *     kept_idx, kept_cnt are caller-owned device buffers.
+ *   - A shape whose scratch need (sparkattn_workspace_bytes(shape, 0, topk))
+ *     exceeds the array returns SPARKATTN_E_WORKSPACE_TOO_SMALL and enqueues
+ *     nothing; the other argument errors are those of sparkattn_select.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and caches it; make that first call before starting
+ *     any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous
+ *     call's contents; the library clears what must start at zero.  Calls whose
+ *     kernels can overlap on the GPU (different streams or threads) race on it:
+ *     serialise them.
+ *   - sparkattn_select_noalloc_status synchronises the stream and returns the
+ *     device status word of the last call on the current device.
+ */
+size_t sparkattn_select_noalloc_max_bytes(void);
+int sparkattn_select_noalloc(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                             int32_t* kept_idx, int32_t* kept_cnt, void* cuda_stream);
+int sparkattn_select_noalloc_status(void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

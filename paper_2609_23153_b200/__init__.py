@@ -34,7 +34,8 @@ FP8_E4M3 = 1
 EXPORTS = (
     "sparkattn_version", "sparkattn_status_string", "sparkattn_workspace_bytes", "sparkattn_select",
     "sparkattn_quant_fp8", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
-    "sparkattn_attention_host",
+    "sparkattn_attention_host", "sparkattn_select_noalloc", "sparkattn_select_noalloc_max_bytes",
+    "sparkattn_select_noalloc_status",
 )
 
 
@@ -86,6 +87,11 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_arena_bytes.argtypes = [sp, i32, i32]
         L.sparkattn_attention_host.restype = ctypes.c_int
         L.sparkattn_attention_host.argtypes = [sp, i32, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+        L.sparkattn_select_noalloc.restype = ctypes.c_int
+        L.sparkattn_select_noalloc.argtypes = [sp, vp, vp, i32, vp, vp, vp]
+        L.sparkattn_select_noalloc_max_bytes.restype = sz
+        L.sparkattn_select_noalloc_status.restype = ctypes.c_int
+        L.sparkattn_select_noalloc_status.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -158,6 +164,20 @@ def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, *,
                                 _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     _check(rc, "sparkattn_select")
     return kept_idx, kept_cnt
+
+
+def select_noalloc(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, kept_idx: torch.Tensor,
+                   kept_cnt: Optional[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
+    """``sparkattn_select_noalloc``: same selection as :func:`select`, for callers that
+    must not allocate device memory at call time.  The caller passes the output
+    buffers; the scratch is a fixed 32 MiB array inside the library, shared by all
+    calls on the device (do not overlap calls; make the first call on a device
+    before any stream capture)."""
+    _same_layout(q, k)
+    shape = make_shape(q, block)
+    rc = lib().sparkattn_select_noalloc(ctypes.byref(shape), _ptr(q), _ptr(k), topk, _ptr(kept_idx), _ptr(kept_cnt),
+                                        _stream_ptr(stream))
+    _check(rc, "sparkattn_select_noalloc")
 
 
 def quant_fp8(x: torch.Tensor, block: int, *, codes: Optional[torch.Tensor] = None,
