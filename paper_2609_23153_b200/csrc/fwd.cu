@@ -6,16 +6,20 @@
 //
 // One CTA owns one (batch, head, query block) work item; two CTAs share an SM
 // so that one item's softmax overlaps the other's tensor-core work.
-//   warps 0-3  softmax: thread r owns query row r.  tcgen05.ld S from TMEM,
-//              fp32 online softmax (row max / row sum need no shuffles: a row
-//              lives in one thread), P written back to TMEM over S in the
-//              input precision, conditional rescale of O, final normalise and
-//              store.
+//   warps 0-3  softmax: thread r owns query row r.  One tcgen05.ld pass brings
+//              the whole S row into registers (this warpgroup raises its
+//              register budget, the other lowers its own), fp32 online softmax
+//              with packed fp32x2 FMA/ADD and 3-input max (row max / row sum
+//              need no shuffles: a row lives in one thread), P written back to
+//              TMEM over S in the input precision, conditional rescale of O,
+//              final normalise and store.
 //   warp 4     TMA producer: Q tile once, then K_j / V_j tiles of each kept
 //              block into one K slot and one V slot (128-byte swizzle).
 //   warp 5     MMA issuer: S = Q K_j^T (operands in shared memory) and
 //              O += P V_j (P from TMEM, V MN-major from shared memory) as
 //              tcgen05.mma with fp32 accumulators in TMEM.
+//   warps 6-7  idle; they complete the second warpgroup so that it can hand
+//              its registers to the softmax warpgroup.
 // TMEM columns: [0, BLK) S (P overlays its first BLK*elt/4 columns), [BLK, BLK+D) O.
 //
 // Every wait on an mbarrier is bounded (common.cuh); a kept index outside
@@ -28,7 +32,9 @@
 
 namespace sparkattn {
 
-constexpr int kFwdThreads = 192;
+constexpr int kFwdThreads = 256;          // warps 0-3 softmax, 4 TMA, 5 MMA, 6-7 idle (fill the warpgroup)
+constexpr int kSoftmaxRegs = 216;         // 128 * 216 + 128 * 40 = half of the SM's register file
+constexpr int kOtherRegs = 40;
 constexpr int kSoftmaxThreads = 128;
 // In log2 units: O and l are only rescaled when the running row maximum grows
 // by more than this; until then P may exceed 1 by at most 2^threshold, which
@@ -129,6 +135,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
   const uint32_t tmem_O = tmem + BLK;
   const bool dead = *s_abort != 0;
 
+  if (warp >= 4) {
+    reg_dec<kOtherRegs>();
+  }
   if (dead) {
     // nothing to do: fall through to the teardown
   } else if (warp == 4) {
@@ -200,8 +209,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         ++n;
       }
     }
-  } else {
+  } else if (warp < 4) {
     // ----------------------------------------------------------------- softmax
+    reg_inc<kSoftmaxRegs>();
     const int row = threadIdx.x;                      // query row inside the block = TMEM lane
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     const int q_row = qb * BLK + row;
@@ -234,20 +244,29 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       if (!ok) break;
       tc_fence_after();
 
-      // pass 1: row maximum of the raw accumulators
-      float mx = -INFINITY;
+      // the whole S row of this thread, one pass over TMEM
+      uint32_t sr[BLK];
 #pragma unroll
-      for (int ch = 0; ch < BLK / 32; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(tmem_S + lane_off + ch * 32, r);
-        tc_wait_ld();
+      for (int ch = 0; ch < BLK / 32; ++ch)
+        tmem_ld32(tmem_S + lane_off + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
+      tc_wait_ld();
+      if (ncols < BLK) {  // ragged last key block: keys >= N get weight 0
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float s = __uint_as_float(r[i]);
-          if (ch * 32 + i < ncols) mx = fmaxf(mx, s);
+        for (int i = 0; i < BLK; ++i)
+          if (i >= ncols) sr[i] = 0xff800000u;
+      }
+      float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+      float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
+#pragma unroll
+      for (int i = 4; i < BLK; i += 8) {
+        mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+        mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+        if (i + 4 < BLK) {
+          mx2 = fmax3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+          mx3 = fmax3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
         }
       }
-      const float m_new = mx * c;
+      const float m_new = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
       float alpha = 1.0f;
       bool need = false;
       if (n == 0) {
@@ -260,51 +279,61 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       if (__any_sync(0xffffffffu, need)) {
         // S_n complete implies O += P_{n-1} V_{n-1} complete: O is quiescent here.
         l *= alpha;
+        const uint64_t a2 = pack_f32x2(alpha, alpha);
 #pragma unroll
         for (int ch = 0; ch < D / 32; ++ch) {
           uint32_t r[32];
           tmem_ld32(tmem_O + lane_off + ch * 32, r);
           tc_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+          for (int i = 0; i < 32; i += 2) {
+            const float2 o2 = unpack_f32x2(fmul2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), a2));
+            r[i] = __float_as_uint(o2.x);
+            r[i + 1] = __float_as_uint(o2.y);
+          }
           tmem_st32(tmem_O + lane_off + ch * 32, r);
         }
       }
 
-      // pass 2: P = exp2(S*c - m) in the input precision, written over S
+      // P = exp2(S*c - m) in the input precision, written over S
       const float neg_m = p_off - m_used;
-      float l_tile = 0.0f;
+      const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
+      uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
+      constexpr int kWordsPerChunk = FP8 ? 8 : 16;   // P words produced from 32 S columns
+      uint32_t w[BLK / 32 * kWordsPerChunk];
 #pragma unroll
       for (int ch = 0; ch < BLK / 32; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(tmem_S + lane_off + ch * 32, r);
-        tc_wait_ld();
-        float pv[32];
+        float e[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float e = fast_exp2(fmaf(__uint_as_float(r[i]), c, neg_m));
-          pv[i] = (ch * 32 + i < ncols) ? e : 0.0f;
-          l_tile += pv[i];
+        for (int i = 0; i < 32; i += 2) {
+          const float2 x = unpack_f32x2(
+              ffma2(pack_f32x2(__uint_as_float(sr[ch * 32 + i]), __uint_as_float(sr[ch * 32 + i + 1])), c2, nm2));
+          e[i] = fast_exp2(x.x);
+          e[i + 1] = fast_exp2(x.y);
+          if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e[i], e[i + 1]));
+          else lsum0 = fadd2(lsum0, pack_f32x2(e[i], e[i + 1]));
         }
         if constexpr (FP8) {
-          uint32_t w[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(pv[4 * i], pv[4 * i + 1]), __NV_SATFINITE, __NV_E4M3);
-            const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(pv[4 * i + 2], pv[4 * i + 3]), __NV_SATFINITE, __NV_E4M3);
-            w[i] = lo | (hi << 16);
+            const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i], e[4 * i + 1]), __NV_SATFINITE, __NV_E4M3);
+            const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i + 2], e[4 * i + 3]), __NV_SATFINITE, __NV_E4M3);
+            w[ch * 8 + i] = lo | (hi << 16);
           }
-          tmem_st8(tmem_P + lane_off + ch * 8, w);
         } else {
-          uint32_t w[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[2 * i], pv[2 * i + 1]);
-            w[i] = *reinterpret_cast<const uint32_t*>(&h2);
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
+            w[ch * 16 + i] = *reinterpret_cast<const uint32_t*>(&h2);
           }
-          tmem_st16(tmem_P + lane_off + ch * 16, w);
         }
       }
+      constexpr int kPWords = BLK / 32 * kWordsPerChunk;   // = Cfg::kPCols
+#pragma unroll
+      for (int i = 0; i < kPWords / 32; ++i)
+        tmem_st32(tmem_P + lane_off + i * 32, *reinterpret_cast<const uint32_t(*)[32]>(&w[i * 32]));
+      const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
+      const float l_tile = ls.x + ls.y;
       if constexpr (FP8) l += l_tile * fast_exp2(-p_off);
       else l += l_tile;
       tc_wait_st();
@@ -336,14 +365,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
           if (row_valid) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              uint32_t w[4];
+              uint32_t ww[4];
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
                 const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[8 * i + 2 * j]) * inv,
                                                                 __uint_as_float(r[8 * i + 2 * j + 1]) * inv);
-                w[j] = *reinterpret_cast<const uint32_t*>(&h2);
+                ww[j] = *reinterpret_cast<const uint32_t*>(&h2);
               }
-              reinterpret_cast<uint4*>(orow + ch * 32)[i] = make_uint4(w[0], w[1], w[2], w[3]);
+              reinterpret_cast<uint4*>(orow + ch * 32)[i] = make_uint4(ww[0], ww[1], ww[2], ww[3]);
             }
           }
         }
