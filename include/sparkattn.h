@@ -123,7 +123,8 @@ int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint
  * dtype      : SPARKATTN_BF16: q,k,v bf16.  SPARKATTN_FP8_E4M3: q,k,v are E4M3
  *              codes from sparkattn_quant_fp8 with q_scale/k_scale/v_scale fp32
  *              [B,H,nb]; requires d = block = 128.  Scales are NULL for bf16.
- * kept_idx   : in, int32 [B,H,nb,kmax]; entries distinct, each in [0, nb)
+ * kept_idx   : in, int32 [B,H,nb,kmax]; entries distinct, each in [0, nb); kmax <= 2048
+ *              (longer lists return SPARKATTN_E_UNSUPPORTED_SHAPE)
  * kept_cnt   : in, int32 [B,H,nb] with 0 <= cnt <= kmax; NULL means cnt = kmax everywhere
  * out_bf16   : out, bf16 [B,H,N,d], same strides as q
  * lse        : out, fp32 [B,H,N] contiguous (natural log); may be NULL

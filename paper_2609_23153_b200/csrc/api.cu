@@ -92,6 +92,7 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
   if (dtype != SPARKATTN_BF16 && dtype != SPARKATTN_FP8_E4M3) return SPARKATTN_E_INVALID_ARG;
   if (!q || !k || !v || !kept_idx || !out_bf16 || !workspace) return SPARKATTN_E_INVALID_ARG;
   if (kmax < 1 || kmax > num_blocks(shape)) return SPARKATTN_E_INVALID_ARG;
+  if (kmax > kFwdMaxKept) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   if (dtype == SPARKATTN_FP8_E4M3) {
     if (!q_scale || !k_scale || !v_scale) return SPARKATTN_E_INVALID_ARG;
     if (!(shape->d == 128 && shape->block == 128)) return SPARKATTN_E_UNSUPPORTED_SHAPE;

@@ -132,6 +132,13 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
   return d;
 }
 
+// A descriptor from its two 32-bit words (the low word carries the start address and LBO).
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+
 // Instruction descriptor, dense, fp32 accumulate.  fmt: 0 = f16 / e4m3 (by
 // kind), 1 = bf16 / e5m2.  b_mn_major: B operand stored with N contiguous.
 __host__ __device__ constexpr uint32_t make_idesc(uint32_t fmt, uint32_t M, uint32_t N, bool b_mn_major) {

@@ -33,8 +33,8 @@
 namespace sparkattn {
 
 constexpr int kFwdThreads = 256;          // warps 0-3 softmax, 4 TMA, 5 MMA, 6-7 idle (fill the warpgroup)
-constexpr int kSoftmaxRegs = 216;         // 128 * 216 + 128 * 40 = half of the SM's register file
-constexpr int kOtherRegs = 40;
+constexpr int kSoftmaxRegs = 176;         // 128 * 176 + 128 * 80 = half of the SM's register file
+constexpr int kOtherRegs = 80;
 constexpr int kSoftmaxThreads = 128;
 // In log2 units: O and l are only rescaled when the running row maximum grows
 // by more than this; until then P may exceed 1 by at most 2^threshold, which
@@ -56,10 +56,11 @@ struct FwdCfg {
   static constexpr int kTileTxBytes = kSlabs * BLK * 128;  // bytes one Q / K / V load delivers
   static constexpr int kUmmaK = 32 / kElt;               // elements per MMA along K
   static constexpr int kQKSteps = 128 / 32;              // MMAs per slab for S
-  static constexpr int kPVSteps = BLK / kUmmaK;          // MMAs for O
-  static constexpr int kPCols = BLK * kElt / 4;
+  static constexpr int kHalf = BLK / 2;                  // keys per pipeline step (half a key block)
+  static constexpr int kPVSteps = kHalf / kUmmaK;        // MMAs for O per half
+  static constexpr int kListCap = kFwdMaxKept;           // kept-list entries staged in shared memory
   static constexpr int kTmemCols = (BLK + D) <= 128 ? 128 : 256;
-  static constexpr int kSmemBytes = 1024 /*align slack*/ + kQBytes + 2 * kKVBytes + 256 /*barriers*/;
+  static constexpr int kSmemBytes = 1024 /*align slack*/ + kQBytes + 2 * kKVBytes + 256 /*barriers*/ + kListCap * 4;
   static_assert(D * kElt % 128 == 0 && BLK % 32 == 0 && D % 32 == 0, "tile shape");
 };
 
@@ -82,6 +83,7 @@ __global__ void __launch_bounds__(kFwdThreads, 2)
 fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
            const __grid_constant__ CUtensorMap tmap_v, const FwdParams p) {
   using Cfg = FwdCfg<D, BLK, FP8>;
+  constexpr int HALF = Cfg::kHalf;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* sQ = smem;
@@ -91,27 +93,30 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
   uint64_t* bar_q_full = bars + 0;
   uint64_t* bar_k_full = bars + 1;
   uint64_t* bar_v_full = bars + 2;
-  uint64_t* bar_s_full = bars + 3;   // S_n complete (also: K slot free)
-  uint64_t* bar_p_full = bars + 4;   // P_n written by all softmax threads
-  uint64_t* bar_o_done = bars + 5;   // O += P_n V_n complete (also: V slot and S/P columns free)
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(bars + 8);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 9);
+  uint64_t* bar_s_full = bars + 3;    // [2] S half complete (half 1 also: K slot free)
+  uint64_t* bar_p_full = bars + 5;    // [2] P half written by all softmax threads
+  uint64_t* bar_pv_done = bars + 7;   // [2] O += P_half V_half complete (half 1 also: V slot free)
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 11);
+  int* s_ntiles = reinterpret_cast<int*>(bars + 12);
+  int32_t* s_list = reinterpret_cast<int32_t*>(bars + 32);   // [kListCap] validated kept block indices
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int qb = blockIdx.x % p.nb;
   const int bh = blockIdx.x / p.nb;
   const int h = bh % p.H, b = bh / p.H;
-  const int cnt = p.kept_cnt ? min(max(p.kept_cnt[(int64_t)bh * p.nb + qb], 0), p.kmax) : p.kmax;
-  const int32_t* list = p.kept_idx + ((int64_t)bh * p.nb + qb) * p.kmax;
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q_full, 1);
     mbar_init(bar_k_full, 1);
     mbar_init(bar_v_full, 1);
-    mbar_init(bar_s_full, 1);
-    mbar_init(bar_p_full, kSoftmaxThreads);
-    mbar_init(bar_o_done, 1);
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      mbar_init(bar_s_full + hf, 1);
+      mbar_init(bar_p_full + hf, kSoftmaxThreads);
+      mbar_init(bar_pv_done + hf, 1);
+    }
     // a timeout recorded by an earlier CTA of this launch makes the rest of the grid drain at once
     *s_abort = (*reinterpret_cast<volatile int32_t*>(p.status) == SPARKATTN_E_DEVICE_TIMEOUT) ? 1 : 0;
     mbar_fence_init();
@@ -125,15 +130,30 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
     __syncwarp();
     tmem_alloc(s_tmem_base, Cfg::kTmemCols);
     tmem_relinquish();
+  } else if (warp == 6) {
+    // Stage the kept list in shared memory, in order, dropping (and reporting) indices outside [0, nb).
+    const int cnt = p.kept_cnt ? min(max(__ldg(p.kept_cnt + (int64_t)bh * p.nb + qb), 0), p.kmax) : p.kmax;
+    const int32_t* list = p.kept_idx + ((int64_t)bh * p.nb + qb) * p.kmax;
+    int out = 0;
+    for (int base = 0; base < cnt; base += 32) {
+      const int t = base + lane;
+      const int kb = (t < cnt) ? __ldg(list + t) : 0;
+      const bool valid = (t < cnt) && kb >= 0 && kb < p.nb;
+      if (t < cnt && !valid) report_status(p.status, SPARKATTN_E_BAD_INDEX, kb);
+      const uint32_t ballot = __ballot_sync(0xffffffffu, valid);
+      if (valid) s_list[out + __popc(ballot & ((1u << lane) - 1u))] = kb;
+      out += __popc(ballot);
+    }
+    if (lane == 0) *s_ntiles = out;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem_base;
-  const uint32_t tmem_S = tmem;
-  const uint32_t tmem_P = tmem;
+  const uint32_t tmem_S = tmem;            // S half hf at columns [hf*HALF, (hf+1)*HALF); P half overlays its start
   const uint32_t tmem_O = tmem + BLK;
   const bool dead = *s_abort != 0;
+  const int ntiles = *s_ntiles;
 
   if (warp >= 4) {
     reg_dec<kOtherRegs>();
@@ -143,70 +163,90 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
   } else if (warp == 4) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int n = 0;
-      for (int t = 0; t < cnt; ++t) {
-        const int kb = __ldg(list + t);
-        if (kb < 0 || kb >= p.nb) continue;
+      for (int n = 0; n < ntiles; ++n) {
+        const int kb = s_list[n];
         if (n == 0) {
           mbar_expect_tx(bar_q_full, Cfg::kTileTxBytes);
 #pragma unroll
           for (int s = 0; s < Cfg::kSlabs; ++s)
             tma_load_4d(sQ + s * Cfg::kQSlabBytes, &tmap_q, bar_q_full, s * Cfg::kSlabElems, qb * BLK, h, b);
         } else {
-          if (!mbar_wait(bar_s_full, (n - 1) & 1, s_abort, p.status, 1)) break;  // K slot free
+          if (!mbar_wait(bar_s_full + 1, (n - 1) & 1, s_abort, p.status, 1)) break;  // K slot free
         }
         mbar_expect_tx(bar_k_full, Cfg::kTileTxBytes);
 #pragma unroll
         for (int s = 0; s < Cfg::kSlabs; ++s)
           tma_load_4d(sK + s * Cfg::kKVSlabBytes, &tmap_k, bar_k_full, s * Cfg::kSlabElems, kb * BLK, h, b);
         if (n > 0) {
-          if (!mbar_wait(bar_o_done, (n - 1) & 1, s_abort, p.status, 2)) break;  // V slot free
+          if (!mbar_wait(bar_pv_done + 1, (n - 1) & 1, s_abort, p.status, 2)) break;  // V slot free
         }
         mbar_expect_tx(bar_v_full, Cfg::kTileTxBytes);
 #pragma unroll
         for (int s = 0; s < Cfg::kSlabs; ++s)
           tma_load_4d(sV + s * Cfg::kKVSlabBytes, &tmap_v, bar_v_full, s * Cfg::kSlabElems, kb * BLK, h, b);
-        ++n;
       }
     }
   } else if (warp == 5) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    // Issue order (one thread; the tensor pipe executes in this order):
+    //   S_0(0) S_1(0) | PV_0(n) S_0(n+1) PV_1(n) S_1(n+1) | ...
+    // S_hf(n+1) overwrites the columns P_hf(n) lives in; it is issued right behind the PV that
+    // reads them, and the softmax threads have finished reading S_hf(n) before they signal P_hf(n).
+    if (lane == 0 && ntiles > 0) {
       constexpr uint32_t kFmt = FP8 ? 0u : 1u;
-      constexpr uint32_t idesc_qk = make_idesc(kFmt, 128, BLK, false);
+      constexpr uint32_t idesc_qk = make_idesc(kFmt, 128, HALF, false);
       constexpr uint32_t idesc_pv = make_idesc(kFmt, 128, D, true);
-      const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
-      int n = 0;
-      for (int t = 0; t < cnt; ++t) {
-        const int kb = __ldg(list + t);
-        if (kb < 0 || kb >= p.nb) continue;
-        if (n == 0) {
-          if (!mbar_wait(bar_q_full, 0, s_abort, p.status, 3)) break;
-        } else {
-          if (!mbar_wait(bar_o_done, (n - 1) & 1, s_abort, p.status, 4)) break;  // P_{n-1} consumed
-        }
-        if (!mbar_wait(bar_k_full, n & 1, s_abort, p.status, 5)) break;
-        tc_fence_after();
+      // Descriptors are built once; per MMA only the 32-bit low word moves (start address in 16-byte
+      // units), which keeps the single issuing thread far ahead of the tensor pipe.
+      const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ), 16);
+      const uint64_t dK = make_smem_desc_sw128(smem_u32(sK), 16);
+      const uint64_t dV = make_smem_desc_sw128(smem_u32(sV), Cfg::kKVSlabBytes);
+      const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32);
+      const uint32_t k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
+      const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
+      auto issue_s = [&](int hf) {
+        const uint32_t kh_lo = k_lo + ((hf * HALF * 128) >> 4);
 #pragma unroll
         for (int s = 0; s < Cfg::kSlabs; ++s) {
 #pragma unroll
           for (int kk = 0; kk < Cfg::kQKSteps; ++kk) {
-            const uint64_t da = make_smem_desc_sw128(aQ + s * Cfg::kQSlabBytes + kk * 32, 16);
-            const uint64_t db = make_smem_desc_sw128(aK + s * Cfg::kKVSlabBytes + kk * 32, 16);
-            mma_ss<FP8>(tmem_S, da, db, idesc_qk, (s | kk) != 0);
+            const uint64_t da = make_desc(q_lo + ((s * Cfg::kQSlabBytes + kk * 32) >> 4), q_hi);
+            const uint64_t db = make_desc(kh_lo + ((s * Cfg::kKVSlabBytes + kk * 32) >> 4), k_hi);
+            mma_ss<FP8>(tmem_S + hf * HALF, da, db, idesc_qk, (s | kk) != 0 ? 1u : 0u);
           }
         }
-        tc_commit(bar_s_full);
-        if (!mbar_wait(bar_v_full, n & 1, s_abort, p.status, 6)) break;
-        if (!mbar_wait(bar_p_full, n & 1, s_abort, p.status, 7)) break;
-        tc_fence_after();
+        tc_commit(bar_s_full + hf);
+      };
+      auto issue_pv = [&](int hf, bool first) {
+        const uint32_t vh_lo = v_lo + ((hf * HALF * 128) >> 4);
 #pragma unroll
         for (int kk = 0; kk < Cfg::kPVSteps; ++kk) {
-          const uint64_t db = make_smem_desc_sw128(aV + kk * Cfg::kUmmaK * 128, Cfg::kKVSlabBytes);
-          mma_ts<FP8>(tmem_O, tmem_P + kk * 8, db, idesc_pv, (n | kk) != 0);
+          const uint64_t db = make_desc(vh_lo + ((kk * Cfg::kUmmaK * 128) >> 4), v_hi);
+          mma_ts<FP8>(tmem_O, tmem_S + hf * HALF + kk * 8, db, idesc_pv, (first && kk == 0) ? 0u : 1u);
         }
-        tc_commit(bar_o_done);
-        ++n;
+        tc_commit(bar_pv_done + hf);
+      };
+      bool ok = mbar_wait(bar_q_full, 0, s_abort, p.status, 3) && mbar_wait(bar_k_full, 0, s_abort, p.status, 5);
+      if (ok) {
+        tc_fence_after();
+        issue_s(0);
+        issue_s(1);
+      }
+      for (int n = 0; ok && n < ntiles; ++n) {
+        const bool more = n + 1 < ntiles;
+        if (!(ok = mbar_wait(bar_v_full, n & 1, s_abort, p.status, 6))) break;
+        if (!(ok = mbar_wait(bar_p_full + 0, n & 1, s_abort, p.status, 7))) break;
+        tc_fence_after();
+        issue_pv(0, n == 0);
+        if (more) {
+          if (!(ok = mbar_wait(bar_k_full, (n + 1) & 1, s_abort, p.status, 5))) break;
+          tc_fence_after();
+          issue_s(0);
+        }
+        if (!(ok = mbar_wait(bar_p_full + 1, n & 1, s_abort, p.status, 7))) break;
+        tc_fence_after();
+        issue_pv(1, false);
+        if (more) issue_s(1);
       }
     }
   } else if (warp < 4) {
@@ -224,14 +264,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       for (int j = 0; j < p.nb; ++j) vm = fmaxf(vm, __ldg(p.v_scale + (int64_t)bh * p.nb + j));
       v_max = vm;
     }
-    int n = 0;
     bool ok = true;
-    for (int t = 0; t < cnt; ++t) {
-      const int kb = __ldg(list + t);
-      if (kb < 0 || kb >= p.nb) {
-        if (threadIdx.x == 0) report_status(p.status, SPARKATTN_E_BAD_INDEX, kb);
-        continue;
-      }
+    for (int n = 0; ok && n < ntiles; ++n) {
+      const int kb = s_list[n];
       const int ncols = min(BLK, p.N - kb * BLK);    // valid keys in this block
       float c = p.scale_log2;                        // logit -> log2 units
       float p_off = 0.0f;                            // log2 of the factor folded into P
@@ -239,119 +274,130 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         c *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb);
         p_off = kFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb) / v_max);
       }
-      ok = mbar_wait(bar_s_full, n & 1, s_abort, p.status, 8);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int nc = ncols - hf * HALF;            // valid keys in this half (may be <= 0)
+        ok = mbar_wait(bar_s_full + hf, n & 1, s_abort, p.status, 8);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
 
-      // the whole S row of this thread, one pass over TMEM
-      uint32_t sr[BLK];
+        // this thread's half row of S, one pass over TMEM
+        uint32_t sr[HALF];
 #pragma unroll
-      for (int ch = 0; ch < BLK / 32; ++ch)
-        tmem_ld32(tmem_S + lane_off + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
-      tc_wait_ld();
-      if (ncols < BLK) {  // ragged last key block: keys >= N get weight 0
+        for (int ch = 0; ch < HALF / 32; ++ch)
+          tmem_ld32(tmem_S + lane_off + hf * HALF + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
+        tc_wait_ld();
+        if (nc < HALF) {  // ragged last key block: keys >= N get weight 0
 #pragma unroll
-        for (int i = 0; i < BLK; ++i)
-          if (i >= ncols) sr[i] = 0xff800000u;
-      }
-      float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
-      float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
-#pragma unroll
-      for (int i = 4; i < BLK; i += 8) {
-        mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
-        mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
-        if (i + 4 < BLK) {
-          mx2 = fmax3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
-          mx3 = fmax3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
+          for (int i = 0; i < HALF; ++i)
+            if (i >= nc) sr[i] = 0xff800000u;
         }
-      }
-      const float m_new = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
-      float alpha = 1.0f;
-      bool need = false;
-      if (n == 0) {
-        m_used = m_new;
-      } else if (m_new > m_used + (FP8 ? 0.0f : kLazyRescaleLog2)) {
-        alpha = fast_exp2(m_used - m_new);
-        m_used = m_new;
-        need = true;
-      }
-      if (__any_sync(0xffffffffu, need)) {
-        // S_n complete implies O += P_{n-1} V_{n-1} complete: O is quiescent here.
-        l *= alpha;
-        const uint64_t a2 = pack_f32x2(alpha, alpha);
+        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+        float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
 #pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
-          uint32_t r[32];
-          tmem_ld32(tmem_O + lane_off + ch * 32, r);
-          tc_wait_ld();
+        for (int i = 4; i < HALF; i += 8) {
+          mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+          mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+          if (i + 4 < HALF) {
+            mx2 = fmax3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+            mx3 = fmax3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
+          }
+        }
+        const float m_new = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
+        float alpha = 1.0f;
+        bool need = false;
+        if (n == 0 && hf == 0) {
+          m_used = m_new;
+        } else if (m_new > m_used + (FP8 ? 0.0f : kLazyRescaleLog2)) {
+          alpha = fast_exp2(m_used - m_new);
+          m_used = m_new;
+          need = true;
+        }
+        if (__any_sync(0xffffffffu, need)) {
+          // O must be quiescent: the last PV issued before this point is the other half's
+          // (previous tile's second half, or this tile's first half).
+          const int prev_hf = hf ^ 1;
+          const int prev_n = hf == 0 ? n - 1 : n;
+          ok = mbar_wait(bar_pv_done + prev_hf, prev_n & 1, s_abort, p.status, 10);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          l *= alpha;
+          const uint64_t a2 = pack_f32x2(alpha, alpha);
+#pragma unroll
+          for (int ch = 0; ch < D / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_O + lane_off + ch * 32, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float2 o2 = unpack_f32x2(fmul2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), a2));
+              r[i] = __float_as_uint(o2.x);
+              r[i + 1] = __float_as_uint(o2.y);
+            }
+            tmem_st32(tmem_O + lane_off + ch * 32, r);
+          }
+        }
+
+        // P = exp2(S*c - m) in the input precision, written over the start of this S half
+        const float neg_m = p_off - m_used;
+        const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
+        uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
+        constexpr int kWordsPerChunk = FP8 ? 8 : 16;   // P words produced from 32 S columns
+        constexpr int kHalfWords = HALF / 32 * kWordsPerChunk;
+        uint32_t w[kHalfWords];
+#pragma unroll
+        for (int ch = 0; ch < HALF / 32; ++ch) {
+          float e[32];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            const float2 o2 = unpack_f32x2(fmul2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), a2));
-            r[i] = __float_as_uint(o2.x);
-            r[i + 1] = __float_as_uint(o2.y);
+            const float2 x = unpack_f32x2(
+                ffma2(pack_f32x2(__uint_as_float(sr[ch * 32 + i]), __uint_as_float(sr[ch * 32 + i + 1])), c2, nm2));
+            e[i] = fast_exp2(x.x);
+            e[i + 1] = fast_exp2(x.y);
+            if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e[i], e[i + 1]));
+            else lsum0 = fadd2(lsum0, pack_f32x2(e[i], e[i + 1]));
           }
-          tmem_st32(tmem_O + lane_off + ch * 32, r);
+          if constexpr (FP8) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i], e[4 * i + 1]), __NV_SATFINITE, __NV_E4M3);
+              const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i + 2], e[4 * i + 3]), __NV_SATFINITE, __NV_E4M3);
+              w[ch * 8 + i] = lo | (hi << 16);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
+              w[ch * 16 + i] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+          }
         }
+        static_assert(kHalfWords == 32 || kHalfWords == 16 || kHalfWords == 8, "P half width");
+        if constexpr (kHalfWords == 32) tmem_st32(tmem_S + lane_off + hf * HALF, *reinterpret_cast<const uint32_t(*)[32]>(&w[0]));
+        else if constexpr (kHalfWords == 16) tmem_st16(tmem_S + lane_off + hf * HALF, w);
+        else tmem_st8(tmem_S + lane_off + hf * HALF, w);
+        const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
+        const float l_tile = ls.x + ls.y;
+        if constexpr (FP8) l += l_tile * fast_exp2(-p_off);
+        else l += l_tile;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p_full + hf);
       }
-
-      // P = exp2(S*c - m) in the input precision, written over S
-      const float neg_m = p_off - m_used;
-      const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
-      uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
-      constexpr int kWordsPerChunk = FP8 ? 8 : 16;   // P words produced from 32 S columns
-      uint32_t w[BLK / 32 * kWordsPerChunk];
-#pragma unroll
-      for (int ch = 0; ch < BLK / 32; ++ch) {
-        float e[32];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float2 x = unpack_f32x2(
-              ffma2(pack_f32x2(__uint_as_float(sr[ch * 32 + i]), __uint_as_float(sr[ch * 32 + i + 1])), c2, nm2));
-          e[i] = fast_exp2(x.x);
-          e[i + 1] = fast_exp2(x.y);
-          if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e[i], e[i + 1]));
-          else lsum0 = fadd2(lsum0, pack_f32x2(e[i], e[i + 1]));
-        }
-        if constexpr (FP8) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i], e[4 * i + 1]), __NV_SATFINITE, __NV_E4M3);
-            const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i + 2], e[4 * i + 3]), __NV_SATFINITE, __NV_E4M3);
-            w[ch * 8 + i] = lo | (hi << 16);
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
-            w[ch * 16 + i] = *reinterpret_cast<const uint32_t*>(&h2);
-          }
-        }
-      }
-      constexpr int kPWords = BLK / 32 * kWordsPerChunk;   // = Cfg::kPCols
-#pragma unroll
-      for (int i = 0; i < kPWords / 32; ++i)
-        tmem_st32(tmem_P + lane_off + i * 32, *reinterpret_cast<const uint32_t(*)[32]>(&w[i * 32]));
-      const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
-      const float l_tile = ls.x + ls.y;
-      if constexpr (FP8) l += l_tile * fast_exp2(-p_off);
-      else l += l_tile;
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(bar_p_full);
-      ++n;
     }
 
     // ---------------------------------------------------------------- epilogue
     __nv_bfloat16* orow = p.out + b * p.stride_b + h * p.stride_h + (int64_t)q_row * p.stride_n;
-    if (n == 0 || !ok) {
+    if (ntiles == 0 || !ok) {
       if (row_valid && ok) {
 #pragma unroll
         for (int ch = 0; ch < D / 8; ++ch) reinterpret_cast<uint4*>(orow)[ch] = make_uint4(0u, 0u, 0u, 0u);
         if (p.lse) p.lse[(int64_t)bh * p.N + q_row] = -INFINITY;
       }
     } else {
-      ok = mbar_wait(bar_o_done, (n - 1) & 1, s_abort, p.status, 9);
+      ok = mbar_wait(bar_pv_done + 1, (ntiles - 1) & 1, s_abort, p.status, 9);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();

@@ -21,6 +21,7 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
                   int32_t* kept_cnt, void* workspace, cudaStream_t stream);
 
 // fwd.cu
+constexpr int kFwdMaxKept = 2048;  // longest kept list (kmax) the forward kernel stages in shared memory
 size_t fwd_workspace_bytes(const sparkattn_shape_t& s);
 int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void* k, const void* v,
                const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
