@@ -57,6 +57,10 @@ struct FwdCfg {
   static constexpr int kUmmaK = 32 / kElt;               // elements per MMA along K
   static constexpr int kQKSteps = 128 / 32;              // MMAs per slab for S
   static constexpr int kHalf = BLK / 2;                  // keys per pipeline step (half a key block)
+  // S = Q K^T per half (N = BLK/2: lets S of the next tile start early, but each MMA is bound by
+  // the shared-memory operand fetch) or per tile (N = BLK: full tensor rate).  Measured on B200:
+  // the split wins when the MMAs are short (FP8), the full width when they are long (bf16).
+  static constexpr bool kSplitS = FP8;
   static constexpr int kPVSteps = kHalf / kUmmaK;        // MMAs for O per half
   static constexpr int kListCap = kFwdMaxKept;           // kept-list entries staged in shared memory
   static constexpr int kTmemCols = (BLK + D) <= 128 ? 128 : 256;
@@ -189,12 +193,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
   } else if (warp == 5) {
     // -------------------------------------------------------------- MMA issuer
     // Issue order (one thread; the tensor pipe executes in this order):
-    //   S_0(0) S_1(0) | PV_0(n) S_0(n+1) PV_1(n) S_1(n+1) | ...
-    // S_hf(n+1) overwrites the columns P_hf(n) lives in; it is issued right behind the PV that
-    // reads them, and the softmax threads have finished reading S_hf(n) before they signal P_hf(n).
+    //   split S:  S_0(0) S_1(0) | PV_0(n) S_0(n+1) PV_1(n) S_1(n+1) | ...
+    //   full S:   S(0)          | PV_0(n) PV_1(n) S(n+1)            | ...
+    // S(n+1) overwrites the columns P(n) lives in; it is issued right behind the PV that reads
+    // them, and the softmax threads have finished reading S(n) before they signal P(n).
     if (lane == 0 && ntiles > 0) {
       constexpr uint32_t kFmt = FP8 ? 0u : 1u;
-      constexpr uint32_t idesc_qk = make_idesc(kFmt, 128, HALF, false);
+      constexpr bool kSplitS = Cfg::kSplitS;
+      constexpr uint32_t idesc_qk = make_idesc(kFmt, 128, kSplitS ? HALF : BLK, false);
       constexpr uint32_t idesc_pv = make_idesc(kFmt, 128, D, true);
       // Descriptors are built once; per MMA only the 32-bit low word moves (start address in 16-byte
       // units), which keeps the single issuing thread far ahead of the tensor pipe.
@@ -204,6 +210,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32);
       const uint32_t k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
       const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
+      // S for half hf (split mode: N = HALF, one commit) or for the whole tile (N = BLK, hf = 0,
+      // both halves' barriers signalled).
       auto issue_s = [&](int hf) {
         const uint32_t kh_lo = k_lo + ((hf * HALF * 128) >> 4);
 #pragma unroll
@@ -216,6 +224,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
           }
         }
         tc_commit(bar_s_full + hf);
+        if constexpr (!kSplitS) tc_commit(bar_s_full + 1);
       };
       auto issue_pv = [&](int hf, bool first) {
         const uint32_t vh_lo = v_lo + ((hf * HALF * 128) >> 4);
@@ -230,7 +239,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       if (ok) {
         tc_fence_after();
         issue_s(0);
-        issue_s(1);
+        if constexpr (kSplitS) issue_s(1);
       }
       for (int n = 0; ok && n < ntiles; ++n) {
         const bool more = n + 1 < ntiles;
@@ -238,15 +247,25 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         if (!(ok = mbar_wait(bar_p_full + 0, n & 1, s_abort, p.status, 7))) break;
         tc_fence_after();
         issue_pv(0, n == 0);
-        if (more) {
-          if (!(ok = mbar_wait(bar_k_full, (n + 1) & 1, s_abort, p.status, 5))) break;
-          tc_fence_after();
-          issue_s(0);
+        if constexpr (kSplitS) {
+          if (more) {
+            if (!(ok = mbar_wait(bar_k_full, (n + 1) & 1, s_abort, p.status, 5))) break;
+            tc_fence_after();
+            issue_s(0);
+          }
         }
         if (!(ok = mbar_wait(bar_p_full + 1, n & 1, s_abort, p.status, 7))) break;
         tc_fence_after();
         issue_pv(1, false);
-        if (more) issue_s(1);
+        if (more) {
+          if constexpr (kSplitS) {
+            issue_s(1);
+          } else {
+            if (!(ok = mbar_wait(bar_k_full, (n + 1) & 1, s_abort, p.status, 5))) break;
+            tc_fence_after();
+            issue_s(0);
+          }
+        }
       }
     }
   } else if (warp < 4) {
