@@ -40,9 +40,9 @@ import workloads  # noqa: E402
 
 METRIC = "block-sparse attn effective TFLOP/s (kept FLOPs), select+fwd, 97% sparse"
 UNIT = "TFLOP/s"
-# DRAM bytes (read + write) of one forward launch on the bench workload, from the
-# ncu capture summarised in profiles/fwd_bf16_wan14b_s97.md (null until captured).
-FWD_DRAM_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) of one bf16 forward launch on the default workload (wan14b, 97 %),
+# from the one-pass ncu capture summarised in profiles/launch_list_wan14b_s97.md.
+FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2404592384 + 760947712}
 
 
 def load_peaks():
@@ -124,26 +124,27 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------- CPU oracle legs
 
-def cpu_oracle_sample(w, target_seconds: float, head: int = 0):
-    """Times the CPU oracle (selection of one head in full + attention on a sample of
-    that head's query blocks) and returns kept-FLOP throughput of the sample."""
+def cpu_oracle_sample(w, target_seconds: float, nheads: int = 4):
+    """Times the CPU oracle (selection of `nheads` heads in full + attention on a sample of
+    those heads' query blocks) and returns kept-FLOP throughput of the sample."""
     import oracle
     cores = oracle.num_threads()
-    w1 = w.with_heads(1)
-    q, k, v = workloads.structured_qkv(w, heads=[head], device="cpu")
+    nheads = min(nheads, w.H)
+    w1 = w.with_heads(nheads)
+    q, k, v = workloads.structured_qkv(w, heads=list(range(nheads)), device="cpu")
     q, k, v = q[0], k[0], v[0]
     t0 = time.perf_counter()
     idx, cnt = oracle.select(q, k, w.block, w.topk)
     t_sel = time.perf_counter() - t0
     # calibrate on one batch of `cores` items, then size the sample for the time target
     g = torch.Generator().manual_seed(1234)
-    order = torch.randperm(w.nb, generator=g).tolist()
-    first = [(0, i) for i in order[:cores]]
+    order = [(int(x) // w.nb, int(x) % w.nb) for x in torch.randperm(nheads * w.nb, generator=g)]
+    first = order[:cores]
     t0 = time.perf_counter()
     oracle.attention(q, k, v, idx, cnt, w.block, items=first)
     t_first = time.perf_counter() - t0
-    n_more = int(max(0, min(w.nb - cores, (target_seconds - t_first - t_sel) / max(t_first, 1e-6) * cores)))
-    rest = [(0, i) for i in order[cores:cores + n_more]]
+    n_more = int(max(0, min(len(order) - cores, (target_seconds - t_first - t_sel) / max(t_first, 1e-6) * cores)))
+    rest = order[cores:cores + n_more]
     t_rest = 0.0
     if rest:
         t0 = time.perf_counter()
@@ -151,10 +152,10 @@ def cpu_oracle_sample(w, target_seconds: float, head: int = 0):
         t_rest = time.perf_counter() - t0
     items = first + rest
     flops = kept_flops(w1, idx, cnt, items)
-    t_total = t_first + t_rest + t_sel * len(items) / w.nb
+    t_total = t_first + t_rest + t_sel * len(items) / (nheads * w.nb)
     return {"value": flops / t_total / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": (f"head {head} of {w.name}: oracle selection of the whole head ({t_sel:.2f} s, charged pro rata) + fp64 "
-                       f"oracle attention on {len(items)} of {w.nb} query blocks ({t_first + t_rest:.2f} s)"),
+            "sample": (f"heads 0-{nheads - 1} of {w.name}: oracle selection of those heads ({t_sel:.2f} s, charged pro rata) + "
+                       f"fp64 oracle attention on {len(items)} of their {nheads * w.nb} query blocks ({t_first + t_rest:.2f} s)"),
             "seconds": t_total, "items": len(items)}
 
 
@@ -305,7 +306,7 @@ def run_ours(args, w):
         "fwd_bf16": {"ms": ms_fwd, "launches_per_step": 1, "TFLOPs": fwd_tflops},
     }
     roofline = {"kernel": "fwd_kernel<128,128,bf16>", "bound": "tensor", "achieved": fwd_tflops, "peak": peaks["bf16"],
-                "unit": "TFLOP/s", "frac": fwd_tflops / peaks["bf16"], "traffic": FWD_DRAM_TRAFFIC_BYTES,
+                "unit": "TFLOP/s", "frac": fwd_tflops / peaks["bf16"], "traffic": FWD_DRAM_TRAFFIC_BYTES.get(w.name) if w.sparsity == 0.97 else None,
                 "peak_source": f"{peaks['source']} bf16 burst (sustained {peaks['bf16_sustained']})",
                 "flops_per_launch": flops, "ms_per_launch": ms_fwd}
 
