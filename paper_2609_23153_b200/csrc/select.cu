@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
             int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* s_pq = reinterpret_cast<float*>(smem_raw);                          // [kRowsPerCta][D]
+  float* s_pq = reinterpret_cast<float*>(smem_raw);                          // [kRowsPerCta][D], 16-byte aligned
   uint32_t* s_key = reinterpret_cast<uint32_t*>(s_pq + kRowsPerCta * D);     // [kRowsPerCta][nbp]
 
   const int64_t bh = blockIdx.x / groups_per_bh;
@@ -118,20 +118,49 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
   }
   __syncthreads();
 
-  // scores: thread j walks the channels in ascending order for 8 query blocks at once
+  // scores: a thread owns up to kJT key blocks (j, j + 256, j + 512) and walks the channels in
+  // ascending order for the CTA's 8 query blocks at once; pooled Q comes from shared memory as
+  // broadcast 16-byte loads, pooled K from L2 coalesced along j.
   const float* kcol = pkT + bh * D * (int64_t)nbp;
-  for (int j = threadIdx.x; j < nb; j += kTopkThreads) {
-    float acc[kRowsPerCta];
+  const float4* s_pq4 = reinterpret_cast<const float4*>(s_pq);
+  constexpr int kJT = 3;
+  for (int j0 = threadIdx.x; j0 < nb; j0 += kTopkThreads * kJT) {
+    int jcl[kJT];
 #pragma unroll
-    for (int r = 0; r < kRowsPerCta; ++r) acc[r] = 0.0f;
-#pragma unroll 4
-    for (int c = 0; c < D; ++c) {
-      const float kv = __ldg(kcol + (int64_t)c * nbp + j);
+    for (int u = 0; u < kJT; ++u) jcl[u] = min(j0 + u * kTopkThreads, nb - 1);  // clamped: loads stay in range
+    float acc[kJT][kRowsPerCta];
 #pragma unroll
-      for (int r = 0; r < kRowsPerCta; ++r) acc[r] = __fmaf_rn(s_pq[r * D + c], kv, acc[r]);
+    for (int u = 0; u < kJT; ++u)
+#pragma unroll
+      for (int r = 0; r < kRowsPerCta; ++r) acc[u][r] = 0.0f;
+#pragma unroll 2
+    for (int c4 = 0; c4 < D / 4; ++c4) {
+      float4 qv[kRowsPerCta];
+#pragma unroll
+      for (int r = 0; r < kRowsPerCta; ++r) qv[r] = s_pq4[r * (D / 4) + c4];
+#pragma unroll
+      for (int u = 0; u < kJT; ++u) {
+        const float* kp = kcol + (int64_t)(4 * c4) * nbp + jcl[u];
+        const float k0 = __ldg(kp), k1 = __ldg(kp + nbp), k2 = __ldg(kp + 2 * nbp), k3 = __ldg(kp + 3 * nbp);
+#pragma unroll
+        for (int r = 0; r < kRowsPerCta; ++r) {
+          float a = acc[u][r];
+          a = __fmaf_rn(qv[r].x, k0, a);
+          a = __fmaf_rn(qv[r].y, k1, a);
+          a = __fmaf_rn(qv[r].z, k2, a);
+          a = __fmaf_rn(qv[r].w, k3, a);
+          acc[u][r] = a;
+        }
+      }
     }
 #pragma unroll
-    for (int r = 0; r < kRowsPerCta; ++r) s_key[r * nbp + j] = score_key(acc[r]);
+    for (int u = 0; u < kJT; ++u) {
+      const int j = j0 + u * kTopkThreads;
+      if (j < nb) {
+#pragma unroll
+        for (int r = 0; r < kRowsPerCta; ++r) s_key[r * nbp + j] = score_key(acc[u][r]);
+      }
+    }
   }
   __syncthreads();
 
@@ -139,9 +168,20 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
   if (warp >= nrows) return;
   const uint32_t* key = s_key + warp * nbp;
 
-  // exact value of the topk-th largest key, one bit per pass from the top
-  uint32_t thr = 0;
-  for (int bit = 31; bit >= 0; --bit) {
+  // exact value of the topk-th largest key, one bit per pass from the top; bits above the
+  // highest bit in which the row's keys differ are common to all keys and need no pass
+  uint32_t kmin = 0xffffffffu, kmaxv = 0u;
+  for (int j = lane; j < nb; j += 32) {
+    kmin = min(kmin, key[j]);
+    kmaxv = max(kmaxv, key[j]);
+  }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmaxv = __reduce_max_sync(0xffffffffu, kmaxv);
+  const uint32_t diff = kmin ^ kmaxv;
+  const int top_bit = 31 - __clz(diff);                       // -1 when all keys are equal
+  uint32_t thr = (top_bit >= 31) ? 0u : (kmaxv & ~((2u << max(top_bit, 0)) - 1u));
+  if (top_bit < 0) thr = kmaxv;
+  for (int bit = top_bit; bit >= 0; --bit) {
     const uint32_t cand = thr | (1u << bit);
     int cnt = 0;
     for (int j = lane; j < nb; j += 32) cnt += (key[j] >= cand);
