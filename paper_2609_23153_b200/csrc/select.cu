@@ -13,17 +13,18 @@
 //                  from HBM (the only HBM-heavy step: 2 bytes per element) and
 //                  writes pooled Q [BH][nb][d] and pooled K transposed [BH][d][nbp].
 //   topk_kernel    one CTA per 8 query blocks of one (batch, head): scores against
-//                  all key blocks (pooled K streamed from L2, coalesced along j),
-//                  then one warp per query block does an exact radix select of the
-//                  topk-th largest key and an ordered ballot compaction.
+//                  all key blocks (pooled K streamed from L2, coalesced along j,
+//                  packed fp32x2 FMAs over row pairs), then one warp per query
+//                  block does an exact radix select of the topk-th largest key
+//                  (keys in registers for nb <= 768) and an ordered ballot compaction.
 #include "common.cuh"
 #include "launch.h"
 
 namespace sparkattn {
 
 constexpr int kPoolThreads = 256;
-constexpr int kTopkThreads = 256;
-constexpr int kRowsPerCta = kTopkThreads / 32;  // query blocks per CTA, one warp each
+constexpr int kTopkThreads = 320;  // 2 x 320 key-block slots per sweep (591 blocks of the 720P shape fit one sweep)
+constexpr int kRowsPerCta = 8;     // query blocks per CTA; warps 0-7 select one row each
 
 static inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
@@ -100,106 +101,41 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
-            int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* s_pq = reinterpret_cast<float*>(smem_raw);                          // [kRowsPerCta][D], 16-byte aligned
-  uint32_t* s_key = reinterpret_cast<uint32_t*>(s_pq + kRowsPerCta * D);     // [kRowsPerCta][nbp]
-
-  const int64_t bh = blockIdx.x / groups_per_bh;
-  const int i0 = (blockIdx.x % groups_per_bh) * kRowsPerCta;
-  const int nrows = min(kRowsPerCta, nb - i0);
-
-  for (int e = threadIdx.x; e < kRowsPerCta * D; e += kTopkThreads) {
-    const int r = e / D;
-    s_pq[e] = (r < nrows) ? pq[(bh * nb + i0 + r) * D + (e % D)] : 0.0f;
-  }
-  __syncthreads();
-
-  // scores: a thread owns up to kJT key blocks (j, j + 256, j + 512) and walks the channels in
-  // ascending order for the CTA's 8 query blocks at once; pooled Q comes from shared memory as
-  // broadcast 16-byte loads, pooled K from L2 coalesced along j.
-  const float* kcol = pkT + bh * D * (int64_t)nbp;
-  const float4* s_pq4 = reinterpret_cast<const float4*>(s_pq);
-  constexpr int kJT = 3;
-  for (int j0 = threadIdx.x; j0 < nb; j0 += kTopkThreads * kJT) {
-    int jcl[kJT];
-#pragma unroll
-    for (int u = 0; u < kJT; ++u) jcl[u] = min(j0 + u * kTopkThreads, nb - 1);  // clamped: loads stay in range
-    float acc[kJT][kRowsPerCta];
-#pragma unroll
-    for (int u = 0; u < kJT; ++u)
-#pragma unroll
-      for (int r = 0; r < kRowsPerCta; ++r) acc[u][r] = 0.0f;
-#pragma unroll 2
-    for (int c4 = 0; c4 < D / 4; ++c4) {
-      float4 qv[kRowsPerCta];
-#pragma unroll
-      for (int r = 0; r < kRowsPerCta; ++r) qv[r] = s_pq4[r * (D / 4) + c4];
-#pragma unroll
-      for (int u = 0; u < kJT; ++u) {
-        const float* kp = kcol + (int64_t)(4 * c4) * nbp + jcl[u];
-        const float k0 = __ldg(kp), k1 = __ldg(kp + nbp), k2 = __ldg(kp + 2 * nbp), k3 = __ldg(kp + 3 * nbp);
-#pragma unroll
-        for (int r = 0; r < kRowsPerCta; ++r) {
-          float a = acc[u][r];
-          a = __fmaf_rn(qv[r].x, k0, a);
-          a = __fmaf_rn(qv[r].y, k1, a);
-          a = __fmaf_rn(qv[r].z, k2, a);
-          a = __fmaf_rn(qv[r].w, k3, a);
-          acc[u][r] = a;
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kJT; ++u) {
-      const int j = j0 + u * kTopkThreads;
-      if (j < nb) {
-#pragma unroll
-        for (int r = 0; r < kRowsPerCta; ++r) s_key[r * nbp + j] = score_key(acc[u][r]);
-      }
-    }
-  }
-  __syncthreads();
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp >= nrows) return;
-  const uint32_t* key = s_key + warp * nbp;
-
-  // exact value of the topk-th largest key, one bit per pass from the top; bits above the
-  // highest bit in which the row's keys differ are common to all keys and need no pass
+// Exact selection of the topk largest keys of one row by one warp (ties: lowest index first),
+// written in ascending index order.  KeyAt(j) returns key j; the keys are visited several times.
+template <typename KeyAt>
+__device__ __forceinline__ void select_row(KeyAt key_at, int nb, int topk, int lane, int32_t* __restrict__ dst) {
+  // value of the topk-th largest key, one bit per pass from the top; bits above the highest bit in
+  // which the row's keys differ are common to all keys and need no pass
   uint32_t kmin = 0xffffffffu, kmaxv = 0u;
   for (int j = lane; j < nb; j += 32) {
-    kmin = min(kmin, key[j]);
-    kmaxv = max(kmaxv, key[j]);
+    const uint32_t kj = key_at(j);
+    kmin = min(kmin, kj);
+    kmaxv = max(kmaxv, kj);
   }
   kmin = __reduce_min_sync(0xffffffffu, kmin);
   kmaxv = __reduce_max_sync(0xffffffffu, kmaxv);
-  const uint32_t diff = kmin ^ kmaxv;
-  const int top_bit = 31 - __clz(diff);                       // -1 when all keys are equal
+  const int top_bit = 31 - __clz(kmin ^ kmaxv);              // -1 when all keys are equal
   uint32_t thr = (top_bit >= 31) ? 0u : (kmaxv & ~((2u << max(top_bit, 0)) - 1u));
   if (top_bit < 0) thr = kmaxv;
   for (int bit = top_bit; bit >= 0; --bit) {
     const uint32_t cand = thr | (1u << bit);
     int cnt = 0;
-    for (int j = lane; j < nb; j += 32) cnt += (key[j] >= cand);
+    for (int j = lane; j < nb; j += 32) cnt += (key_at(j) >= cand);
     cnt = __reduce_add_sync(0xffffffffu, cnt);
     if (cnt >= topk) thr = cand;
   }
   int ngreater = 0;
-  for (int j = lane; j < nb; j += 32) ngreater += (key[j] > thr);
+  for (int j = lane; j < nb; j += 32) ngreater += (key_at(j) > thr);
   ngreater = __reduce_add_sync(0xffffffffu, ngreater);
   const int ties_allowed = topk - ngreater;  // >= 1: lowest indices among the keys equal to thr
 
-  int32_t* dst = kept_idx + (bh * nb + i0 + warp) * (int64_t)topk;
   int out = 0, ties_seen = 0;
   const uint32_t lt_mask = (1u << lane) - 1u;
   for (int base = 0; base < nb; base += 32) {
     const int j = base + lane;
-    const uint32_t kj = (j < nb) ? key[j] : 0u;
     const bool valid = j < nb;
+    const uint32_t kj = valid ? key_at(j) : 0u;
     const bool tie = valid && (kj == thr);
     const uint32_t tie_ballot = __ballot_sync(0xffffffffu, tie);
     const int tie_rank = ties_seen + __popc(tie_ballot & lt_mask);
@@ -208,6 +144,134 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
     if (keep) dst[out + __popc(keep_ballot & lt_mask)] = j;
     out += __popc(keep_ballot);
     ties_seen += __popc(tie_ballot);
+  }
+}
+
+constexpr int kKeysInRegs = 24;   // rows with nb <= 32 * 24 keep their keys in registers during the selection
+
+template <int D>
+__global__ void __launch_bounds__(kTopkThreads)
+topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
+            int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  // pooled Q of the CTA's 8 query blocks, channel-major: s_pq[c][r], so that one 16-byte load
+  // yields four rows of one channel as two packed fp32x2 operands
+  float* s_pq = reinterpret_cast<float*>(smem_raw);                          // [D][kRowsPerCta]
+  uint32_t* s_key = reinterpret_cast<uint32_t*>(s_pq + kRowsPerCta * D);     // [kRowsPerCta][nbp]
+
+  const int64_t bh = blockIdx.x / groups_per_bh;
+  const int i0 = (blockIdx.x % groups_per_bh) * kRowsPerCta;
+  const int nrows = min(kRowsPerCta, nb - i0);
+
+  for (int e = threadIdx.x; e < kRowsPerCta * D; e += kTopkThreads) {
+    const int r = e / D, c = e % D;
+    s_pq[c * kRowsPerCta + r] = (r < nrows) ? pq[(bh * nb + i0 + r) * D + c] : 0.0f;
+  }
+  __syncthreads();
+
+  // scores: a thread owns kJT key blocks (j, j + kTopkThreads) and walks the channels in ascending
+  // order for the CTA's 8 query blocks at once.  fma.rn.f32x2 is a pair of IEEE fmaf, so every
+  // accumulator still sees exactly the chain a = fmaf(pq[i,c], pk[j,c], a), c ascending.
+  const float* kcol = pkT + bh * D * (int64_t)nbp;
+  const ulonglong2* s_pq2 = reinterpret_cast<const ulonglong2*>(s_pq);       // [D][kRowsPerCta / 4]
+  constexpr int kJT = 2;
+  constexpr int kPairs = kRowsPerCta / 2;
+  for (int j0 = threadIdx.x; j0 < nb; j0 += kTopkThreads * kJT) {
+    int jcl[kJT];
+#pragma unroll
+    for (int u = 0; u < kJT; ++u) jcl[u] = min(j0 + u * kTopkThreads, nb - 1);  // clamped: loads stay in range
+    uint64_t acc[kJT][kPairs];
+#pragma unroll
+    for (int u = 0; u < kJT; ++u)
+#pragma unroll
+      for (int r = 0; r < kPairs; ++r) acc[u][r] = pack_f32x2(0.0f, 0.0f);
+    constexpr int kCB = 16;  // channels per batch of loads (2 x 16 loads in flight per thread)
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += kCB) {
+      float kv[kJT][kCB];
+#pragma unroll
+      for (int u = 0; u < kJT; ++u)
+#pragma unroll
+        for (int cc = 0; cc < kCB; ++cc) kv[u][cc] = __ldg(kcol + (int64_t)(c0 + cc) * nbp + jcl[u]);
+#pragma unroll
+      for (int cc = 0; cc < kCB; ++cc) {
+        const ulonglong2 qa = s_pq2[(c0 + cc) * 2], qb = s_pq2[(c0 + cc) * 2 + 1];   // rows (0,1),(2,3) | (4,5),(6,7)
+#pragma unroll
+        for (int u = 0; u < kJT; ++u) {
+          const uint64_t k2 = pack_f32x2(kv[u][cc], kv[u][cc]);
+          acc[u][0] = ffma2(qa.x, k2, acc[u][0]);
+          acc[u][1] = ffma2(qa.y, k2, acc[u][1]);
+          acc[u][2] = ffma2(qb.x, k2, acc[u][2]);
+          acc[u][3] = ffma2(qb.y, k2, acc[u][3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kJT; ++u) {
+      const int j = j0 + u * kTopkThreads;
+      if (j < nb) {
+#pragma unroll
+        for (int r = 0; r < kPairs; ++r) {
+          const float2 a = unpack_f32x2(acc[u][r]);
+          s_key[(2 * r) * nbp + j] = score_key(a.x);
+          s_key[(2 * r + 1) * nbp + j] = score_key(a.y);
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp >= nrows) return;   // (warps beyond the 8 rows of the CTA have no row)
+  const uint32_t* key = s_key + warp * nbp;
+  int32_t* dst = kept_idx + (bh * nb + i0 + warp) * (int64_t)topk;
+  if (nb <= 32 * kKeysInRegs) {
+    uint32_t kr[kKeysInRegs];
+#pragma unroll
+    for (int u = 0; u < kKeysInRegs; ++u) kr[u] = (lane + 32 * u < nb) ? key[lane + 32 * u] : 0u;
+    // same algorithm as select_row, with the key loops unrolled over registers; a padding key
+    // of 0 is below every candidate (candidates are >= 1) and is excluded by index where needed
+    uint32_t kmin = 0xffffffffu, kmaxv = 0u;
+#pragma unroll
+    for (int u = 0; u < kKeysInRegs; ++u)
+      if (lane + 32 * u < nb) { kmin = min(kmin, kr[u]); kmaxv = max(kmaxv, kr[u]); }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmaxv = __reduce_max_sync(0xffffffffu, kmaxv);
+    const int top_bit = 31 - __clz(kmin ^ kmaxv);
+    uint32_t thr = (top_bit >= 31) ? 0u : (kmaxv & ~((2u << max(top_bit, 0)) - 1u));
+    if (top_bit < 0) thr = kmaxv;
+    for (int bit = top_bit; bit >= 0; --bit) {
+      const uint32_t cand = thr | (1u << bit);
+      int cnt = 0;
+#pragma unroll
+      for (int u = 0; u < kKeysInRegs; ++u) cnt += (kr[u] >= cand);
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if (cnt >= topk) thr = cand;
+    }
+    int ngreater = 0;
+#pragma unroll
+    for (int u = 0; u < kKeysInRegs; ++u) ngreater += (lane + 32 * u < nb) && (kr[u] > thr);
+    ngreater = __reduce_add_sync(0xffffffffu, ngreater);
+    const int ties_allowed = topk - ngreater;
+    int out = 0, ties_seen = 0;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+    for (int u = 0; u < kKeysInRegs; ++u) {
+      if (32 * u < nb) {
+        const int j = lane + 32 * u;
+        const bool valid = j < nb;
+        const bool tie = valid && (kr[u] == thr);
+        const uint32_t tie_ballot = __ballot_sync(0xffffffffu, tie);
+        const int tie_rank = ties_seen + __popc(tie_ballot & lt_mask);
+        const bool keep = valid && ((kr[u] > thr) || (tie && tie_rank < ties_allowed));
+        const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
+        if (keep) dst[out + __popc(keep_ballot & lt_mask)] = j;
+        out += __popc(keep_ballot);
+        ties_seen += __popc(tie_ballot);
+      }
+    }
+  } else {
+    select_row([&](int j) { return key[j]; }, nb, topk, lane, dst);
   }
   if (lane == 0 && kept_cnt != nullptr) kept_cnt[bh * nb + i0 + warp] = topk;
 }
