@@ -410,6 +410,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["wan14b", "wan1p3b"], default="wan14b")
     ap.add_argument("--sparsity", type=float, default=None)
+    ap.add_argument("--block", type=int, default=None, help="token block size (default: the workload's; 64 = the paper's trained size)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fp8", action="store_true")
@@ -421,6 +422,8 @@ def main():
     w = workloads.WORKLOADS[args.workload]
     if args.sparsity is not None:
         w = w.with_sparsity(args.sparsity)
+    if args.block is not None and args.block != w.block:
+        w = workloads.Workload(f"{w.name}_b{args.block}", w.cfg_id, w.B, w.H, w.d, w.grid, args.block, w.sparsity)
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -49,7 +49,7 @@ extern "C" {
 typedef enum {
   SPARKATTN_OK = 0,
   SPARKATTN_E_INVALID_ARG = -1,       /* NULL pointer, non-positive size, topk/kmax out of range      */
-  SPARKATTN_E_UNSUPPORTED_SHAPE = -2, /* (d, block) not one of (64,64), (128,128); nb too large        */
+  SPARKATTN_E_UNSUPPORTED_SHAPE = -2, /* (d, block) not one of (64,64), (128,64), (128,128); nb too large */
   SPARKATTN_E_MISALIGNED = -3,        /* pointer not 16-byte aligned or stride * elem not 16-byte mult. */
   SPARKATTN_E_WORKSPACE_TOO_SMALL = -4,
   SPARKATTN_E_CUDA = -5,              /* launch or driver error; cudaGetLastError has the detail       */
@@ -122,7 +122,7 @@ int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint
  *
  * dtype      : SPARKATTN_BF16: q,k,v bf16.  SPARKATTN_FP8_E4M3: q,k,v are E4M3
  *              codes from sparkattn_quant_fp8 with q_scale/k_scale/v_scale fp32
- *              [B,H,nb]; requires d = block = 128.  Scales are NULL for bf16.
+ *              [B,H,nb]; requires d = 128 (block 64 or 128).  Scales are NULL for bf16.
  * kept_idx   : in, int32 [B,H,nb,kmax]; entries distinct, each in [0, nb); kmax <= 2048
  *              (longer lists return SPARKATTN_E_UNSUPPORTED_SHAPE)
  * kept_cnt   : in, int32 [B,H,nb] with 0 <= cnt <= kmax; NULL means cnt = kmax everywhere

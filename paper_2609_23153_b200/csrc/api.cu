@@ -20,7 +20,8 @@ int check_shape(const sparkattn_shape_t* s) {
   if (s->struct_size != sizeof(sparkattn_shape_t) || s->version != SPARKATTN_VERSION) return SPARKATTN_E_INVALID_ARG;
   if (s->B < 1 || s->H < 1 || s->N < 1 || s->reserved != 0 || s->pad != 0) return SPARKATTN_E_INVALID_ARG;
   if (!(s->softmax_scale >= 0.0f) || isinf(s->softmax_scale)) return SPARKATTN_E_INVALID_ARG;
-  if (!((s->d == 64 && s->block == 64) || (s->d == 128 && s->block == 128))) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (!((s->d == 64 && s->block == 64) || (s->d == 128 && (s->block == 128 || s->block == 64))))
+    return SPARKATTN_E_UNSUPPORTED_SHAPE;
   if (s->stride_n < s->d || s->stride_h < 1 || s->stride_b < 1) return SPARKATTN_E_INVALID_ARG;
   // 16-byte rule for vector loads and TMA, for 2-byte and for 1-byte elements
   if (s->stride_n % 16 || s->stride_h % 16 || s->stride_b % 16) return SPARKATTN_E_MISALIGNED;
@@ -95,7 +96,7 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
   if (kmax > kFwdMaxKept) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   if (dtype == SPARKATTN_FP8_E4M3) {
     if (!q_scale || !k_scale || !v_scale) return SPARKATTN_E_INVALID_ARG;
-    if (!(shape->d == 128 && shape->block == 128)) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+    if (shape->d != 128) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   }
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out_bf16) || !aligned256(workspace))
     return SPARKATTN_E_MISALIGNED;

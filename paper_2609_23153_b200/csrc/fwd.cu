@@ -541,6 +541,10 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
     return fp8 ? launch_fwd_t<128, 128, true>(s, mq, mk, mv, prm, stream)
                : launch_fwd_t<128, 128, false>(s, mq, mk, mv, prm, stream);
   }
+  if (s.d == 128 && s.block == 64) {
+    return fp8 ? launch_fwd_t<128, 64, true>(s, mq, mk, mv, prm, stream)
+               : launch_fwd_t<128, 64, false>(s, mq, mk, mv, prm, stream);
+  }
   if (s.d == 64 && s.block == 64 && !fp8) return launch_fwd_t<64, 64, false>(s, mq, mk, mv, prm, stream);
   return SPARKATTN_E_UNSUPPORTED_SHAPE;
 }

@@ -95,6 +95,9 @@ int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, 
   if (s.d == 128 && s.block == 128) {
     quant_fp8_kernel<128, 128><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
         xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
+  } else if (s.d == 128 && s.block == 64) {
+    quant_fp8_kernel<128, 64><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
   } else if (s.d == 64 && s.block == 64) {
     quant_fp8_kernel<64, 64><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
         xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);

@@ -105,3 +105,32 @@ def test_host_buffer_call_matches_device_call():
         out = sa.attention_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), w.block, w.topk, dtype=dtype, kept_idx=hidx)
         assert torch.equal(out, ref.cpu())
         assert torch.equal(hidx, idx.cpu())
+
+
+def test_fullsize_paper_block_size_64_bf16_and_fp8():
+    """Wan2.1-14B-720P shape with the paper's trained 64x64 blocks (nb = 1182, 35 kept at 97 %)."""
+    w64 = workloads.Workload("wan14b_b64", 3, 1, 40, 128, (21, 45, 80), 64, 0.97)
+    assert w64.nb == 1182 and w64.topk == 35
+    heads = [0, 21, 39]
+    q, k, v = workloads.structured_qkv(w64, device=DEV)
+    idx, cnt = sa.select(q, k, w64.block, w64.topk)
+    out = sa.fwd(q, k, v, idx, cnt, w64.block, check_status=True)
+    qh, kh, vh = (t[0, heads].cpu() for t in (q, k, v))
+    ref_idx, ref_cnt = oracle.select(qh, kh, w64.block, w64.topk)
+    assert torch.equal(idx[0, heads].cpu(), ref_idx)
+    local = _sample_items(w64, range(len(heads)), 6, seed=17)
+    items = [(heads[h], i) for h, i in local]
+    ref_out, _ = oracle.attention(qh, kh, vh, ref_idx, ref_cnt, w64.block, items=local)
+    rel, mx = _relrms(_gather(out[0], items, w64), _ref_rows(ref_out, local, w64))
+    print(f"wan14b 64x64 bf16: {len(items)} work items, relRMS {rel:.3e}, max abs {mx:.3e}")
+    assert rel <= 1e-2 and mx <= 3e-2
+    cs = [sa.quant_fp8(t, w64.block) for t in (q, k, v)]
+    out8 = sa.fwd(cs[0][0], cs[1][0], cs[2][0], idx, cnt, w64.block, scales=tuple(s for _, s in cs), check_status=True)
+    rc, rs = oracle.quant_fp8(kh, w64.block)
+    assert torch.equal(cs[1][0][0, heads].cpu(), rc) and torch.equal(cs[1][1][0, heads].cpu().view(torch.int32), rs.view(torch.int32))
+    local8 = local[:9]
+    ref8, _ = oracle.attention(*(c[0, heads].cpu() for c, _ in cs), ref_idx, ref_cnt, w64.block, items=local8,
+                               scales=tuple(s[0, heads].cpu() for _, s in cs))
+    rel8, mx8 = _relrms(_gather(out8[0], [(heads[h], i) for h, i in local8], w64), _ref_rows(ref8, local8, w64))
+    print(f"wan14b 64x64 fp8: {len(local8)} work items, relRMS {rel8:.3e}, max abs {mx8:.3e}")
+    assert rel8 <= 5e-2

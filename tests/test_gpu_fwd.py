@@ -63,6 +63,7 @@ SMALL = [
     _small(33, 2, 64, (3, 10, 21), 64, 0.8),      # N=630, tail 54
     _small(34, 2, 128, (4, 11, 23), 128, 0.0),    # dense, N=1012, tail 116
     _small(35, 1, 128, (1, 1, 5), 128, 0.0),      # single ragged block of 5 tokens
+    _small(39, 2, 128, (4, 9, 25), 64, 0.75),     # d=128 with the paper's 64x64 blocks: N=900, tail 4
 ]
 
 
@@ -151,7 +152,7 @@ def test_deterministic_and_rows_past_n_untouched():
     assert torch.equal(a, b)
 
 
-@pytest.mark.parametrize("w", [SMALL[0], SMALL[1], SMALL[3]], ids=lambda w: f"{w.name}-N{w.N}-s{w.sparsity}")
+@pytest.mark.parametrize("w", [SMALL[0], SMALL[1], SMALL[3], SMALL[5]], ids=lambda w: f"{w.name}-N{w.N}-b{w.block}-s{w.sparsity}")
 def test_small_structured_full_parity_fp8(w):
     q, k, v = workloads.structured_qkv(w)
     idx, cnt = oracle.select(q[0], k[0], w.block, w.topk)      # selection always reads bf16

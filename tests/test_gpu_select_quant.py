@@ -17,6 +17,7 @@ def _small_cases():
         workloads.small_structured(H=2, d=64, grid=(3, 10, 21), block=64, sparsity=0.9, cfg_id=13),     # N=630: tail 54
         workloads.small_structured(H=1, d=64, grid=(1, 1, 37), block=64, sparsity=0.0, cfg_id=14),      # one ragged block
         workloads.small_structured(H=2, d=128, grid=(1, 1, 1), block=128, sparsity=0.0, cfg_id=15),     # N=1
+        workloads.small_structured(H=2, d=128, grid=(4, 9, 25), block=64, sparsity=0.9, cfg_id=17),     # d=128, 64-token blocks, tail 4
     ]
 
 

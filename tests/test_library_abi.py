@@ -94,7 +94,9 @@ def test_argument_errors_are_caught_on_the_host(lib):
     assert r == sa.E_INVALID_ARG
     r = lib.sparkattn_fwd(ctypes.byref(s), sa.FP8_E4M3, fake, fake, fake, fake, fake, fake, fake, null, 4, fake,
                           null, fake, 256, st)
-    assert r == sa.E_UNSUPPORTED_SHAPE
+    assert r == sa.E_UNSUPPORTED_SHAPE            # FP8 needs d = 128
+    assert sa.workspace_bytes(_shape(d=128, block=64), 1, 4) == 256
+    assert sa.workspace_bytes(_shape(d=64, block=128), 1, 4) == 0
     r = lib.sparkattn_fwd(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 40, fake,
                           null, fake, 256, st)
     assert r == sa.E_INVALID_ARG
