@@ -114,6 +114,21 @@ int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint
                         uint32_t flags, void* cuda_stream);
 
 /*
+ * Per-token FP8 quantisation: the activation-quantisation kernel as the paper
+ * states it (Sec. 4.3: activations "scaled dynamically per token", scale and
+ * cast in one pass).  Same arithmetic as sparkattn_quant_fp8 with the token
+ * block replaced by one token row: amax over the row's d channels, clamped at
+ * 1e-12; scale = amax / 448; code = e4m3_rne_satfinite(x * (448 / amax)).
+ * Not consumed by sparkattn_fwd (which takes per-block scales); provided for
+ * the activation path around it.  `shape->block` is ignored beyond validation.
+ * x_bf16 : in,  bf16 [B,H,N,d] (strides of `shape`)
+ * codes  : out, uint8 E4M3 codes, same element strides as x
+ * scales : out, fp32 [B,H,N] contiguous
+ */
+int sparkattn_quant_fp8_per_token(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes,
+                                  float* scales, void* cuda_stream);
+
+/*
  * Block-sparse attention forward (Sec. 2 dense attention formula restricted
  * to the kept tiles; Sec. 4.1 sparse branch).  For query token i in query
  * block qb, over the keys j of the kept key blocks kept_idx[b,h,qb,0..cnt):

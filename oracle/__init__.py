@@ -45,6 +45,7 @@ def _load():
         L.oracle_select.restype = ctypes.c_int
         L.oracle_select_f64_diff.restype = ctypes.c_int64
         L.oracle_quant_fp8.restype = None
+        L.oracle_quant_fp8_per_token.restype = None
         L.oracle_pool.restype = None
         L.oracle_num_threads.restype = ctypes.c_int
         _lib = L
@@ -182,4 +183,15 @@ def quant_fp8(x: torch.Tensor, block: int):
     scales = torch.zeros((H, nb), dtype=torch.float32)
     L.oracle_quant_fp8(_ptr(_raw16(x)), ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d),
                        ctypes.c_int(block), _ptr(codes), _ptr(scales))
+    return codes, scales
+
+
+def quant_fp8_per_token(x: torch.Tensor):
+    """QNT-1 with one scale per token.  x: [H, N, d] bf16.  Returns (codes uint8 [H, N, d], scales fp32 [H, N])."""
+    L = _load()
+    H, N, d = x.shape
+    codes = torch.zeros((H, N, d), dtype=torch.uint8)
+    scales = torch.zeros((H, N), dtype=torch.float32)
+    L.oracle_quant_fp8_per_token(_ptr(_raw16(x)), ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d),
+                                 _ptr(codes), _ptr(scales))
     return codes, scales

@@ -21,7 +21,8 @@
  *                             here is spelled out step by step below).
  *   QNT-1  oracle_quant_fp8   per-(head, token-block) absmax scale + E4M3
  *                             round-to-nearest-even encode (Sec. 4.3 names FP8
- *                             E4M3 with scale-and-cast in one pass).
+ *                             E4M3 with scale-and-cast in one pass);
+ *          oracle_quant_fp8_per_token   the same with one scale per token.
  *
  * OpenMP only distributes independent work items (one (head, query block) or
  * one (head, block) each); inside an item everything is a scalar loop in the
@@ -320,6 +321,25 @@ void oracle_quant_fp8(const uint16_t* x, int H, int N, int d, int blk, uint8_t* 
         const float y = bf16_to_f32(x[(h * N + t) * d + c]) * inv;
         codes[(h * N + t) * d + c] = oracle_e4m3_encode(y);
       }
+  }
+}
+
+/* Per-token variant (the granularity the paper's Sec. 4.3 states for activations: one dynamic
+ * scale per token): the same QNT-1 steps with the block replaced by a single token row. */
+void oracle_quant_fp8_per_token(const uint16_t* x, int H, int N, int d, uint8_t* codes /* [H][N][d] */,
+                                float* scales /* [H][N] */) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < (int64_t)H * N; ++r) {
+    float amax = 0.0f;
+    for (int c = 0; c < d; ++c) {
+      float a = fabsf(bf16_to_f32(x[r * d + c]));
+      if (a > amax) amax = a;
+    }
+    if (amax < 1e-12f) amax = 1e-12f;
+    const float scale = amax / 448.0f;
+    const float inv = 448.0f / amax;
+    scales[r] = scale;
+    for (int c = 0; c < d; ++c) codes[r * d + c] = oracle_e4m3_encode(bf16_to_f32(x[r * d + c]) * inv);
   }
 }
 

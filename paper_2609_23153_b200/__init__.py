@@ -33,7 +33,7 @@ FP8_E4M3 = 1
 
 EXPORTS = (
     "sparkattn_version", "sparkattn_status_string", "sparkattn_workspace_bytes", "sparkattn_select",
-    "sparkattn_quant_fp8", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
+    "sparkattn_quant_fp8", "sparkattn_quant_fp8_per_token", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
     "sparkattn_attention_host", "sparkattn_select_noalloc", "sparkattn_select_noalloc_max_bytes",
     "sparkattn_select_noalloc_status",
 )
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_select.argtypes = [sp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.sparkattn_quant_fp8.restype = ctypes.c_int
         L.sparkattn_quant_fp8.argtypes = [sp, vp, vp, vp, ctypes.c_uint32, vp]
+        L.sparkattn_quant_fp8_per_token.restype = ctypes.c_int
+        L.sparkattn_quant_fp8_per_token.argtypes = [sp, vp, vp, vp, vp]
         L.sparkattn_fwd.restype = ctypes.c_int
         L.sparkattn_fwd.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.sparkattn_read_status.restype = ctypes.c_int
@@ -193,6 +195,21 @@ def quant_fp8(x: torch.Tensor, block: int, *, codes: Optional[torch.Tensor] = No
         scales = torch.empty((B, H, nb), dtype=torch.float32, device=x.device)
     rc = lib().sparkattn_quant_fp8(ctypes.byref(shape), _ptr(x), _ptr(codes), _ptr(scales), 0, _stream_ptr(stream))
     _check(rc, "sparkattn_quant_fp8")
+    return codes, scales
+
+
+def quant_fp8_per_token(x: torch.Tensor, *, codes: Optional[torch.Tensor] = None,
+                        scales: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+                        ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_quant_fp8_per_token``: x bf16 [B,H,N,d] -> (codes uint8, same strides; scales fp32 [B,H,N])."""
+    shape = make_shape(x, 64 if x.shape[-1] == 64 else 128)
+    B, H, N, _ = x.shape
+    if codes is None:
+        codes = torch.empty_strided(x.shape, x.stride(), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty((B, H, N), dtype=torch.float32, device=x.device)
+    rc = lib().sparkattn_quant_fp8_per_token(ctypes.byref(shape), _ptr(x), _ptr(codes), _ptr(scales), _stream_ptr(stream))
+    _check(rc, "sparkattn_quant_fp8_per_token")
     return codes, scales
 
 

@@ -84,6 +84,15 @@ int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint
   return launch_quant_fp8(*shape, x_bf16, codes, scales, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int sparkattn_quant_fp8_per_token(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes,
+                                  float* scales, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!x_bf16 || !codes || !scales) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned16(x_bf16) || !aligned16(codes)) return SPARKATTN_E_MISALIGNED;
+  return launch_quant_fp8_per_token(*shape, x_bf16, codes, scales, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
                   const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                   const int32_t* kept_cnt, int32_t kmax, void* out_bf16, float* lse, void* workspace,

@@ -14,6 +14,9 @@ namespace sparkattn {
 int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
                      cudaStream_t stream);
 
+int launch_quant_fp8_per_token(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
+                               cudaStream_t stream);
+
 // select.cu
 constexpr int kSelectMaxBlocks = 4096;  // largest nb the selection kernel holds in shared memory
 size_t select_workspace_bytes(const sparkattn_shape_t& s);

@@ -86,6 +86,93 @@ quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ code
   }
 }
 
+// Per-token variant: a token row (d channels) is spread over d/8 lanes, 16 bytes per lane, so a
+// warp covers 32/(d/8) rows per step; it walks kTokenSteps steps with all loads issued first
+// (128 bytes in flight per thread).  absmax by shuffles inside the lane group, then scale,
+// encode and store from the same registers: one HBM read, one write.
+constexpr int kTokenSteps = 8;
+
+template <int D>
+__global__ void __launch_bounds__(kQuantThreads)
+quant_fp8_token_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ scales,
+                       int H, int N, int64_t stride_b, int64_t stride_h, int64_t stride_n, int64_t n_rows) {
+  constexpr int LPR = D / 8;                     // lanes per row: 16 (d=128) or 8 (d=64)
+  constexpr int RPS = 32 / LPR;                  // rows per warp step
+  const int lane = threadIdx.x & 31;
+  const int sub = lane / LPR, chunk = lane % LPR;
+  const int64_t warp_id = (int64_t)blockIdx.x * (kQuantThreads / 32) + (threadIdx.x >> 5);
+  const int64_t row0 = warp_id * (kTokenSteps * RPS);
+  uint4 v[kTokenSteps];
+  int64_t off[kTokenSteps];
+  // (batch, head, token) of this lane's first row: divisions once, then the rows just count up
+  const uint32_t first = (uint32_t)(row0 + sub);            // n_rows < 2^31 (checked by the launcher)
+  const uint32_t bh0 = first / (uint32_t)N;
+  int n = (int)(first - bh0 * (uint32_t)N);
+  int b = (int)(bh0 / (uint32_t)H), h = (int)(bh0 - (uint32_t)b * (uint32_t)H);
+#pragma unroll
+  for (int u = 0; u < kTokenSteps; ++u) {
+    const int64_t r = row0 + u * RPS + sub;
+    off[u] = b * stride_b + h * stride_h + (int64_t)n * stride_n + chunk * 8;
+    n += RPS;
+    while (n >= N) {
+      n -= N;
+      if (++h == H) { h = 0; ++b; }
+    }
+    v[u] = (r < n_rows) ? __ldg(reinterpret_cast<const uint4*>(x + off[u])) : make_uint4(0u, 0u, 0u, 0u);
+  }
+#pragma unroll
+  for (int u = 0; u < kTokenSteps; ++u) {
+    const int64_t r = row0 + u * RPS + sub;
+    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v[u]);
+    float f[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 t = __bfloat1622float2(p2[j]);
+      f[2 * j] = t.x;
+      f[2 * j + 1] = t.y;
+    }
+    float amax = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(f[j]));
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    amax = fmaxf(amax, 1e-12f);
+    const float inv = __fdiv_rn(448.0f, amax);
+    if (r >= n_rows) continue;
+    if (chunk == 0) scales[r] = __fdiv_rn(amax, 448.0f);
+    uint32_t w[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f[4 * j], inv), __fmul_rn(f[4 * j + 1], inv)),
+                                                    __NV_SATFINITE, __NV_E4M3);
+      const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f[4 * j + 2], inv), __fmul_rn(f[4 * j + 3], inv)),
+                                                    __NV_SATFINITE, __NV_E4M3);
+      w[j] = lo | (hi << 16);
+    }
+    *reinterpret_cast<uint2*>(codes + off[u]) = make_uint2(w[0], w[1]);
+  }
+}
+
+int launch_quant_fp8_per_token(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
+                               cudaStream_t stream) {
+  const int64_t n_rows = (int64_t)s.B * s.H * s.N;
+  if (n_rows >= (1LL << 31) - 4096) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  const int64_t rows_per_cta = (kQuantThreads / 32) * kTokenSteps * (32 / (s.d / 8));
+  const int64_t ctas = (n_rows + rows_per_cta - 1) / rows_per_cta;
+  if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+  if (s.d == 128) {
+    quant_fp8_token_kernel<128><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, s.stride_b, s.stride_h, s.stride_n, n_rows);
+  } else if (s.d == 64) {
+    quant_fp8_token_kernel<64><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, s.stride_b, s.stride_h, s.stride_n, n_rows);
+  } else {
+    return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  }
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
 int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
                      cudaStream_t stream) {
   const int nb = (s.N + s.block - 1) / s.block;

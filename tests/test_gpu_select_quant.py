@@ -106,3 +106,27 @@ def test_select_and_quant_are_deterministic():
     c1 = sa.quant_fp8(v, w.block)[0].clone()
     c2 = sa.quant_fp8(v, w.block)[0].clone()
     assert torch.equal(c1, c2)
+
+
+@pytest.mark.parametrize("w", _small_cases(), ids=lambda w: f"{w.name}-N{w.N}-d{w.d}")
+def test_per_token_quant_matches_oracle(w):
+    q, _, v = workloads.structured_qkv(w)
+    v = v * torch.logspace(-2, 1, w.N)[None, None, :, None].to(torch.bfloat16)   # widely varying row magnitudes
+    v[0, 0, w.N // 2] = 0
+    for x in (q, v):
+        ref_codes, ref_scales = oracle.quant_fp8_per_token(x[0])
+        codes, scales = sa.quant_fp8_per_token(x.to(DEV))
+        torch.cuda.synchronize()
+        assert torch.equal(scales[0].cpu().view(torch.int32), ref_scales.view(torch.int32))
+        assert torch.equal(codes[0].cpu(), ref_codes)
+
+
+def test_per_token_quant_strided_and_fullsize_sample():
+    w = workloads.WAN_1P3B_480P
+    q, _, _ = workloads.structured_qkv(w, device=DEV)
+    qs = q.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)          # [B,N,H,d] storage
+    codes, scales = sa.quant_fp8_per_token(qs)
+    assert codes.stride() == qs.stride()
+    for h in (0, 11):
+        rc, rs = oracle.quant_fp8_per_token(q[0, h:h + 1].cpu())
+        assert torch.equal(codes[0, h:h + 1].cpu(), rc) and torch.equal(scales[0, h:h + 1].cpu().view(torch.int32), rs.view(torch.int32))

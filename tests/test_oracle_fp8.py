@@ -146,3 +146,25 @@ def test_block_quant_scales_and_codes():
     err = (deq - x.double()).abs()
     bound = scales.double().repeat_interleave(block, 1)[:, :N, None] * 16.0 + 1e-30  # half of the largest step (32)
     assert torch.all(err <= bound)
+
+
+def test_per_token_quant_scales_and_codes():
+    H, N, d = 2, 37, 32
+    g = torch.Generator().manual_seed(8)
+    x = (torch.randn((H, N, d), generator=g) * torch.logspace(-3, 2, N)[None, :, None]).to(torch.bfloat16)
+    x[1, 5] = 0                         # an all-zero token
+    x[0, 7, 3] = -9.0; x[0, 7].clamp_(-9, 9)
+    codes, scales = oracle.quant_fp8_per_token(x)
+    for h in range(H):
+        for n in range(N):
+            row = x[h, n].float().numpy()
+            amax = np.float32(max(float(np.abs(row).max()), 1e-12))
+            assert scales[h, n].item() == float(amax / np.float32(448.0))
+            y = row * (np.float32(448.0) / amax)
+            ref = torch.from_numpy(np.clip(y, -448, 448)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+            assert np.array_equal(ref, codes[h, n].numpy())
+    assert codes[0, 7, 3].item() == 0xFE
+    assert set(np.unique(codes[1, 5].numpy()).tolist()) <= {0x00, 0x80}
+    # a block of one token reproduces the block-wise routine
+    c1, s1 = oracle.quant_fp8(x[:, :1].contiguous(), 64)
+    assert torch.equal(c1, codes[:, :1]) and torch.equal(s1[:, 0], scales[:, 0])
