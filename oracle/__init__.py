@@ -46,6 +46,8 @@ def _load():
         L.oracle_select_f64_diff.restype = ctypes.c_int64
         L.oracle_quant_fp8.restype = None
         L.oracle_quant_fp8_per_token.restype = None
+        L.oracle_comp_state.restype = None
+        L.oracle_comp_apply.restype = None
         L.oracle_pool.restype = None
         L.oracle_num_threads.restype = ctypes.c_int
         _lib = L
@@ -195,3 +197,36 @@ def quant_fp8_per_token(x: torch.Tensor):
     L.oracle_quant_fp8_per_token(_ptr(_raw16(x)), ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d),
                                  _ptr(codes), _ptr(scales))
     return codes, scales
+
+
+def comp_state(k: torch.Tensor, v: torch.Tensor, pk: torch.Tensor, grid, axis: torch.Tensor, freq: torch.Tensor):
+    """CMP-0, state: C[h] = sum_j k~_j v_j^T.  k, v bf16 [H, N, d]; pk bf16 [H, r, d]; grid (T, Hg, Wg);
+    axis int32 [r/2] (0 = t, 1 = y, 2 = x); freq fp32 [r/2].  Returns fp64 [H, r, d]."""
+    L = _load()
+    H, N, d = k.shape
+    r = pk.shape[1]
+    assert grid[0] * grid[1] * grid[2] == N and pk.shape == (H, r, d)
+    state = torch.zeros((H, r, d), dtype=torch.float64)
+    g = torch.tensor(list(grid), dtype=torch.int32)
+    L.oracle_comp_state(_ptr(_raw16(k)), _ptr(_raw16(v)), _ptr(_raw16(pk)), ctypes.c_int(H), ctypes.c_int(N),
+                        ctypes.c_int(d), ctypes.c_int(r), _ptr(g), _ptr(axis.contiguous().to(torch.int32)),
+                        _ptr(freq.contiguous().float()), _ptr(state))
+    return state
+
+
+def comp_apply(q: torch.Tensor, pq: torch.Tensor, state: torch.Tensor, gate: torch.Tensor, o_sparse: torch.Tensor,
+               grid, axis: torch.Tensor, freq: torch.Tensor, rows, eps: float = 1e-6):
+    """CMP-0, apply: O_i = O_s,i + g_i r_i RMSNorm(q~_i^T C) for the (head, token) pairs in ``rows``.
+    Returns fp64 [len(rows), d]."""
+    L = _load()
+    H, N, d = q.shape
+    r = pq.shape[1]
+    rr = torch.tensor(list(rows), dtype=torch.int32).reshape(-1, 2).contiguous()
+    out = torch.zeros((rr.shape[0], d), dtype=torch.float64)
+    g = torch.tensor(list(grid), dtype=torch.int32)
+    L.oracle_comp_apply(_ptr(_raw16(q)), _ptr(_raw16(pq)), _ptr(state.contiguous().double()),
+                        _ptr(gate.contiguous().float()), _ptr(_raw16(o_sparse)), ctypes.c_int(H), ctypes.c_int(N),
+                        ctypes.c_int(d), ctypes.c_int(r), _ptr(g), _ptr(axis.contiguous().to(torch.int32)),
+                        _ptr(freq.contiguous().float()), ctypes.c_double(eps), _ptr(rr), ctypes.c_int(rr.shape[0]),
+                        _ptr(out))
+    return out

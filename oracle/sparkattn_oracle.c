@@ -23,6 +23,8 @@
  *                             round-to-nearest-even encode (Sec. 4.3 names FP8
  *                             E4M3 with scale-and-cast in one pass);
  *          oracle_quant_fp8_per_token   the same with one scale per token.
+ *   CMP-0  oracle_comp_state / oracle_comp_apply   low-rank compensation branch and
+ *                             token-wise gate fusion (Sec. 4.1), fp64.
  *
  * OpenMP only distributes independent work items (one (head, query block) or
  * one (head, block) each); inside an item everything is a scalar loop in the
@@ -340,6 +342,87 @@ void oracle_quant_fp8_per_token(const uint16_t* x, int H, int N, int d, uint8_t*
     const float inv = 448.0f / amax;
     scales[r] = scale;
     for (int c = 0; c < d; ++c) codes[r * d + c] = oracle_e4m3_encode(bf16_to_f32(x[r * d + c]) * inv);
+  }
+}
+
+/* ---------- CMP-0: low-rank compensation branch and gate (paper Sec. 4.1) ---------- */
+/*
+ * For head h, token i at grid position (t, y, x) (raster order n = (t*Hg + y)*Wg + x):
+ *   u      = P x                      P is [r][d] (P_q for queries, P_k for keys), x the token's q or k row
+ *   a_m    = pos_{axis[m]}(i) * freq[m]                      m = 0 .. r/2-1   (rank-truncated 3-D RoPE)
+ *   z      = silu(u) ,  silu(s) = s / (1 + exp(-s))
+ *   x~[2m]   = z[2m] cos a_m - z[2m+1] sin a_m
+ *   x~[2m+1] = z[2m] sin a_m + z[2m+1] cos a_m
+ *   C      = sum_j k~_j v_j^T                                 [r][d] per head
+ *   y_i    = q~_i^T C ;  O_lr,i = y_i / sqrt(mean_c y_i[c]^2 + eps)          (RMSNorm, no learned weight)
+ *   r_i    = sqrt(mean_c O_s[i,c]^2)                          (RMS of the sparse-branch output row)
+ *   O_i    = O_s,i + g_i * r_i * O_lr,i
+ * Everything in fp64 from the stored bf16 inputs; nothing is rounded in between.
+ */
+static void comp_feature(const uint16_t* xrow, const uint16_t* P /* [r][d] */, int d, int r, const int32_t* axis,
+                         const float* freq, const int pos[3], double* outv /* [r] */) {
+  for (int a = 0; a < r; ++a) {
+    double u = 0.0;
+    for (int c = 0; c < d; ++c) u += (double)bf16_to_f32(P[a * d + c]) * (double)bf16_to_f32(xrow[c]);
+    outv[a] = u / (1.0 + exp(-u));
+  }
+  for (int m = 0; m < r / 2; ++m) {
+    const double ang = (double)pos[axis[m]] * (double)freq[m];
+    const double cs = cos(ang), sn = sin(ang);
+    const double z0 = outv[2 * m], z1 = outv[2 * m + 1];
+    outv[2 * m] = z0 * cs - z1 * sn;
+    outv[2 * m + 1] = z0 * sn + z1 * cs;
+  }
+}
+
+/* state [H][r][d] fp64 ; k, v [H][N][d] bf16 ; pk [H][r][d] bf16 ; grid = (T, Hg, Wg) with T*Hg*Wg == N */
+void oracle_comp_state(const uint16_t* k, const uint16_t* v, const uint16_t* pk, int H, int N, int d, int r,
+                       const int32_t* grid, const int32_t* axis, const float* freq, double* state) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int h = 0; h < H; ++h) {
+    double* C = state + (int64_t)h * r * d;
+    double* kt = (double*)malloc(sizeof(double) * r);
+    for (int64_t e = 0; e < (int64_t)r * d; ++e) C[e] = 0.0;
+    for (int64_t j = 0; j < N; ++j) {
+      const int pos[3] = {(int)(j / ((int64_t)grid[1] * grid[2])), (int)((j / grid[2]) % grid[1]), (int)(j % grid[2])};
+      comp_feature(k + ((int64_t)h * N + j) * d, pk + (int64_t)h * r * d, d, r, axis, freq, pos, kt);
+      for (int a = 0; a < r; ++a)
+        for (int c = 0; c < d; ++c) C[a * d + c] += kt[a] * (double)bf16_to_f32(v[((int64_t)h * N + j) * d + c]);
+    }
+    free(kt);
+  }
+}
+
+/* out [n_rows][d] fp64 for the listed (h, token) pairs ; o_sparse [H][N][d] bf16 ; gate [H][N] fp32 */
+void oracle_comp_apply(const uint16_t* q, const uint16_t* pq, const double* state, const float* gate,
+                       const uint16_t* o_sparse, int H, int N, int d, int r, const int32_t* grid,
+                       const int32_t* axis, const float* freq, double eps, const int32_t* rows, int n_rows,
+                       double* out) {
+  (void)H;
+#pragma omp parallel for schedule(static)
+  for (int it = 0; it < n_rows; ++it) {
+    const int h = rows[2 * it];
+    const int64_t i = rows[2 * it + 1];
+    const int pos[3] = {(int)(i / ((int64_t)grid[1] * grid[2])), (int)((i / grid[2]) % grid[1]), (int)(i % grid[2])};
+    double* qt = (double*)malloc(sizeof(double) * r);
+    double* y = (double*)malloc(sizeof(double) * d);
+    comp_feature(q + ((int64_t)h * N + i) * d, pq + (int64_t)h * r * d, d, r, axis, freq, pos, qt);
+    const double* C = state + (int64_t)h * r * d;
+    double ss = 0.0, so = 0.0;
+    for (int c = 0; c < d; ++c) {
+      double acc = 0.0;
+      for (int a = 0; a < r; ++a) acc += qt[a] * C[a * d + c];
+      y[c] = acc;
+      ss += acc * acc;
+      const double os = (double)bf16_to_f32(o_sparse[((int64_t)h * N + i) * d + c]);
+      so += os * os;
+    }
+    const double inv = 1.0 / sqrt(ss / d + eps);
+    const double ri = sqrt(so / d);
+    const double g = (double)gate[(int64_t)h * N + i];
+    for (int c = 0; c < d; ++c)
+      out[(int64_t)it * d + c] = (double)bf16_to_f32(o_sparse[((int64_t)h * N + i) * d + c]) + g * ri * y[c] * inv;
+    free(qt); free(y);
   }
 }
 

@@ -182,3 +182,38 @@ def shard_heads(H: int, world_size: int, rank: int) -> range:
     base, extra = divmod(H, world_size)
     start = rank * base + min(rank, extra)
     return range(start, start + base + (1 if rank < extra else 0))
+
+
+def rope_schedule(d: int, rank: int, theta: float = 10000.0):
+    """Rank-truncated 3-D rotary schedule: the d/2 rotary pairs of a head are split over the axes
+    (t, y, x) as (d/2 - 2*(d/6), d/6, d/6) pairs (22 / 21 / 21 for d = 128, the split video DiTs of
+    this family use), pair p of an axis with n_a pairs has frequency theta^(-p / n_a); the
+    compensation branch keeps the first rank/2 pairs.  Returns (axis int32 [rank/2], freq fp32 [rank/2])."""
+    half = d // 2
+    n_y = n_x = d // 6
+    n_t = half - n_y - n_x
+    axis, freq = [], []
+    for a, n_a in enumerate((n_t, n_y, n_x)):
+        for pidx in range(n_a):
+            axis.append(a)
+            freq.append(theta ** (-pidx / n_a))
+    axis = torch.tensor(axis[: rank // 2], dtype=torch.int32)
+    freq = torch.tensor(freq[: rank // 2], dtype=torch.float32)
+    return axis, freq
+
+
+def compensation_params(w: Workload, rank: int = 64, heads: Optional[Sequence[int]] = None, device: str = "cpu",
+                        gate_scale: float = 0.3):
+    """Seeded stand-ins for the trained parts of the compensation branch: low-rank projections
+    P_q, P_k ~ N(0, 1/d) (bf16 [H, rank, d]) and a token-wise gate g ~ U(0, gate_scale) (fp32
+    [B, H, N]; the trained gate starts near zero, a visible one is used so that the branch matters
+    in parity tests)."""
+    heads = list(range(w.H)) if heads is None else list(heads)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(w.cfg_id * 7919 + 13)
+    pq = (torch.randn((w.H, rank, w.d), generator=g) / math.sqrt(w.d)).to(torch.bfloat16)[heads]
+    pk = (torch.randn((w.H, rank, w.d), generator=g) / math.sqrt(w.d)).to(torch.bfloat16)[heads]
+    gd = torch.Generator(device=device)
+    gd.manual_seed(w.cfg_id * 7919 + 14)
+    gate = torch.rand((w.B, len(heads), w.N), generator=gd, device=device, dtype=torch.float32) * gate_scale
+    return pq.to(device), pk.to(device), gate
