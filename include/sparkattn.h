@@ -170,6 +170,47 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
                              int32_t* kept_idx_host, void* arena, size_t arena_bytes, void* cuda_stream);
 
 /*
+ * Low-rank compensation branch and gate fusion (Sec. 4.1, "low-rank
+ * compensation branch" and the fused output O = O_s + g * r * O_lr).
+ * With rank r = 64 projections P_q, P_k per head and the rank-truncated rotary
+ * rotation R_r (adjacent feature pairs (2m, 2m+1) rotated by the angle
+ * pos_axis[m] * freq[m], pos = the token's (t, y, x) coordinate on the latent
+ * grid, raster token order n = (t * Hg + y) * Wg + x):
+ *   q~_i = R_r(p_i) silu(P_q q_i)        k~_j = R_r(p_j) silu(P_k k_j)
+ *   C    = sum_j k~_j v_j^T              (r x d per (batch, head): sparkattn_comp_state)
+ *   y_i  = q~_i^T C ;  O_lr,i = y_i / sqrt(mean_c y_i[c]^2 + eps)      (RMSNorm, no weight)
+ *   r_i  = sqrt(mean_c O_s,i[c]^2)  ;    O_i = O_s,i + g_i * r_i * O_lr,i   (sparkattn_comp_apply)
+ * Linear in N.  Requires d = 128 and rank = 64; `shape->block` is validated but not used.
+ *
+ * Arithmetic: projections, C and y are tensor-core products of bf16 operands
+ * with fp32 accumulation (q~, k~ and, in the apply pass, C are rounded to
+ * bf16 first); silu, rotation, norms and the fusion are fp32; the state is
+ * summed over fixed token chunks in a fixed order.
+ *
+ * k, v, q, o_sparse : in,  bf16 [B,H,N,d] with the strides of `shape`
+ * pk, pq            : in,  bf16 [H, rank, d] contiguous, 16-byte aligned
+ * grid_host         : in,  HOST int32[3] = (T, Hg, Wg), T*Hg*Wg = N
+ * rope_axis_host    : in,  HOST int32[rank/2], entries 0 (t), 1 (y) or 2 (x)
+ * rope_freq_host    : in,  HOST fp32[rank/2]
+ * state             : comp_state out / comp_apply in, fp32 [B,H,rank,d] contiguous
+ * gate              : in,  fp32 [B,H,N] contiguous (the token-wise gate g)
+ * out_bf16          : out, bf16 [B,H,N,d], strides of `shape`; may alias o_sparse
+ * eps               : RMSNorm epsilon (> 0)
+ * workspace         : >= sparkattn_comp_workspace_bytes(shape) bytes, 256-byte aligned;
+ *                     first word = device status (sparkattn_read_status)
+ * The host arrays are read during the call only.
+ */
+size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape);
+int sparkattn_comp_state(const sparkattn_shape_t* shape, const void* k_bf16, const void* v_bf16, const void* pk_bf16,
+                         int32_t rank, const int32_t* grid_host, const int32_t* rope_axis_host,
+                         const float* rope_freq_host, float* state, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream);
+int sparkattn_comp_apply(const sparkattn_shape_t* shape, const void* q_bf16, const void* pq_bf16, int32_t rank,
+                         const int32_t* grid_host, const int32_t* rope_axis_host, const float* rope_freq_host,
+                         const float* state, const float* gate, const void* o_sparse_bf16, void* out_bf16, float eps,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Block selection without any allocation (the paper has no counterpart: this
  * is a packaging variant of sparkattn_select, same rule, same outputs).
  *

@@ -35,7 +35,8 @@ EXPORTS = (
     "sparkattn_version", "sparkattn_status_string", "sparkattn_workspace_bytes", "sparkattn_select",
     "sparkattn_quant_fp8", "sparkattn_quant_fp8_per_token", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
     "sparkattn_attention_host", "sparkattn_select_noalloc", "sparkattn_select_noalloc_max_bytes",
-    "sparkattn_select_noalloc_status",
+    "sparkattn_select_noalloc_status", "sparkattn_comp_workspace_bytes", "sparkattn_comp_state",
+    "sparkattn_comp_apply",
 )
 
 
@@ -94,6 +95,12 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_select_noalloc_max_bytes.restype = sz
         L.sparkattn_select_noalloc_status.restype = ctypes.c_int
         L.sparkattn_select_noalloc_status.argtypes = [vp]
+        L.sparkattn_comp_workspace_bytes.restype = sz
+        L.sparkattn_comp_workspace_bytes.argtypes = [sp]
+        L.sparkattn_comp_state.restype = ctypes.c_int
+        L.sparkattn_comp_state.argtypes = [sp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.sparkattn_comp_apply.restype = ctypes.c_int
+        L.sparkattn_comp_apply.argtypes = [sp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -262,4 +269,71 @@ def attention_host(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, block: int
     rc = lib().sparkattn_attention_host(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), topk, _ptr(out),
                                         _ptr(kept_idx), _ptr(arena), arena.numel(), _stream_ptr(stream))
     _check(rc, "sparkattn_attention_host")
+    return out
+
+
+def _rope_host(grid, axis: torch.Tensor, freq: torch.Tensor):
+    g = (ctypes.c_int32 * 3)(*[int(x) for x in grid])
+    a = axis.detach().to("cpu", torch.int32).contiguous()
+    f = freq.detach().to("cpu", torch.float32).contiguous()
+    if a.numel() != f.numel():
+        raise ValueError("rope axis and frequency tables must have rank/2 entries each")
+    return g, a, f
+
+
+def comp_workspace_bytes(shape: Shape) -> int:
+    return int(lib().sparkattn_comp_workspace_bytes(ctypes.byref(shape)))
+
+
+def comp_state(k: torch.Tensor, v: torch.Tensor, pk: torch.Tensor, grid, axis: torch.Tensor, freq: torch.Tensor, *,
+               state: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+               stream: Optional[torch.cuda.Stream] = None, check_status: bool = False) -> torch.Tensor:
+    """``sparkattn_comp_state``: k, v bf16 [B,H,N,d]; pk bf16 [H,r,d]; grid (T,Hg,Wg); axis/freq the
+    rotary tables (rank/2 entries, any device).  Returns the state fp32 [B,H,r,d]."""
+    _same_layout(k, v)
+    shape = make_shape(k, 128)
+    B, H, _, d = k.shape
+    rank = pk.shape[1]
+    g, a, f = _rope_host(grid, axis, freq)
+    if not pk.is_contiguous() or pk.shape != (H, rank, d):
+        raise ValueError("pk must be contiguous [H, rank, d]")
+    if state is None:
+        state = torch.empty((B, H, rank, d), dtype=torch.float32, device=k.device)
+    if workspace is None:
+        workspace = torch.empty(max(comp_workspace_bytes(shape), 256), dtype=torch.uint8, device=k.device)
+    rc = lib().sparkattn_comp_state(ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(pk), rank, g, _ptr(a), _ptr(f),
+                                    _ptr(state), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_comp_state")
+    if check_status:
+        _check(read_status(workspace, stream), "sparkattn_comp_state (device status)")
+    return state
+
+
+def comp_apply(q: torch.Tensor, pq: torch.Tensor, state: torch.Tensor, gate: torch.Tensor, o_sparse: torch.Tensor,
+               grid, axis: torch.Tensor, freq: torch.Tensor, *, eps: float = 1e-6,
+               out: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+               stream: Optional[torch.cuda.Stream] = None, check_status: bool = False) -> torch.Tensor:
+    """``sparkattn_comp_apply``: q, o_sparse bf16 [B,H,N,d]; pq bf16 [H,r,d]; state fp32 [B,H,r,d];
+    gate fp32 [B,H,N].  Returns the fused output bf16 [B,H,N,d]."""
+    _same_layout(q, o_sparse)
+    shape = make_shape(q, 128)
+    B, H, N, d = q.shape
+    rank = pq.shape[1]
+    g, a, f = _rope_host(grid, axis, freq)
+    if not pq.is_contiguous() or pq.shape != (H, rank, d):
+        raise ValueError("pq must be contiguous [H, rank, d]")
+    if not state.is_contiguous() or state.shape != (B, H, rank, d) or state.dtype != torch.float32:
+        raise ValueError("state must be contiguous fp32 [B, H, rank, d]")
+    if not gate.is_contiguous() or gate.shape != (B, H, N) or gate.dtype != torch.float32:
+        raise ValueError("gate must be contiguous fp32 [B, H, N]")
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=torch.bfloat16, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=q.device)
+    rc = lib().sparkattn_comp_apply(ctypes.byref(shape), _ptr(q), _ptr(pq), rank, g, _ptr(a), _ptr(f), _ptr(state),
+                                    _ptr(gate), _ptr(o_sparse), _ptr(out), ctypes.c_float(eps), _ptr(workspace),
+                                    workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_comp_apply")
+    if check_status:
+        _check(read_status(workspace, stream), "sparkattn_comp_apply (device status)")
     return out

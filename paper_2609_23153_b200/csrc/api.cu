@@ -114,6 +114,56 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
                     workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
+namespace {
+int check_comp(const sparkattn_shape_t* s, int32_t rank, const int32_t* grid, const int32_t* axis, const float* freq) {
+  int rc = check_shape(s);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!grid || !axis || !freq) return SPARKATTN_E_INVALID_ARG;
+  if (s->d != 128 || rank != kCompRank) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (grid[0] < 1 || grid[1] < 1 || grid[2] < 1 || (long long)grid[0] * grid[1] * grid[2] != (long long)s->N)
+    return SPARKATTN_E_INVALID_ARG;
+  for (int m = 0; m < rank / 2; ++m)
+    if (axis[m] < 0 || axis[m] > 2 || !isfinite(freq[m])) return SPARKATTN_E_INVALID_ARG;
+  return SPARKATTN_OK;
+}
+}  // namespace
+
+size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape) {
+  if (check_shape(shape) != SPARKATTN_OK || shape->d != 128) return 0;
+  return comp_workspace_bytes(*shape);
+}
+
+int sparkattn_comp_state(const sparkattn_shape_t* shape, const void* k_bf16, const void* v_bf16, const void* pk_bf16,
+                         int32_t rank, const int32_t* grid_host, const int32_t* rope_axis_host,
+                         const float* rope_freq_host, float* state, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream) {
+  int rc = check_comp(shape, rank, grid_host, rope_axis_host, rope_freq_host);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!k_bf16 || !v_bf16 || !pk_bf16 || !state || !workspace) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned16(k_bf16) || !aligned16(v_bf16) || !aligned16(pk_bf16) || !aligned16(state) || !aligned256(workspace))
+    return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < comp_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  return launch_comp_state(*shape, k_bf16, v_bf16, pk_bf16, grid_host, rope_axis_host, rope_freq_host, state,
+                           workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sparkattn_comp_apply(const sparkattn_shape_t* shape, const void* q_bf16, const void* pq_bf16, int32_t rank,
+                         const int32_t* grid_host, const int32_t* rope_axis_host, const float* rope_freq_host,
+                         const float* state, const float* gate, const void* o_sparse_bf16, void* out_bf16, float eps,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = check_comp(shape, rank, grid_host, rope_axis_host, rope_freq_host);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!q_bf16 || !pq_bf16 || !state || !gate || !o_sparse_bf16 || !out_bf16 || !workspace)
+    return SPARKATTN_E_INVALID_ARG;
+  if (!(eps > 0.0f) || isinf(eps)) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned16(q_bf16) || !aligned16(pq_bf16) || !aligned16(state) || !aligned16(o_sparse_bf16) ||
+      !aligned16(out_bf16) || !aligned256(workspace))
+    return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < (size_t)kWorkspaceHeaderBytes) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  return launch_comp_apply(*shape, q_bf16, pq_bf16, grid_host, rope_axis_host, rope_freq_host, state, gate,
+                           o_sparse_bf16, out_bf16, eps, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int sparkattn_read_status(void* workspace, void* cuda_stream) {
   if (!workspace) return SPARKATTN_E_INVALID_ARG;
   int32_t word = 0;

@@ -1,0 +1,536 @@
+// Low-rank compensation branch and gate fusion of the paper's attention module (Sec. 4.1):
+//   q~_i = R_r(p_i) silu(P_q q_i),  k~_j = R_r(p_j) silu(P_k k_j),  C = sum_j k~_j v_j^T,
+//   O_lr,i = RMSNorm(q~_i^T C),  O_i = O_s,i + g_i r_i O_lr,i,  r_i = RMS(O_s,i).
+// Linear in the sequence length; both passes are streaming and HBM-bound, their contractions
+// (projection to rank r = 64, k~ v^T accumulation, q~ C) run as tcgen05 MMAs with TMEM accumulators.
+//
+//   comp_state_kernel   CTA = one chunk of 128-token tiles of one (batch, head).  Per tile:
+//                       T = K P_k^T (MMA) -> silu + rotary on the T rows (one thread per token)
+//                       -> k~ as bf16 into shared memory -> C^T += V^T k~ (MMA, both operands
+//                       MN-major straight from the row-major tiles).  The chunk's C^T goes to
+//                       the workspace; comp_reduce_kernel adds the chunks in a fixed order.
+//   comp_apply_kernel   CTA = a few 128-token tiles of one (batch, head).  Per tile:
+//                       T = Q P_q^T -> silu + rotary -> q~ (bf16, shared memory) -> Y = q~ C
+//                       (MMA, C as bf16 in shared memory) -> per row RMSNorm, RMS of the sparse
+//                       output row, gate, add, store.
+// Every mbarrier wait is bounded; rows past N are zero tiles (TMA fill) and are never stored.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace sparkattn {
+
+constexpr int kCompThreads = 192;     // warps 0-3: one thread per token row; warp 4: TMA; warp 5: MMA issue
+constexpr int kRank = 64;
+constexpr int kCD = 128;              // head dimension handled by this file
+constexpr int kTileTok = 128;
+constexpr int kApplyTilesPerCta = 4;
+
+struct RopeTable {
+  int32_t axis[kRank / 2];            // 0 = t, 1 = y, 2 = x
+  float freq[kRank / 2];
+  int32_t T, Hg, Wg;
+};
+
+struct CompParams {
+  RopeTable rope;
+  int H, N, nt;                       // nt = number of 128-token tiles
+  int tiles_per_cta, nchunks;
+  int64_t stride_b, stride_h, stride_n;
+  float* partial;                     // state: [BH][nchunks][d][r] fp32
+  const float* state;                 // apply: [BH][r][d] fp32
+  const float* gate;                  // apply: [BH][N]
+  const __nv_bfloat16* o_sparse;      // apply
+  __nv_bfloat16* out;                 // apply
+  float eps;
+  int32_t* status;
+};
+
+// silu, then the rank-truncated rotary rotation of adjacent pairs; v holds the 64 features of one token
+__device__ __forceinline__ void silu_rope(float (&v)[kRank], const RopeTable& rope, int token) {
+  const int x = token % rope.Wg;
+  const int y = (token / rope.Wg) % rope.Hg;
+  const int t = token / (rope.Wg * rope.Hg);
+#pragma unroll
+  for (int a = 0; a < kRank; ++a) v[a] = __fdividef(v[a], 1.0f + __expf(-v[a]));
+#pragma unroll
+  for (int m = 0; m < kRank / 2; ++m) {
+    const int ax = rope.axis[m];
+    const float pos = (float)(ax == 0 ? t : (ax == 1 ? y : x));
+    float sn, cs;
+    sincosf(pos * rope.freq[m], &sn, &cs);
+    const float z0 = v[2 * m], z1 = v[2 * m + 1];
+    v[2 * m] = z0 * cs - z1 * sn;
+    v[2 * m + 1] = z0 * sn + z1 * cs;
+  }
+}
+
+// one token's 64 features as bf16 into row `row` of a [128 rows x 128 B] tile with 128-byte swizzle
+__device__ __forceinline__ void store_feature_row(unsigned char* tile, int row, const float (&v)[kRank]) {
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * c + 2 * j], v[8 * c + 2 * j + 1]);
+      w[j] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+    *reinterpret_cast<uint4*>(tile + row * 128 + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// instruction descriptor with both major bits explicit (bf16 in, fp32 accumulate)
+__host__ __device__ constexpr uint32_t comp_idesc(uint32_t M, uint32_t N, bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((N >> 3) << 17) |
+         ((M >> 4) << 24);
+}
+
+// T[128 tokens x 64] = X[128 x 128] P^T : X tile K-major (2 slabs of 16 KB), P K-major (2 slabs of 8 KB)
+__device__ __forceinline__ void issue_projection(uint32_t tmem_T, uint32_t x_smem, uint32_t p_smem) {
+  const uint64_t dX = make_smem_desc_sw128(x_smem, 16), dP = make_smem_desc_sw128(p_smem, 16);
+  const uint32_t x_lo = (uint32_t)dX, x_hi = (uint32_t)(dX >> 32), p_lo = (uint32_t)dP, p_hi = (uint32_t)(dP >> 32);
+  constexpr uint32_t idesc = comp_idesc(128, kRank, false, false);
+#pragma unroll
+  for (int s = 0; s < 2; ++s)
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk)
+      mma_ss<false>(tmem_T, make_desc(x_lo + ((s * 16384 + kk * 32) >> 4), x_hi),
+                    make_desc(p_lo + ((s * 8192 + kk * 32) >> 4), p_hi), idesc, (s | kk) != 0 ? 1u : 0u);
+}
+
+constexpr int kStateSmem = 1024 + 16384 /*P*/ + 32768 /*K*/ + 32768 /*V*/ + 16384 /*k~*/ + 256;
+constexpr int kApplySmem = 1024 + 16384 /*P*/ + 16384 /*C*/ + 32768 /*Q*/ + 16384 /*q~*/ + 256;
+
+__global__ void __launch_bounds__(kCompThreads, 2)
+comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                  const __grid_constant__ CUtensorMap tmap_p, const CompParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* sP = smem;
+  unsigned char* sK = sP + 16384;
+  unsigned char* sV = sK + 32768;
+  unsigned char* sF = sV + 32768;                 // k~ tile: [128 tokens][64] bf16
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sF + 16384);
+  uint64_t* bar_p_full = bars + 0;
+  uint64_t* bar_k_full = bars + 1;
+  uint64_t* bar_v_full = bars + 2;
+  uint64_t* bar_t_full = bars + 3;                // projection done (also: K slot free)
+  uint64_t* bar_f_full = bars + 4;                // features written by all 128 threads
+  uint64_t* bar_acc = bars + 5;                   // accumulation MMA done (also: V slot and k~ tile free)
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 6);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 7);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x, bh = blockIdx.y;
+  const int h = bh % p.H, b = bh / p.H;
+  const int tile0 = chunk * p.tiles_per_cta;
+  const int ntiles = max(0, min(p.tiles_per_cta, p.nt - tile0));
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_p_full, 1); mbar_init(bar_k_full, 1); mbar_init(bar_v_full, 1);
+    mbar_init(bar_t_full, 1); mbar_init(bar_f_full, 128); mbar_init(bar_acc, 1);
+    *s_abort = 0;
+    mbar_fence_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(s_tmem, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+  const uint32_t tmem_T = tmem, tmem_C = tmem + 64;
+
+  if (warp == 4) {
+    if (lane == 0 && ntiles > 0) {
+      mbar_expect_tx(bar_p_full, 16384);
+      tma_load_4d(sP, &tmap_p, bar_p_full, 0, 0, h, 0);
+      tma_load_4d(sP + 8192, &tmap_p, bar_p_full, 64, 0, h, 0);
+      for (int i = 0; i < ntiles; ++i) {
+        const int row = (tile0 + i) * kTileTok;
+        if (i > 0 && !mbar_wait(bar_t_full, (i - 1) & 1, s_abort, p.status, 50)) break;
+        mbar_expect_tx(bar_k_full, 32768);
+        tma_load_4d(sK, &tmap_k, bar_k_full, 0, row, h, b);
+        tma_load_4d(sK + 16384, &tmap_k, bar_k_full, 64, row, h, b);
+        if (i > 0 && !mbar_wait(bar_acc, (i - 1) & 1, s_abort, p.status, 51)) break;
+        mbar_expect_tx(bar_v_full, 32768);
+        tma_load_4d(sV, &tmap_v, bar_v_full, 0, row, h, b);
+        tma_load_4d(sV + 16384, &tmap_v, bar_v_full, 64, row, h, b);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0 && ntiles > 0) {
+      // C^T[128 d x 64 r] += V^T k~ : A = V tile (MN-major: d contiguous, two 64-column slabs),
+      // B = k~ tile (MN-major: r contiguous), 16 tokens per MMA
+      const uint64_t dV = make_smem_desc_sw128(smem_u32(sV), 16384), dF = make_smem_desc_sw128(smem_u32(sF), 16);
+      const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32), f_lo = (uint32_t)dF, f_hi = (uint32_t)(dF >> 32);
+      constexpr uint32_t idesc_acc = comp_idesc(128, kRank, true, true);
+      bool ok = mbar_wait(bar_p_full, 0, s_abort, p.status, 52);
+      for (int i = 0; ok && i < ntiles; ++i) {
+        if (!(ok = mbar_wait(bar_k_full, i & 1, s_abort, p.status, 53))) break;
+        tc_fence_after();
+        issue_projection(tmem_T, smem_u32(sK), smem_u32(sP));
+        tc_commit(bar_t_full);
+        if (!(ok = mbar_wait(bar_v_full, i & 1, s_abort, p.status, 54))) break;
+        if (!(ok = mbar_wait(bar_f_full, i & 1, s_abort, p.status, 55))) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          mma_ss<false>(tmem_C, make_desc(v_lo + ((kk * 2048) >> 4), v_hi), make_desc(f_lo + ((kk * 2048) >> 4), f_hi),
+                        idesc_acc, (i | kk) != 0 ? 1u : 0u);
+        tc_commit(bar_acc);
+      }
+    }
+  } else {
+    const int row = threadIdx.x;                       // token row of the tile = TMEM lane
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    bool ok = true;
+    for (int i = 0; ok && i < ntiles; ++i) {
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full, i & 1, s_abort, p.status, 56));
+      if (!ok) break;
+      tc_fence_after();
+      float v[kRank];
+      {
+        uint32_t r[kRank];
+        tmem_ld32(tmem_T + lane_off, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld32(tmem_T + lane_off + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+        tc_wait_ld();
+#pragma unroll
+        for (int a = 0; a < kRank; ++a) v[a] = __uint_as_float(r[a]);
+      }
+      silu_rope(v, p.rope, min((tile0 + i) * kTileTok + row, p.N - 1));   // rows past N are zero anyway
+      if (i > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, (i - 1) & 1, s_abort, p.status, 57));   // k~ tile free
+        if (!ok) break;
+      }
+      store_feature_row(sF, row, v);
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(bar_f_full);
+    }
+    if (ok && ntiles > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, (ntiles - 1) & 1, s_abort, p.status, 58));
+      if (ok) {
+        tc_fence_after();
+        // thread = channel c of d; its TMEM row holds C^T[c][0..63]
+        float* dst = p.partial + (((int64_t)bh * p.nchunks + chunk) * kCD + row) * kRank;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t r[32];
+          tmem_ld32(tmem_C + lane_off + half * 32, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            reinterpret_cast<uint4*>(dst + half * 32)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        }
+      }
+    } else if (ntiles == 0) {
+      float* dst = p.partial + (((int64_t)bh * p.nchunks + chunk) * kCD + row) * kRank;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) reinterpret_cast<uint4*>(dst)[j] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    if (*s_abort) __nanosleep(200000);
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+// state[bh][r][d] = sum over chunks (ascending) of partial[bh][chunk][d][r]
+__global__ void comp_reduce_kernel(const float* __restrict__ partial, float* __restrict__ state, int nchunks) {
+  const int bh = blockIdx.x;
+  for (int e = threadIdx.x; e < kRank * kCD; e += blockDim.x) {
+    const int a = e / kCD, c = e % kCD;
+    float acc = 0.0f;
+    for (int k = 0; k < nchunks; ++k) acc += partial[(((int64_t)bh * nchunks + k) * kCD + c) * kRank + a];
+    state[((int64_t)bh * kRank + a) * kCD + c] = acc;
+  }
+}
+
+__global__ void __launch_bounds__(kCompThreads, 2)
+comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_p,
+                  const CompParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* sP = smem;
+  unsigned char* sC = sP + 16384;                 // C as bf16, [64 r rows][128 d], two 64-column slabs of 8 KB
+  unsigned char* sQ = sC + 16384;
+  unsigned char* sF = sQ + 32768;                 // q~ tile: [128 tokens][64] bf16
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sF + 16384);
+  uint64_t* bar_p_full = bars + 0;
+  uint64_t* bar_q_full = bars + 1;
+  uint64_t* bar_t_full = bars + 2;                // projection done (also: Q slot free)
+  uint64_t* bar_f_full = bars + 3;                // q~ written by all 128 threads (first use: C staged too)
+  uint64_t* bar_y_full = bars + 4;                // Y = q~ C done
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 6);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 7);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y;
+  const int h = bh % p.H, b = bh / p.H;
+  const int tile0 = blockIdx.x * p.tiles_per_cta;
+  const int ntiles = max(0, min(p.tiles_per_cta, p.nt - tile0));
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_p_full, 1); mbar_init(bar_q_full, 1); mbar_init(bar_t_full, 1);
+    mbar_init(bar_f_full, 128); mbar_init(bar_y_full, 1);
+    *s_abort = 0;
+    mbar_fence_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(s_tmem, 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+  const uint32_t tmem_T = tmem, tmem_Y = tmem + 64;
+
+  if (warp == 4) {
+    if (lane == 0 && ntiles > 0) {
+      mbar_expect_tx(bar_p_full, 16384);
+      tma_load_4d(sP, &tmap_p, bar_p_full, 0, 0, h, 0);
+      tma_load_4d(sP + 8192, &tmap_p, bar_p_full, 64, 0, h, 0);
+      for (int i = 0; i < ntiles; ++i) {
+        const int row = (tile0 + i) * kTileTok;
+        if (i > 0 && !mbar_wait(bar_t_full, (i - 1) & 1, s_abort, p.status, 60)) break;
+        mbar_expect_tx(bar_q_full, 32768);
+        tma_load_4d(sQ, &tmap_q, bar_q_full, 0, row, h, b);
+        tma_load_4d(sQ + 16384, &tmap_q, bar_q_full, 64, row, h, b);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0 && ntiles > 0) {
+      // Y[128 tokens x 128 d] = q~ C : A = q~ tile (K-major: r contiguous), B = C (MN-major: d contiguous, two slabs)
+      const uint64_t dF = make_smem_desc_sw128(smem_u32(sF), 16), dC = make_smem_desc_sw128(smem_u32(sC), 8192);
+      const uint32_t f_lo = (uint32_t)dF, f_hi = (uint32_t)(dF >> 32), c_lo = (uint32_t)dC, c_hi = (uint32_t)(dC >> 32);
+      constexpr uint32_t idesc_y = comp_idesc(128, kCD, false, true);
+      bool ok = mbar_wait(bar_p_full, 0, s_abort, p.status, 61);
+      for (int i = 0; ok && i < ntiles; ++i) {
+        if (!(ok = mbar_wait(bar_q_full, i & 1, s_abort, p.status, 62))) break;
+        tc_fence_after();
+        issue_projection(tmem_T, smem_u32(sQ), smem_u32(sP));
+        tc_commit(bar_t_full);
+        if (!(ok = mbar_wait(bar_f_full, i & 1, s_abort, p.status, 63))) break;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ss<false>(tmem_Y, make_desc(f_lo + ((kk * 32) >> 4), f_hi), make_desc(c_lo + ((kk * 2048) >> 4), c_hi),
+                        idesc_y, kk != 0 ? 1u : 0u);
+        tc_commit(bar_y_full);
+      }
+    }
+  } else {
+    const int row = threadIdx.x;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    if (ntiles > 0) {
+      // stage C: thread j converts row a = j/2, columns [64*(j%2), +64) of the fp32 state to bf16
+      const int a = row >> 1, half = row & 1;
+      const float* src = p.state + ((int64_t)bh * kRank + a) * kCD + half * 64;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float4 lo = __ldg(reinterpret_cast<const float4*>(src + 8 * c));
+        const float4 hi = __ldg(reinterpret_cast<const float4*>(src + 8 * c + 4));
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(lo.x, lo.y), h1 = __floats2bfloat162_rn(lo.z, lo.w);
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(hi.x, hi.y), h3 = __floats2bfloat162_rn(hi.z, hi.w);
+        *reinterpret_cast<uint4*>(sC + half * 8192 + a * 128 + ((c ^ (a & 7)) << 4)) =
+            make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                       *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+      }
+    }
+    bool ok = true;
+    for (int i = 0; ok && i < ntiles; ++i) {
+      const int token = (tile0 + i) * kTileTok + row;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full, i & 1, s_abort, p.status, 64));
+      if (!ok) break;
+      tc_fence_after();
+      {
+        float v[kRank];
+        uint32_t r[kRank];
+        tmem_ld32(tmem_T + lane_off, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+        tmem_ld32(tmem_T + lane_off + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+        tc_wait_ld();
+#pragma unroll
+        for (int a = 0; a < kRank; ++a) v[a] = __uint_as_float(r[a]);
+        silu_rope(v, p.rope, min(token, p.N - 1));
+        store_feature_row(sF, row, v);     // the previous tile's Y (which read this buffer) was waited for below
+      }
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(bar_f_full);
+
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_y_full, i & 1, s_abort, p.status, 65));
+      if (!ok) break;
+      tc_fence_after();
+      const bool valid = token < p.N;
+      const int64_t off = b * p.stride_b + h * p.stride_h + (int64_t)min(token, p.N - 1) * p.stride_n;
+      // RMS of the sparse-branch row and the gate
+      uint4 os[16];
+      float so = 0.0f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        os[c] = valid ? __ldg(reinterpret_cast<const uint4*>(p.o_sparse + off) + c) : make_uint4(0u, 0u, 0u, 0u);
+        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&os[c]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 f = __bfloat1622float2(h2[j]);
+          so = fmaf(f.x, f.x, fmaf(f.y, f.y, so));
+        }
+      }
+      const float g = valid ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
+      // two passes over Y in TMEM: sum of squares, then the fused output
+      float ss = 0.0f;
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_Y + lane_off + ch * 32, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) ss = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ss);
+      }
+      const float coef = g * sqrtf(so * (1.0f / kCD)) * rsqrtf(ss * (1.0f / kCD) + p.eps);
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_Y + lane_off + ch * 32, r);
+        tc_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&os[ch * 4 + c]);
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float2 f = __bfloat1622float2(h2[j]);
+              const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(coef, __uint_as_float(r[8 * c + 2 * j]), f.x),
+                                                              fmaf(coef, __uint_as_float(r[8 * c + 2 * j + 1]), f.y));
+              w[j] = *reinterpret_cast<const uint32_t*>(&o2);
+            }
+            reinterpret_cast<uint4*>(p.out + off)[ch * 4 + c] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      tc_fence_before();
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    if (*s_abort) __nanosleep(200000);
+    tc_fence_after();
+    tmem_dealloc(tmem, 256);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn comp_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  return fn;
+}
+
+static int comp_map(CUtensorMap* map, const void* base, cuuint64_t d0, cuuint64_t d1, cuuint64_t d2, cuuint64_t d3,
+                    cuuint64_t s1, cuuint64_t s2, cuuint64_t s3, cuuint32_t box_rows) {
+  EncodeTiledFn enc = comp_encode_fn();
+  if (!enc) return SPARKATTN_E_NO_DEVICE;
+  const cuuint64_t dims[4] = {d0, d1, d2, d3};
+  const cuuint64_t strides[3] = {s1 * 2, s2 * 2, s3 * 2};
+  const cuuint32_t box[4] = {64u, box_rows, 1u, 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+static int state_chunks(const sparkattn_shape_t& s) {
+  const int nt = (s.N + kTileTok - 1) / kTileTok;
+  const long long bh = (long long)s.B * s.H;
+  long long want = (296 + bh - 1) / bh;        // about two CTAs per SM of a 148-SM part
+  if (want < 1) want = 1;
+  if (want > nt) want = nt;
+  return (int)want;
+}
+
+size_t comp_workspace_bytes(const sparkattn_shape_t& s) {
+  return kWorkspaceHeaderBytes + (size_t)s.B * s.H * state_chunks(s) * kCD * kRank * sizeof(float);
+}
+
+static void fill_rope(CompParams& prm, const int32_t* grid, const int32_t* axis, const float* freq) {
+  for (int m = 0; m < kRank / 2; ++m) { prm.rope.axis[m] = axis[m]; prm.rope.freq[m] = freq[m]; }
+  prm.rope.T = grid[0]; prm.rope.Hg = grid[1]; prm.rope.Wg = grid[2];
+}
+
+int launch_comp_state(const sparkattn_shape_t& s, const void* k, const void* v, const void* pk, const int32_t* grid,
+                      const int32_t* axis, const float* freq, float* state, void* workspace, cudaStream_t stream) {
+  CUtensorMap mk, mv, mp;
+  int rc;
+  if ((rc = comp_map(&mk, k, s.d, s.N, s.H, s.B, s.stride_n, s.stride_h, s.stride_b, kTileTok)) != SPARKATTN_OK) return rc;
+  if ((rc = comp_map(&mv, v, s.d, s.N, s.H, s.B, s.stride_n, s.stride_h, s.stride_b, kTileTok)) != SPARKATTN_OK) return rc;
+  if ((rc = comp_map(&mp, pk, kCD, kRank, s.H, 1, kCD, (cuuint64_t)kRank * kCD, (cuuint64_t)s.H * kRank * kCD, kRank)) != SPARKATTN_OK)
+    return rc;
+  CompParams prm{};
+  fill_rope(prm, grid, axis, freq);
+  prm.H = s.H; prm.N = s.N; prm.nt = (s.N + kTileTok - 1) / kTileTok;
+  prm.nchunks = state_chunks(s);
+  prm.tiles_per_cta = (prm.nt + prm.nchunks - 1) / prm.nchunks;
+  prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
+  prm.partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + kWorkspaceHeaderBytes);
+  prm.status = static_cast<int32_t*>(workspace);
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  if (cudaFuncSetAttribute(comp_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStateSmem) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  const dim3 grid_dim((unsigned)prm.nchunks, (unsigned)(s.B * s.H));
+  comp_state_kernel<<<grid_dim, kCompThreads, kStateSmem, stream>>>(mk, mv, mp, prm);
+  comp_reduce_kernel<<<(unsigned)(s.B * s.H), 256, 0, stream>>>(prm.partial, state, prm.nchunks);
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq, const int32_t* grid,
+                      const int32_t* axis, const float* freq, const float* state, const float* gate,
+                      const void* o_sparse, void* out, float eps, void* workspace, cudaStream_t stream) {
+  CUtensorMap mq, mp;
+  int rc;
+  if ((rc = comp_map(&mq, q, s.d, s.N, s.H, s.B, s.stride_n, s.stride_h, s.stride_b, kTileTok)) != SPARKATTN_OK) return rc;
+  if ((rc = comp_map(&mp, pq, kCD, kRank, s.H, 1, kCD, (cuuint64_t)kRank * kCD, (cuuint64_t)s.H * kRank * kCD, kRank)) != SPARKATTN_OK)
+    return rc;
+  CompParams prm{};
+  fill_rope(prm, grid, axis, freq);
+  prm.H = s.H; prm.N = s.N; prm.nt = (s.N + kTileTok - 1) / kTileTok;
+  prm.tiles_per_cta = kApplyTilesPerCta;
+  prm.nchunks = (prm.nt + kApplyTilesPerCta - 1) / kApplyTilesPerCta;
+  prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
+  prm.state = state; prm.gate = gate;
+  prm.o_sparse = static_cast<const __nv_bfloat16*>(o_sparse);
+  prm.out = static_cast<__nv_bfloat16*>(out);
+  prm.eps = eps;
+  prm.status = static_cast<int32_t*>(workspace);
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  if (cudaFuncSetAttribute(comp_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kApplySmem) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  const dim3 grid_dim((unsigned)prm.nchunks, (unsigned)(s.B * s.H));
+  comp_apply_kernel<<<grid_dim, kCompThreads, kApplySmem, stream>>>(mq, mp, prm);
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+}  // namespace sparkattn

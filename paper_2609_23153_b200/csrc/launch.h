@@ -30,4 +30,13 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream);
 
+// comp.cu
+constexpr int kCompRank = 64;  // rank of the compensation branch the kernels are built for
+size_t comp_workspace_bytes(const sparkattn_shape_t& s);
+int launch_comp_state(const sparkattn_shape_t& s, const void* k, const void* v, const void* pk, const int32_t* grid,
+                      const int32_t* axis, const float* freq, float* state, void* workspace, cudaStream_t stream);
+int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq, const int32_t* grid,
+                      const int32_t* axis, const float* freq, const float* state, const float* gate,
+                      const void* o_sparse, void* out, float eps, void* workspace, cudaStream_t stream);
+
 }  // namespace sparkattn
