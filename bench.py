@@ -344,6 +344,41 @@ def run_ours(args, w):
                "note": "FP8 peak = measured bf16 peak x 2 (nominal ratio); torch._scaled_mm 8192^3 measured 3122 TFLOP/s on this pool"}
         del codes
 
+    # ---- compensation branch + gate fusion (d = 128 only): state pass over K, V, then the fused apply pass
+    comp = None
+    if not args.no_comp and w.d == 128:
+        pq, pk, gate = workloads.compensation_params(wr, 64, device=dev)
+        axis, freq = workloads.rope_schedule(w.d, 64)
+        ws_c = torch.empty(sa.comp_workspace_bytes(shape, w.grid), dtype=torch.uint8, device=dev)
+        state = torch.empty((w.B, w.H, 64, w.d), dtype=torch.float32, device=dev)
+        fused = torch.empty_like(q)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        eva = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+
+        def stepc(i):
+            if i >= 0:
+                evs[i][0].record(stream)
+            sa.comp_state(k, v, pk, w.grid, axis, freq, state=state, workspace=ws_c)
+            if i >= 0:
+                evs[i][1].record(stream); eva[i][0].record(stream)
+            sa.comp_apply(q, pq, state, gate, out, w.grid, axis, freq, out=fused, workspace=ws_c)
+            if i >= 0:
+                eva[i][1].record(stream)
+
+        msc = time_region(stepc, K, args.warmup, stream, dist_on) / K
+        if sa.read_status(ws_c) != sa.OK:
+            raise RuntimeError("device status after compensation")
+        ms_s = statistics.mean(a.elapsed_time(b) for a, b in evs)
+        ms_a = statistics.mean(a.elapsed_time(b) for a, b in eva)
+        sbytes = 2 * elems * 2
+        abytes = 3 * elems * 2 + gate.numel() * 4
+        comp = {"rank": 64, "ms_per_step": msc, "state_ms": ms_s, "state_GBps": sbytes / (ms_s * 1e-3) / 1e9,
+                "state_frac_of_hbm_peak": sbytes / (ms_s * 1e-3) / 1e9 / peaks["hbm"],
+                "apply_ms": ms_a, "apply_GBps": abytes / (ms_a * 1e-3) / 1e9,
+                "apply_frac_of_hbm_peak": abytes / (ms_a * 1e-3) / 1e9 / peaks["hbm"],
+                "launches_per_step": 3}
+        del fused, state, ws_c, pq, pk, gate
+
     # ---- sparsity sweep (optional): fwd only, lists from sparkattn_select
     sweep = None
     if args.sweep:
@@ -394,7 +429,7 @@ def run_ours(args, w):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": config_dict(w, "bf16"),
             "kept_flops_per_step_per_gpu": flops, "clocks": clocks, "gpu_launches": 3 * K,
-            "kernels": kernels, "roofline": roofline, "fp8": fp8, "e2e": e2e, "cpu_baseline": cpu,
+            "kernels": kernels, "roofline": roofline, "fp8": fp8, "compensation": comp, "e2e": e2e, "cpu_baseline": cpu,
         }
         if sweep is not None:
             line["sweep"] = sweep
@@ -415,6 +450,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fp8", action="store_true")
+    ap.add_argument("--no-comp", action="store_true", help="skip the compensation-branch leg")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

@@ -196,11 +196,12 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
  * gate              : in,  fp32 [B,H,N] contiguous (the token-wise gate g)
  * out_bf16          : out, bf16 [B,H,N,d], strides of `shape`; may alias o_sparse
  * eps               : RMSNorm epsilon (> 0)
- * workspace         : >= sparkattn_comp_workspace_bytes(shape) bytes, 256-byte aligned;
- *                     first word = device status (sparkattn_read_status)
+ * workspace         : >= sparkattn_comp_workspace_bytes(shape, grid_host) bytes, 256-byte aligned
+ *                     (sized for the state pass; the apply pass needs only its first
+ *                     256 + 16 * rank * max(T, Hg, Wg) bytes); first word = device status
  * The host arrays are read during the call only.
  */
-size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape);
+size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape, const int32_t* grid_host);
 int sparkattn_comp_state(const sparkattn_shape_t* shape, const void* k_bf16, const void* v_bf16, const void* pk_bf16,
                          int32_t rank, const int32_t* grid_host, const int32_t* rope_axis_host,
                          const float* rope_freq_host, float* state, void* workspace, size_t workspace_bytes,

@@ -96,7 +96,7 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_select_noalloc_status.restype = ctypes.c_int
         L.sparkattn_select_noalloc_status.argtypes = [vp]
         L.sparkattn_comp_workspace_bytes.restype = sz
-        L.sparkattn_comp_workspace_bytes.argtypes = [sp]
+        L.sparkattn_comp_workspace_bytes.argtypes = [sp, vp]
         L.sparkattn_comp_state.restype = ctypes.c_int
         L.sparkattn_comp_state.argtypes = [sp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
         L.sparkattn_comp_apply.restype = ctypes.c_int
@@ -281,8 +281,9 @@ def _rope_host(grid, axis: torch.Tensor, freq: torch.Tensor):
     return g, a, f
 
 
-def comp_workspace_bytes(shape: Shape) -> int:
-    return int(lib().sparkattn_comp_workspace_bytes(ctypes.byref(shape)))
+def comp_workspace_bytes(shape: Shape, grid) -> int:
+    g = (ctypes.c_int32 * 3)(*[int(x) for x in grid])
+    return int(lib().sparkattn_comp_workspace_bytes(ctypes.byref(shape), g))
 
 
 def comp_state(k: torch.Tensor, v: torch.Tensor, pk: torch.Tensor, grid, axis: torch.Tensor, freq: torch.Tensor, *,
@@ -300,7 +301,7 @@ def comp_state(k: torch.Tensor, v: torch.Tensor, pk: torch.Tensor, grid, axis: t
     if state is None:
         state = torch.empty((B, H, rank, d), dtype=torch.float32, device=k.device)
     if workspace is None:
-        workspace = torch.empty(max(comp_workspace_bytes(shape), 256), dtype=torch.uint8, device=k.device)
+        workspace = torch.empty(max(comp_workspace_bytes(shape, grid), 256), dtype=torch.uint8, device=k.device)
     rc = lib().sparkattn_comp_state(ctypes.byref(shape), _ptr(k), _ptr(v), _ptr(pk), rank, g, _ptr(a), _ptr(f),
                                     _ptr(state), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     _check(rc, "sparkattn_comp_state")
@@ -329,7 +330,7 @@ def comp_apply(q: torch.Tensor, pq: torch.Tensor, state: torch.Tensor, gate: tor
     if out is None:
         out = torch.empty_strided(q.shape, q.stride(), dtype=torch.bfloat16, device=q.device)
     if workspace is None:
-        workspace = torch.empty(256, dtype=torch.uint8, device=q.device)
+        workspace = torch.empty(max(comp_workspace_bytes(shape, grid), 256), dtype=torch.uint8, device=q.device)
     rc = lib().sparkattn_comp_apply(ctypes.byref(shape), _ptr(q), _ptr(pq), rank, g, _ptr(a), _ptr(f), _ptr(state),
                                     _ptr(gate), _ptr(o_sparse), _ptr(out), ctypes.c_float(eps), _ptr(workspace),
                                     workspace.numel(), _stream_ptr(stream))

@@ -128,9 +128,12 @@ int check_comp(const sparkattn_shape_t* s, int32_t rank, const int32_t* grid, co
 }
 }  // namespace
 
-size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape) {
-  if (check_shape(shape) != SPARKATTN_OK || shape->d != 128) return 0;
-  return comp_workspace_bytes(*shape);
+size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape, const int32_t* grid_host) {
+  if (check_shape(shape) != SPARKATTN_OK || shape->d != 128 || !grid_host) return 0;
+  if (grid_host[0] < 1 || grid_host[1] < 1 || grid_host[2] < 1 ||
+      (long long)grid_host[0] * grid_host[1] * grid_host[2] != (long long)shape->N)
+    return 0;
+  return comp_workspace_bytes(*shape, grid_host, true);
 }
 
 int sparkattn_comp_state(const sparkattn_shape_t* shape, const void* k_bf16, const void* v_bf16, const void* pk_bf16,
@@ -142,7 +145,7 @@ int sparkattn_comp_state(const sparkattn_shape_t* shape, const void* k_bf16, con
   if (!k_bf16 || !v_bf16 || !pk_bf16 || !state || !workspace) return SPARKATTN_E_INVALID_ARG;
   if (!aligned16(k_bf16) || !aligned16(v_bf16) || !aligned16(pk_bf16) || !aligned16(state) || !aligned256(workspace))
     return SPARKATTN_E_MISALIGNED;
-  if (workspace_bytes < comp_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < comp_workspace_bytes(*shape, grid_host, true)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   return launch_comp_state(*shape, k_bf16, v_bf16, pk_bf16, grid_host, rope_axis_host, rope_freq_host, state,
                            workspace, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -159,7 +162,7 @@ int sparkattn_comp_apply(const sparkattn_shape_t* shape, const void* q_bf16, con
   if (!aligned16(q_bf16) || !aligned16(pq_bf16) || !aligned16(state) || !aligned16(o_sparse_bf16) ||
       !aligned16(out_bf16) || !aligned256(workspace))
     return SPARKATTN_E_MISALIGNED;
-  if (workspace_bytes < (size_t)kWorkspaceHeaderBytes) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < comp_workspace_bytes(*shape, grid_host, false)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   return launch_comp_apply(*shape, q_bf16, pq_bf16, grid_host, rope_axis_host, rope_freq_host, state, gate,
                            o_sparse_bf16, out_bf16, eps, workspace, static_cast<cudaStream_t>(cuda_stream));
 }

@@ -44,25 +44,44 @@ struct CompParams {
   const __nv_bfloat16* o_sparse;      // apply
   __nv_bfloat16* out;                 // apply
   float eps;
+  const float2* rope_table;           // [rank/2][rope_stride] (cos, sin)
+  int rope_stride;
   int32_t* status;
 };
 
+// cos/sin of every (rotary pair, coordinate) the grid can produce: table[m * stride + e] =
+// (cos, sin)(e * freq[m]) for e < extent(axis[m]).  A few thousand entries; the feature loops read
+// it through L1 instead of running a full-range sincosf per (token, pair).
+__global__ void rope_table_kernel(const RopeTable rope, float2* __restrict__ table, int stride) {
+  const int m = blockIdx.x;
+  const int ax = rope.axis[m];
+  const int extent = ax == 0 ? rope.T : (ax == 1 ? rope.Hg : rope.Wg);
+  for (int e = threadIdx.x; e < extent; e += blockDim.x) {
+    float sn, cs;
+    sincosf((float)e * rope.freq[m], &sn, &cs);
+    table[m * stride + e] = make_float2(cs, sn);
+  }
+}
+
 // silu, then the rank-truncated rotary rotation of adjacent pairs; v holds the 64 features of one token
-__device__ __forceinline__ void silu_rope(float (&v)[kRank], const RopeTable& rope, int token) {
+__device__ __forceinline__ void silu_rope(float (&v)[kRank], const RopeTable& rope, const float2* __restrict__ table,
+                                          int stride, int token) {
   const int x = token % rope.Wg;
   const int y = (token / rope.Wg) % rope.Hg;
   const int t = token / (rope.Wg * rope.Hg);
+  float2 cs[kRank / 2];
+#pragma unroll
+  for (int m = 0; m < kRank / 2; ++m) {
+    const int ax = rope.axis[m];
+    cs[m] = __ldg(table + m * stride + (ax == 0 ? t : (ax == 1 ? y : x)));
+  }
 #pragma unroll
   for (int a = 0; a < kRank; ++a) v[a] = __fdividef(v[a], 1.0f + __expf(-v[a]));
 #pragma unroll
   for (int m = 0; m < kRank / 2; ++m) {
-    const int ax = rope.axis[m];
-    const float pos = (float)(ax == 0 ? t : (ax == 1 ? y : x));
-    float sn, cs;
-    sincosf(pos * rope.freq[m], &sn, &cs);
     const float z0 = v[2 * m], z1 = v[2 * m + 1];
-    v[2 * m] = z0 * cs - z1 * sn;
-    v[2 * m + 1] = z0 * sn + z1 * cs;
+    v[2 * m] = z0 * cs[m].x - z1 * cs[m].y;
+    v[2 * m + 1] = z0 * cs[m].y + z1 * cs[m].x;
   }
 }
 
@@ -204,7 +223,7 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
 #pragma unroll
         for (int a = 0; a < kRank; ++a) v[a] = __uint_as_float(r[a]);
       }
-      silu_rope(v, p.rope, min((tile0 + i) * kTileTok + row, p.N - 1));   // rows past N are zero anyway
+      silu_rope(v, p.rope, p.rope_table, p.rope_stride, min((tile0 + i) * kTileTok + row, p.N - 1));   // rows past N are zero anyway
       if (i > 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, (i - 1) & 1, s_abort, p.status, 57));   // k~ tile free
         if (!ok) break;
@@ -362,7 +381,7 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         tc_wait_ld();
 #pragma unroll
         for (int a = 0; a < kRank; ++a) v[a] = __uint_as_float(r[a]);
-        silu_rope(v, p.rope, min(token, p.N - 1));
+        silu_rope(v, p.rope, p.rope_table, p.rope_stride, min(token, p.N - 1));
         store_feature_row(sF, row, v);     // the previous tile's Y (which read this buffer) was waited for below
       }
       fence_proxy_async_smem();
@@ -472,8 +491,32 @@ static int state_chunks(const sparkattn_shape_t& s) {
   return (int)want;
 }
 
-size_t comp_workspace_bytes(const sparkattn_shape_t& s) {
-  return kWorkspaceHeaderBytes + (size_t)s.B * s.H * state_chunks(s) * kCD * kRank * sizeof(float);
+static int rope_stride(const int32_t* grid) {
+  int e = grid[0] > grid[1] ? grid[0] : grid[1];
+  if (grid[2] > e) e = grid[2];
+  return (e + 3) / 4 * 4;
+}
+static size_t rope_table_bytes(const int32_t* grid) {
+  return ((size_t)(kRank / 2) * rope_stride(grid) * sizeof(float2) + 255) / 256 * 256;
+}
+
+size_t comp_workspace_bytes(const sparkattn_shape_t& s, const int32_t* grid, bool with_state) {
+  size_t bytes = kWorkspaceHeaderBytes + rope_table_bytes(grid);
+  if (with_state) bytes += (size_t)s.B * s.H * state_chunks(s) * kCD * kRank * sizeof(float);
+  return bytes;
+}
+
+// header | rotary table | (state pass only) per-chunk partial states
+static int prepare_workspace(CompParams& prm, const int32_t* grid, void* workspace, cudaStream_t stream) {
+  char* base = static_cast<char*>(workspace);
+  prm.status = reinterpret_cast<int32_t*>(base);
+  float2* table = reinterpret_cast<float2*>(base + kWorkspaceHeaderBytes);
+  prm.rope_table = table;
+  prm.rope_stride = rope_stride(grid);
+  prm.partial = reinterpret_cast<float*>(base + kWorkspaceHeaderBytes + rope_table_bytes(grid));
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  rope_table_kernel<<<kRank / 2, 128, 0, stream>>>(prm.rope, table, prm.rope_stride);
+  return SPARKATTN_OK;
 }
 
 static void fill_rope(CompParams& prm, const int32_t* grid, const int32_t* axis, const float* freq) {
@@ -495,9 +538,7 @@ int launch_comp_state(const sparkattn_shape_t& s, const void* k, const void* v, 
   prm.nchunks = state_chunks(s);
   prm.tiles_per_cta = (prm.nt + prm.nchunks - 1) / prm.nchunks;
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
-  prm.partial = reinterpret_cast<float*>(static_cast<char*>(workspace) + kWorkspaceHeaderBytes);
-  prm.status = static_cast<int32_t*>(workspace);
-  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  if ((rc = prepare_workspace(prm, grid, workspace, stream)) != SPARKATTN_OK) return rc;
   if (cudaFuncSetAttribute(comp_state_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStateSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const dim3 grid_dim((unsigned)prm.nchunks, (unsigned)(s.B * s.H));
@@ -524,8 +565,7 @@ int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq,
   prm.o_sparse = static_cast<const __nv_bfloat16*>(o_sparse);
   prm.out = static_cast<__nv_bfloat16*>(out);
   prm.eps = eps;
-  prm.status = static_cast<int32_t*>(workspace);
-  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  if ((rc = prepare_workspace(prm, grid, workspace, stream)) != SPARKATTN_OK) return rc;
   if (cudaFuncSetAttribute(comp_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kApplySmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const dim3 grid_dim((unsigned)prm.nchunks, (unsigned)(s.B * s.H));

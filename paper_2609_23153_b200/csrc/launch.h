@@ -32,7 +32,8 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
 
 // comp.cu
 constexpr int kCompRank = 64;  // rank of the compensation branch the kernels are built for
-size_t comp_workspace_bytes(const sparkattn_shape_t& s);
+// header + rotary table (+ the per-chunk partial states of the state pass)
+size_t comp_workspace_bytes(const sparkattn_shape_t& s, const int32_t* grid, bool with_state);
 int launch_comp_state(const sparkattn_shape_t& s, const void* k, const void* v, const void* pk, const int32_t* grid,
                       const int32_t* axis, const float* freq, float* state, void* workspace, cudaStream_t stream);
 int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq, const int32_t* grid,
