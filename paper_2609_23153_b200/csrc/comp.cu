@@ -4,16 +4,20 @@
 // Linear in the sequence length; both passes are streaming and HBM-bound, their contractions
 // (projection to rank r = 64, k~ v^T accumulation, q~ C) run as tcgen05 MMAs with TMEM accumulators.
 //
-//   comp_state_kernel   CTA = one chunk of 128-token tiles of one (batch, head).  Per tile:
-//                       T = K P_k^T (MMA) -> silu + rotary on the T rows (one thread per token)
-//                       -> k~ as bf16 into shared memory -> C^T += V^T k~ (MMA, both operands
-//                       MN-major straight from the row-major tiles).  The chunk's C^T goes to
-//                       the workspace; comp_reduce_kernel adds the chunks in a fixed order.
-//   comp_apply_kernel   CTA = a few 128-token tiles of one (batch, head).  Per tile:
-//                       T = Q P_q^T -> silu + rotary -> q~ (bf16, shared memory) -> Y = q~ C
-//                       (MMA, C as bf16 in shared memory) -> per row RMSNorm, RMS of the sparse
-//                       output row, gate, add, store.
-// Every mbarrier wait is bounded; rows past N are zero tiles (TMA fill) and are never stored.
+// Both kernels run one CTA per SM over a contiguous chunk of 128-token tiles of one (batch, head),
+// with three feature warpgroups that take the tiles round-robin (a thread owns one token row), one
+// TMA producer warp and one MMA-issuing warp:
+//   comp_state_kernel   per tile: T = K P_k^T (MMA) -> silu + rotary on the T rows -> k~ as bf16
+//                       into shared memory -> C^T += V^T k~ (MMA, both operands MN-major straight
+//                       from the row-major tiles).  The chunk's C^T goes to the workspace;
+//                       comp_reduce_kernel adds the chunks in a fixed order.
+//   comp_apply_kernel   per tile: T = Q P_q^T -> silu + rotary -> q~ (bf16, shared memory) ->
+//                       Y = q~ C (MMA, C as bf16 in shared memory; Y overwrites T in TMEM) ->
+//                       per row RMSNorm, RMS of the sparse output row, gate, add, store.
+// The MMA warp polls for whichever product is ready next (projection of a new tile, or the second
+// product of the oldest tile whose features are written), so the three warpgroups, the loads and
+// the tensor pipe overlap.  Every wait is bounded; rows past N are zero tiles (TMA fill) and are
+// never stored.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -21,11 +25,15 @@
 
 namespace sparkattn {
 
-constexpr int kCompThreads = 192;     // warps 0-3: one thread per token row; warp 4: TMA; warp 5: MMA issue
+constexpr int kFeatWGs = 3;
+constexpr int kCompThreads = kFeatWGs * 128 + 128;  // feature warpgroups, then a warpgroup holding the TMA warp and the MMA warp
+constexpr int kFeatRegs = 152, kCtrlRegs = 56;      // register split between the two kinds of warpgroup
+constexpr int kProducerWarp = kFeatWGs * 4;
+constexpr int kMmaWarp = kFeatWGs * 4 + 1;
 constexpr int kRank = 64;
 constexpr int kCD = 128;              // head dimension handled by this file
 constexpr int kTileTok = 128;
-constexpr int kApplyTilesPerCta = 4;
+constexpr int kNumSMs = 148;          // chunking target (B200); any other count only changes the balance
 
 struct RopeTable {
   int32_t axis[kRank / 2];            // 0 = t, 1 = y, 2 = x
@@ -63,44 +71,48 @@ __global__ void rope_table_kernel(const RopeTable rope, float2* __restrict__ tab
   }
 }
 
-// silu, then the rank-truncated rotary rotation of adjacent pairs; v holds the 64 features of one token
-__device__ __forceinline__ void silu_rope(float (&v)[kRank], const RopeTable& rope, const float2* __restrict__ table,
-                                          int stride, int token) {
-  const int x = token % rope.Wg;
-  const int y = (token / rope.Wg) % rope.Hg;
-  const int t = token / (rope.Wg * rope.Hg);
-  float2 cs[kRank / 2];
-#pragma unroll
-  for (int m = 0; m < kRank / 2; ++m) {
-    const int ax = rope.axis[m];
-    cs[m] = __ldg(table + m * stride + (ax == 0 ? t : (ax == 1 ? y : x)));
-  }
-#pragma unroll
-  for (int a = 0; a < kRank; ++a) v[a] = __fdividef(v[a], 1.0f + __expf(-v[a]));
-#pragma unroll
-  for (int m = 0; m < kRank / 2; ++m) {
-    const float z0 = v[2 * m], z1 = v[2 * m + 1];
-    v[2 * m] = z0 * cs[m].x - z1 * cs[m].y;
-    v[2 * m + 1] = z0 * cs[m].y + z1 * cs[m].x;
-  }
-}
-
-// one token's 64 features as bf16 into row `row` of a [128 rows x 128 B] tile with 128-byte swizzle
-__device__ __forceinline__ void store_feature_row(unsigned char* tile, int row, const float (&v)[kRank]) {
-#pragma unroll
-  for (int c = 0; c < 8; ++c) {
-    uint32_t w[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[8 * c + 2 * j], v[8 * c + 2 * j + 1]);
-      w[j] = *reinterpret_cast<const uint32_t*>(&h2);
-    }
-    *reinterpret_cast<uint4*>(tile + row * 128 + ((c ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-  }
-}
-
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// One token row of T (64 fp32 columns at `taddr`) -> silu -> rank-truncated rotary rotation of the
+// adjacent pairs -> bf16 -> row `row` of a [128 rows x 128 B] tile with 128-byte swizzle.
+// Done in two halves of 32 columns to bound the live registers.
+__device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile, int row, const RopeTable& rope,
+                                            const float2* __restrict__ table, int stride, int token) {
+  const int x = token % rope.Wg;
+  const int yy = token / rope.Wg;
+  const int y = yy % rope.Hg;
+  const int t = yy / rope.Hg;
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    uint32_t r[32];
+    tmem_ld32(taddr + half * 32, r);
+    float2 cs[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int m = half * 16 + j;
+      const int ax = rope.axis[m];
+      cs[j] = __ldg(table + m * stride + (ax == 0 ? t : (ax == 1 ? y : x)));
+    }
+    tc_wait_ld();
+    uint32_t w[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float u0 = __uint_as_float(r[2 * j]), u1 = __uint_as_float(r[2 * j + 1]);
+      const float2 e = unpack_f32x2(fadd2(pack_f32x2(fast_exp2(u0 * -1.4426950408889634f), fast_exp2(u1 * -1.4426950408889634f)),
+                                          pack_f32x2(1.0f, 1.0f)));
+      const float z0 = __fdividef(u0, e.x), z1 = __fdividef(u1, e.y);
+      const float o0 = fmaf(z0, cs[j].x, -z1 * cs[j].y);
+      const float o1 = fmaf(z0, cs[j].y, z1 * cs[j].x);
+      const __nv_bfloat162 h2 = __floats2bfloat162_rn(o0, o1);
+      w[j] = *reinterpret_cast<const uint32_t*>(&h2);
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      *reinterpret_cast<uint4*>(tile + row * 128 + (((half * 4 + c) ^ (row & 7)) << 4)) =
+          make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+  }
 }
 
 // instruction descriptor with both major bits explicit (bf16 in, fp32 accumulate)
@@ -122,27 +134,56 @@ __device__ __forceinline__ void issue_projection(uint32_t tmem_T, uint32_t x_sme
                     make_desc(p_lo + ((s * 8192 + kk * 32) >> 4), p_hi), idesc, (s | kk) != 0 ? 1u : 0u);
 }
 
-constexpr int kStateSmem = 1024 + 16384 /*P*/ + 32768 /*K*/ + 32768 /*V*/ + 16384 /*k~*/ + 256;
-constexpr int kApplySmem = 1024 + 16384 /*P*/ + 16384 /*C*/ + 32768 /*Q*/ + 16384 /*q~*/ + 256;
+// Idle bookkeeping of the polling MMA warp: false once the CTA was aborted or nothing became ready
+// for kWaitLimitNs.
+struct IdleGuard {
+  uint64_t t0;
+  uint32_t polls;
+  __device__ __forceinline__ void reset() { polls = 0; }
+  __device__ __forceinline__ bool idle(volatile int* abort_flag, int32_t* status, int wait_id) {
+    if (polls == 0) t0 = global_timer_ns();
+    if ((++polls & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        report_status(status, SPARKATTN_E_DEVICE_TIMEOUT, wait_id);
+        return false;
+      }
+    }
+    return true;
+  }
+};
 
-__global__ void __launch_bounds__(kCompThreads, 2)
+// state kernel shared memory: P | K ring (2) | V ring (2) | k~ tiles (one per warpgroup) | barriers
+constexpr int kStateOffK = 16384, kStateOffV = kStateOffK + 2 * 32768, kStateOffF = kStateOffV + 2 * 32768;
+constexpr int kStateOffBar = kStateOffF + kFeatWGs * 16384;
+constexpr int kStateSmem = 1024 + kStateOffBar + 256;
+// apply kernel shared memory: P | C | Q ring (3) | q~ tiles | barriers
+constexpr int kApplyOffC = 16384, kApplyOffQ = 32768, kApplyOffF = kApplyOffQ + kFeatWGs * 32768;
+constexpr int kApplyOffBar = kApplyOffF + kFeatWGs * 16384;
+constexpr int kApplySmem = 1024 + kApplyOffBar + 256;
+
+__global__ void __launch_bounds__(kCompThreads, 1)
 comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                   const __grid_constant__ CUtensorMap tmap_p, const CompParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* sP = smem;
-  unsigned char* sK = sP + 16384;
-  unsigned char* sV = sK + 32768;
-  unsigned char* sF = sV + 32768;                 // k~ tile: [128 tokens][64] bf16
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sF + 16384);
+  unsigned char* sK = smem + kStateOffK;
+  unsigned char* sV = smem + kStateOffV;
+  unsigned char* sF = smem + kStateOffF;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStateOffBar);
   uint64_t* bar_p_full = bars + 0;
-  uint64_t* bar_k_full = bars + 1;
-  uint64_t* bar_v_full = bars + 2;
-  uint64_t* bar_t_full = bars + 3;                // projection done (also: K slot free)
-  uint64_t* bar_f_full = bars + 4;                // features written by all 128 threads
-  uint64_t* bar_acc = bars + 5;                   // accumulation MMA done (also: V slot and k~ tile free)
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 6);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 7);
+  uint64_t* bar_k_full = bars + 1;    // [2] TMA landed
+  uint64_t* bar_k_empty = bars + 3;   // [2] projection MMAs done
+  uint64_t* bar_v_full = bars + 5;    // [2]
+  uint64_t* bar_v_empty = bars + 7;   // [2] accumulation MMAs done
+  uint64_t* bar_t_full = bars + 9;    // [3] projection of a tile in T[g]
+  uint64_t* bar_f_full = bars + 12;   // [3] k~ tile g written (128 arrivals)
+  uint64_t* bar_f_empty = bars + 15;  // [3] accumulation MMAs that read k~ tile g done
+  uint64_t* bar_acc = bars + 18;      // everything issued is complete
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 20);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 21);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x, bh = blockIdx.y;
@@ -151,94 +192,115 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
   const int ntiles = max(0, min(p.tiles_per_cta, p.nt - tile0));
 
   if (threadIdx.x == 0) {
-    mbar_init(bar_p_full, 1); mbar_init(bar_k_full, 1); mbar_init(bar_v_full, 1);
-    mbar_init(bar_t_full, 1); mbar_init(bar_f_full, 128); mbar_init(bar_acc, 1);
+    mbar_init(bar_p_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_k_full + i, 1); mbar_init(bar_k_empty + i, 1);
+      mbar_init(bar_v_full + i, 1); mbar_init(bar_v_empty + i, 1);
+    }
+    for (int g = 0; g < kFeatWGs; ++g) {
+      mbar_init(bar_t_full + g, 1); mbar_init(bar_f_full + g, 128); mbar_init(bar_f_empty + g, 1);
+    }
+    mbar_init(bar_acc, 1);
     *s_abort = 0;
     mbar_fence_init();
   }
-  if (warp == 4) {
-    tmem_alloc(s_tmem, 128);
+  if (warp == kProducerWarp) {
+    tmem_alloc(s_tmem, 256);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
-  const uint32_t tmem_T = tmem, tmem_C = tmem + 64;
+  const uint32_t tmem_C = tmem + kFeatWGs * 64;    // T[g] at column 64 g, C^T behind them
 
-  if (warp == 4) {
+  if (warp >= kProducerWarp) reg_dec<kCtrlRegs>();
+  if (warp == kProducerWarp) {
     if (lane == 0 && ntiles > 0) {
       mbar_expect_tx(bar_p_full, 16384);
       tma_load_4d(sP, &tmap_p, bar_p_full, 0, 0, h, 0);
       tma_load_4d(sP + 8192, &tmap_p, bar_p_full, 64, 0, h, 0);
       for (int i = 0; i < ntiles; ++i) {
-        const int row = (tile0 + i) * kTileTok;
-        if (i > 0 && !mbar_wait(bar_t_full, (i - 1) & 1, s_abort, p.status, 50)) break;
-        mbar_expect_tx(bar_k_full, 32768);
-        tma_load_4d(sK, &tmap_k, bar_k_full, 0, row, h, b);
-        tma_load_4d(sK + 16384, &tmap_k, bar_k_full, 64, row, h, b);
-        if (i > 0 && !mbar_wait(bar_acc, (i - 1) & 1, s_abort, p.status, 51)) break;
-        mbar_expect_tx(bar_v_full, 32768);
-        tma_load_4d(sV, &tmap_v, bar_v_full, 0, row, h, b);
-        tma_load_4d(sV + 16384, &tmap_v, bar_v_full, 64, row, h, b);
+        const int row = (tile0 + i) * kTileTok, st = i & 1, n = i >> 1;
+        if (n > 0 && !mbar_wait(bar_k_empty + st, (n - 1) & 1, s_abort, p.status, 50)) break;
+        mbar_expect_tx(bar_k_full + st, 32768);
+        tma_load_4d(sK + st * 32768, &tmap_k, bar_k_full + st, 0, row, h, b);
+        tma_load_4d(sK + st * 32768 + 16384, &tmap_k, bar_k_full + st, 64, row, h, b);
+        if (n > 0 && !mbar_wait(bar_v_empty + st, (n - 1) & 1, s_abort, p.status, 51)) break;
+        mbar_expect_tx(bar_v_full + st, 32768);
+        tma_load_4d(sV + st * 32768, &tmap_v, bar_v_full + st, 0, row, h, b);
+        tma_load_4d(sV + st * 32768 + 16384, &tmap_v, bar_v_full + st, 64, row, h, b);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     if (lane == 0 && ntiles > 0) {
       // C^T[128 d x 64 r] += V^T k~ : A = V tile (MN-major: d contiguous, two 64-column slabs),
       // B = k~ tile (MN-major: r contiguous), 16 tokens per MMA
-      const uint64_t dV = make_smem_desc_sw128(smem_u32(sV), 16384), dF = make_smem_desc_sw128(smem_u32(sF), 16);
-      const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32), f_lo = (uint32_t)dF, f_hi = (uint32_t)(dF >> 32);
       constexpr uint32_t idesc_acc = comp_idesc(128, kRank, true, true);
       bool ok = mbar_wait(bar_p_full, 0, s_abort, p.status, 52);
-      for (int i = 0; ok && i < ntiles; ++i) {
-        if (!(ok = mbar_wait(bar_k_full, i & 1, s_abort, p.status, 53))) break;
-        tc_fence_after();
-        issue_projection(tmem_T, smem_u32(sK), smem_u32(sP));
-        tc_commit(bar_t_full);
-        if (!(ok = mbar_wait(bar_v_full, i & 1, s_abort, p.status, 54))) break;
-        if (!(ok = mbar_wait(bar_f_full, i & 1, s_abort, p.status, 55))) break;
-        tc_fence_after();
+      int s1 = 0, s2 = 0;              // next tile to project / to accumulate
+      IdleGuard guard;
+      guard.reset();
+      while (ok && s2 < ntiles) {
+        bool progressed = false;
+        // T[s1 % 3] is free once the features of tile s1 - 3 were consumed, i.e. s2 > s1 - 3
+        if (s1 < ntiles && s1 - s2 < kFeatWGs && mbar_try_wait(bar_k_full + (s1 & 1), (s1 >> 1) & 1)) {
+          tc_fence_after();
+          issue_projection(tmem + (s1 % kFeatWGs) * 64, smem_u32(sK + (s1 & 1) * 32768), smem_u32(sP));
+          tc_commit(bar_t_full + s1 % kFeatWGs);
+          tc_commit(bar_k_empty + (s1 & 1));
+          ++s1;
+          progressed = true;
+        }
+        if (s2 < s1 && mbar_try_wait(bar_f_full + s2 % kFeatWGs, (s2 / kFeatWGs) & 1) &&
+            mbar_try_wait(bar_v_full + (s2 & 1), (s2 >> 1) & 1)) {
+          tc_fence_after();
+          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + (s2 & 1) * 32768), 16384);
+          const uint64_t dF = make_smem_desc_sw128(smem_u32(sF + (s2 % kFeatWGs) * 16384), 16);
+          const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32), f_lo = (uint32_t)dF, f_hi = (uint32_t)(dF >> 32);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          mma_ss<false>(tmem_C, make_desc(v_lo + ((kk * 2048) >> 4), v_hi), make_desc(f_lo + ((kk * 2048) >> 4), f_hi),
-                        idesc_acc, (i | kk) != 0 ? 1u : 0u);
-        tc_commit(bar_acc);
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ss<false>(tmem_C, make_desc(v_lo + ((kk * 2048) >> 4), v_hi), make_desc(f_lo + ((kk * 2048) >> 4), f_hi),
+                          idesc_acc, (s2 | kk) != 0 ? 1u : 0u);
+          tc_commit(bar_v_empty + (s2 & 1));
+          tc_commit(bar_f_empty + s2 % kFeatWGs);
+          ++s2;
+          progressed = true;
+        }
+        if (progressed) guard.reset();
+        else ok = guard.idle(s_abort, p.status, 53);
       }
+      if (ok) tc_commit(bar_acc);
     }
-  } else {
-    const int row = threadIdx.x;                       // token row of the tile = TMEM lane
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+  } else if (warp < kProducerWarp) {
+    reg_inc<kFeatRegs>();
+    const int g = warp >> 2;                              // warpgroup = tile slot
+    const int row = threadIdx.x & 127;                    // token row of the tile = TMEM lane
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    unsigned char* tileF = sF + g * 16384;
     bool ok = true;
-    for (int i = 0; ok && i < ntiles; ++i) {
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full, i & 1, s_abort, p.status, 56));
+    for (int i = g, u = 0; ok && i < ntiles; i += kFeatWGs, ++u) {
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full + g, u & 1, s_abort, p.status, 56));
       if (!ok) break;
-      tc_fence_after();
-      float v[kRank];
-      {
-        uint32_t r[kRank];
-        tmem_ld32(tmem_T + lane_off, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-        tmem_ld32(tmem_T + lane_off + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-        tc_wait_ld();
-#pragma unroll
-        for (int a = 0; a < kRank; ++a) v[a] = __uint_as_float(r[a]);
-      }
-      silu_rope(v, p.rope, p.rope_table, p.rope_stride, min((tile0 + i) * kTileTok + row, p.N - 1));   // rows past N are zero anyway
-      if (i > 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, (i - 1) & 1, s_abort, p.status, 57));   // k~ tile free
+      if (u > 0) {                                        // k~ tile g still read by the previous accumulation?
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_f_empty + g, (u - 1) & 1, s_abort, p.status, 57));
         if (!ok) break;
       }
-      store_feature_row(sF, row, v);
+      tc_fence_after();
+      feature_row(tmem + g * 64 + lane_off, tileF, row, p.rope, p.rope_table, p.rope_stride,
+                  min((tile0 + i) * kTileTok + row, p.N - 1));       // rows past N are zero anyway
       fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(bar_f_full);
+      mbar_arrive(bar_f_full + g);
     }
-    if (ok && ntiles > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, (ntiles - 1) & 1, s_abort, p.status, 58));
-      if (ok) {
+    if (g == 0) {
+      float* dst = p.partial + (((int64_t)bh * p.nchunks + chunk) * kCD + row) * kRank;
+      if (ntiles == 0) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) reinterpret_cast<uint4*>(dst)[j] = make_uint4(0u, 0u, 0u, 0u);
+      } else if (ok && __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, s_abort, p.status, 58))) {
         tc_fence_after();
         // thread = channel c of d; its TMEM row holds C^T[c][0..63]
-        float* dst = p.partial + (((int64_t)bh * p.nchunks + chunk) * kCD + row) * kRank;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           uint32_t r[32];
@@ -249,18 +311,14 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
             reinterpret_cast<uint4*>(dst + half * 32)[j] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
         }
       }
-    } else if (ntiles == 0) {
-      float* dst = p.partial + (((int64_t)bh * p.nchunks + chunk) * kCD + row) * kRank;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) reinterpret_cast<uint4*>(dst)[j] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     if (*s_abort) __nanosleep(200000);
     tc_fence_after();
-    tmem_dealloc(tmem, 128);
+    tmem_dealloc(tmem, 256);
   }
 }
 
@@ -275,23 +333,26 @@ __global__ void comp_reduce_kernel(const float* __restrict__ partial, float* __r
   }
 }
 
-__global__ void __launch_bounds__(kCompThreads, 2)
+__global__ void __launch_bounds__(kCompThreads, 1)
 comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_p,
                   const CompParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* sP = smem;
-  unsigned char* sC = sP + 16384;                 // C as bf16, [64 r rows][128 d], two 64-column slabs of 8 KB
-  unsigned char* sQ = sC + 16384;
-  unsigned char* sF = sQ + 32768;                 // q~ tile: [128 tokens][64] bf16
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sF + 16384);
+  unsigned char* sC = smem + kApplyOffC;           // C as bf16, [64 r rows][128 d], two 64-column slabs of 8 KB
+  unsigned char* sQ = smem + kApplyOffQ;           // ring of 3, stage = tile % 3
+  unsigned char* sF = smem + kApplyOffF;           // q~ tiles, one per warpgroup
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kApplyOffBar);
   uint64_t* bar_p_full = bars + 0;
-  uint64_t* bar_q_full = bars + 1;
-  uint64_t* bar_t_full = bars + 2;                // projection done (also: Q slot free)
-  uint64_t* bar_f_full = bars + 3;                // q~ written by all 128 threads (first use: C staged too)
-  uint64_t* bar_y_full = bars + 4;                // Y = q~ C done
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 6);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 7);
+  uint64_t* bar_c_full = bars + 1;                 // C staged (128 arrivals)
+  uint64_t* bar_q_full = bars + 2;                 // [3]
+  uint64_t* bar_q_empty = bars + 5;                // [3] projection MMAs done
+  uint64_t* bar_t_full = bars + 8;                 // [3]
+  uint64_t* bar_f_full = bars + 11;                // [3] q~ tile written (128 arrivals)
+  uint64_t* bar_y_full = bars + 14;                // [3] Y = q~ C done
+  uint64_t* bar_y_empty = bars + 17;               // [3] epilogue has read Y (128 arrivals)
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 20);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 21);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = blockIdx.y;
@@ -300,105 +361,128 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   const int ntiles = max(0, min(p.tiles_per_cta, p.nt - tile0));
 
   if (threadIdx.x == 0) {
-    mbar_init(bar_p_full, 1); mbar_init(bar_q_full, 1); mbar_init(bar_t_full, 1);
-    mbar_init(bar_f_full, 128); mbar_init(bar_y_full, 1);
+    mbar_init(bar_p_full, 1);
+    mbar_init(bar_c_full, 128);
+    for (int g = 0; g < kFeatWGs; ++g) {
+      mbar_init(bar_q_full + g, 1); mbar_init(bar_q_empty + g, 1); mbar_init(bar_t_full + g, 1);
+      mbar_init(bar_f_full + g, 128); mbar_init(bar_y_full + g, 1); mbar_init(bar_y_empty + g, 128);
+    }
     *s_abort = 0;
     mbar_fence_init();
   }
-  if (warp == 4) {
-    tmem_alloc(s_tmem, 256);
+  if (warp == kProducerWarp) {
+    tmem_alloc(s_tmem, 512);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *s_tmem;
-  const uint32_t tmem_T = tmem, tmem_Y = tmem + 64;
+  const uint32_t tmem = *s_tmem;                   // warpgroup g: columns [128 g, 128 g + 128): T in the first 64, then Y over all
 
-  if (warp == 4) {
+  if (warp >= kProducerWarp) reg_dec<kCtrlRegs>();
+  if (warp == kProducerWarp) {
     if (lane == 0 && ntiles > 0) {
       mbar_expect_tx(bar_p_full, 16384);
       tma_load_4d(sP, &tmap_p, bar_p_full, 0, 0, h, 0);
       tma_load_4d(sP + 8192, &tmap_p, bar_p_full, 64, 0, h, 0);
       for (int i = 0; i < ntiles; ++i) {
-        const int row = (tile0 + i) * kTileTok;
-        if (i > 0 && !mbar_wait(bar_t_full, (i - 1) & 1, s_abort, p.status, 60)) break;
-        mbar_expect_tx(bar_q_full, 32768);
-        tma_load_4d(sQ, &tmap_q, bar_q_full, 0, row, h, b);
-        tma_load_4d(sQ + 16384, &tmap_q, bar_q_full, 64, row, h, b);
+        const int row = (tile0 + i) * kTileTok, st = i % kFeatWGs, n = i / kFeatWGs;
+        if (n > 0 && !mbar_wait(bar_q_empty + st, (n - 1) & 1, s_abort, p.status, 60)) break;
+        mbar_expect_tx(bar_q_full + st, 32768);
+        tma_load_4d(sQ + st * 32768, &tmap_q, bar_q_full + st, 0, row, h, b);
+        tma_load_4d(sQ + st * 32768 + 16384, &tmap_q, bar_q_full + st, 64, row, h, b);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     if (lane == 0 && ntiles > 0) {
       // Y[128 tokens x 128 d] = q~ C : A = q~ tile (K-major: r contiguous), B = C (MN-major: d contiguous, two slabs)
-      const uint64_t dF = make_smem_desc_sw128(smem_u32(sF), 16), dC = make_smem_desc_sw128(smem_u32(sC), 8192);
-      const uint32_t f_lo = (uint32_t)dF, f_hi = (uint32_t)(dF >> 32), c_lo = (uint32_t)dC, c_hi = (uint32_t)(dC >> 32);
+      const uint64_t dC = make_smem_desc_sw128(smem_u32(sC), 8192);
+      const uint32_t c_lo = (uint32_t)dC, c_hi = (uint32_t)(dC >> 32);
       constexpr uint32_t idesc_y = comp_idesc(128, kCD, false, true);
-      bool ok = mbar_wait(bar_p_full, 0, s_abort, p.status, 61);
-      for (int i = 0; ok && i < ntiles; ++i) {
-        if (!(ok = mbar_wait(bar_q_full, i & 1, s_abort, p.status, 62))) break;
-        tc_fence_after();
-        issue_projection(tmem_T, smem_u32(sQ), smem_u32(sP));
-        tc_commit(bar_t_full);
-        if (!(ok = mbar_wait(bar_f_full, i & 1, s_abort, p.status, 63))) break;
-        tc_fence_after();
+      bool ok = mbar_wait(bar_p_full, 0, s_abort, p.status, 61) && mbar_wait(bar_c_full, 0, s_abort, p.status, 62);
+      int s1 = 0, s2 = 0;
+      IdleGuard guard;
+      guard.reset();
+      while (ok && s2 < ntiles) {
+        bool progressed = false;
+        const int g1 = s1 % kFeatWGs, n1 = s1 / kFeatWGs;
+        // the projection of tile s1 overwrites the Y columns of tile s1 - 3: its epilogue must be done
+        if (s1 < ntiles && mbar_try_wait(bar_q_full + g1, n1 & 1) &&
+            (n1 == 0 || mbar_try_wait(bar_y_empty + g1, (n1 - 1) & 1))) {
+          tc_fence_after();
+          issue_projection(tmem + g1 * 128, smem_u32(sQ + g1 * 32768), smem_u32(sP));
+          tc_commit(bar_t_full + g1);
+          tc_commit(bar_q_empty + g1);
+          ++s1;
+          progressed = true;
+        }
+        const int g2 = s2 % kFeatWGs;
+        if (s2 < s1 && mbar_try_wait(bar_f_full + g2, (s2 / kFeatWGs) & 1)) {
+          tc_fence_after();
+          const uint64_t dF = make_smem_desc_sw128(smem_u32(sF + g2 * 16384), 16);
+          const uint32_t f_lo = (uint32_t)dF, f_hi = (uint32_t)(dF >> 32);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          mma_ss<false>(tmem_Y, make_desc(f_lo + ((kk * 32) >> 4), f_hi), make_desc(c_lo + ((kk * 2048) >> 4), c_hi),
-                        idesc_y, kk != 0 ? 1u : 0u);
-        tc_commit(bar_y_full);
+          for (int kk = 0; kk < 4; ++kk)
+            mma_ss<false>(tmem + g2 * 128, make_desc(f_lo + ((kk * 32) >> 4), f_hi),
+                          make_desc(c_lo + ((kk * 2048) >> 4), c_hi), idesc_y, kk != 0 ? 1u : 0u);
+          tc_commit(bar_y_full + g2);
+          ++s2;
+          progressed = true;
+        }
+        if (progressed) guard.reset();
+        else ok = guard.idle(s_abort, p.status, 63);
       }
     }
-  } else {
-    const int row = threadIdx.x;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    if (ntiles > 0) {
-      // stage C: thread j converts row a = j/2, columns [64*(j%2), +64) of the fp32 state to bf16
-      const int a = row >> 1, half = row & 1;
-      const float* src = p.state + ((int64_t)bh * kRank + a) * kCD + half * 64;
+  } else if (warp < kProducerWarp) {
+    reg_inc<kFeatRegs>();
+    const int g = warp >> 2;
+    const int row = threadIdx.x & 127;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    unsigned char* tileF = sF + g * 16384;
+    const uint32_t tmem_g = tmem + g * 128 + lane_off;
+    if (g == 0) {
+      if (ntiles > 0) {
+        // stage C: thread j converts row a = j/2, columns [64*(j%2), +64) of the fp32 state to bf16
+        const int a = row >> 1, half = row & 1;
+        const float* src = p.state + ((int64_t)bh * kRank + a) * kCD + half * 64;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float4 lo = __ldg(reinterpret_cast<const float4*>(src + 8 * c));
-        const float4 hi = __ldg(reinterpret_cast<const float4*>(src + 8 * c + 4));
-        const __nv_bfloat162 h0 = __floats2bfloat162_rn(lo.x, lo.y), h1 = __floats2bfloat162_rn(lo.z, lo.w);
-        const __nv_bfloat162 h2 = __floats2bfloat162_rn(hi.x, hi.y), h3 = __floats2bfloat162_rn(hi.z, hi.w);
-        *reinterpret_cast<uint4*>(sC + half * 8192 + a * 128 + ((c ^ (a & 7)) << 4)) =
-            make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
-                       *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+        for (int c = 0; c < 8; ++c) {
+          const float4 lo = __ldg(reinterpret_cast<const float4*>(src + 8 * c));
+          const float4 hi = __ldg(reinterpret_cast<const float4*>(src + 8 * c + 4));
+          const __nv_bfloat162 h0 = __floats2bfloat162_rn(lo.x, lo.y), h1 = __floats2bfloat162_rn(lo.z, lo.w);
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(hi.x, hi.y), h3 = __floats2bfloat162_rn(hi.z, hi.w);
+          *reinterpret_cast<uint4*>(sC + half * 8192 + a * 128 + ((c ^ (a & 7)) << 4)) =
+              make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                         *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+        }
+        fence_proxy_async_smem();
       }
+      mbar_arrive(bar_c_full);
     }
     bool ok = true;
-    for (int i = 0; ok && i < ntiles; ++i) {
+    for (int i = g, u = 0; ok && i < ntiles; i += kFeatWGs, ++u) {
       const int token = (tile0 + i) * kTileTok + row;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full, i & 1, s_abort, p.status, 64));
+      const bool valid = token < p.N;
+      const int tok_c = min(token, p.N - 1);
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full + g, u & 1, s_abort, p.status, 64));
       if (!ok) break;
       tc_fence_after();
-      {
-        float v[kRank];
-        uint32_t r[kRank];
-        tmem_ld32(tmem_T + lane_off, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-        tmem_ld32(tmem_T + lane_off + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-        tc_wait_ld();
-#pragma unroll
-        for (int a = 0; a < kRank; ++a) v[a] = __uint_as_float(r[a]);
-        silu_rope(v, p.rope, p.rope_table, p.rope_stride, min(token, p.N - 1));
-        store_feature_row(sF, row, v);     // the previous tile's Y (which read this buffer) was waited for below
-      }
+      // the previous tile of this warpgroup has passed its Y wait, so the q~ tile is free
+      feature_row(tmem_g, tileF, row, p.rope, p.rope_table, p.rope_stride, tok_c);
       fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(bar_f_full);
+      mbar_arrive(bar_f_full + g);
 
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_y_full, i & 1, s_abort, p.status, 65));
-      if (!ok) break;
-      tc_fence_after();
-      const bool valid = token < p.N;
-      const int64_t off = b * p.stride_b + h * p.stride_h + (int64_t)min(token, p.N - 1) * p.stride_n;
-      // RMS of the sparse-branch row and the gate
+      // sparse-branch row and gate, loaded while the second product runs
+      const int64_t off = b * p.stride_b + h * p.stride_h + (int64_t)tok_c * p.stride_n;
       uint4 os[16];
       float so = 0.0f;
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
+      for (int c = 0; c < 16; ++c)
         os[c] = valid ? __ldg(reinterpret_cast<const uint4*>(p.o_sparse + off) + c) : make_uint4(0u, 0u, 0u, 0u);
+      const float gte = valid ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
         const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&os[c]);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -406,22 +490,24 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
           so = fmaf(f.x, f.x, fmaf(f.y, f.y, so));
         }
       }
-      const float g = valid ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_y_full + g, u & 1, s_abort, p.status, 65));
+      if (!ok) break;
+      tc_fence_after();
       // two passes over Y in TMEM: sum of squares, then the fused output
       float ss = 0.0f;
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t r[32];
-        tmem_ld32(tmem_Y + lane_off + ch * 32, r);
+        tmem_ld32(tmem_g + ch * 32, r);
         tc_wait_ld();
 #pragma unroll
         for (int j = 0; j < 32; ++j) ss = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ss);
       }
-      const float coef = g * sqrtf(so * (1.0f / kCD)) * rsqrtf(ss * (1.0f / kCD) + p.eps);
+      const float coef = gte * sqrtf(so * (1.0f / kCD)) * rsqrtf(ss * (1.0f / kCD) + p.eps);
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t r[32];
-        tmem_ld32(tmem_Y + lane_off + ch * 32, r);
+        tmem_ld32(tmem_g + ch * 32, r);
         tc_wait_ld();
         if (valid) {
 #pragma unroll
@@ -440,14 +526,15 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         }
       }
       tc_fence_before();
+      mbar_arrive(bar_y_empty + g);
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     if (*s_abort) __nanosleep(200000);
     tc_fence_after();
-    tmem_dealloc(tmem, 256);
+    tmem_dealloc(tmem, 512);
   }
 }
 
@@ -482,13 +569,24 @@ static int comp_map(CUtensorMap* map, const void* base, cuuint64_t d0, cuuint64_
   return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
-static int state_chunks(const sparkattn_shape_t& s) {
+// Chunks of token tiles per (batch, head): CTAs = B*H*chunks should fill whole waves of one CTA per
+// SM.  Takes the smallest wave count whose last wave is at least 90 % full (else the fullest).
+static int comp_chunks(const sparkattn_shape_t& s) {
   const int nt = (s.N + kTileTok - 1) / kTileTok;
   const long long bh = (long long)s.B * s.H;
-  long long want = (296 + bh - 1) / bh;        // about two CTAs per SM of a 148-SM part
-  if (want < 1) want = 1;
-  if (want > nt) want = nt;
-  return (int)want;
+  int best = 1;
+  double best_fill = 0.0;
+  for (int waves = 1; waves <= 6; ++waves) {
+    long long nch = (long long)kNumSMs * waves / bh;
+    if (nch < 1) continue;
+    if (nch > nt) nch = nt;
+    const int tpc = (int)((nt + nch - 1) / nch);
+    nch = (nt + tpc - 1) / tpc;
+    const double fill = (double)(bh * nch) / ((double)kNumSMs * waves);
+    if (fill > best_fill + 1e-9) { best_fill = fill; best = (int)nch; }
+    if (fill >= 0.9) break;
+  }
+  return best;
 }
 
 static int rope_stride(const int32_t* grid) {
@@ -502,7 +600,7 @@ static size_t rope_table_bytes(const int32_t* grid) {
 
 size_t comp_workspace_bytes(const sparkattn_shape_t& s, const int32_t* grid, bool with_state) {
   size_t bytes = kWorkspaceHeaderBytes + rope_table_bytes(grid);
-  if (with_state) bytes += (size_t)s.B * s.H * state_chunks(s) * kCD * kRank * sizeof(float);
+  if (with_state) bytes += (size_t)s.B * s.H * comp_chunks(s) * kCD * kRank * sizeof(float);
   return bytes;
 }
 
@@ -535,7 +633,7 @@ int launch_comp_state(const sparkattn_shape_t& s, const void* k, const void* v, 
   CompParams prm{};
   fill_rope(prm, grid, axis, freq);
   prm.H = s.H; prm.N = s.N; prm.nt = (s.N + kTileTok - 1) / kTileTok;
-  prm.nchunks = state_chunks(s);
+  prm.nchunks = comp_chunks(s);
   prm.tiles_per_cta = (prm.nt + prm.nchunks - 1) / prm.nchunks;
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
   if ((rc = prepare_workspace(prm, grid, workspace, stream)) != SPARKATTN_OK) return rc;
@@ -558,8 +656,8 @@ int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq,
   CompParams prm{};
   fill_rope(prm, grid, axis, freq);
   prm.H = s.H; prm.N = s.N; prm.nt = (s.N + kTileTok - 1) / kTileTok;
-  prm.tiles_per_cta = kApplyTilesPerCta;
-  prm.nchunks = (prm.nt + kApplyTilesPerCta - 1) / kApplyTilesPerCta;
+  prm.tiles_per_cta = (prm.nt + comp_chunks(s) - 1) / comp_chunks(s);
+  prm.nchunks = (prm.nt + prm.tiles_per_cta - 1) / prm.tiles_per_cta;
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
   prm.state = state; prm.gate = gate;
   prm.o_sparse = static_cast<const __nv_bfloat16*>(o_sparse);
