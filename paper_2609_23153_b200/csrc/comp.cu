@@ -13,7 +13,8 @@
 //                       comp_reduce_kernel adds the chunks in a fixed order.
 //   comp_apply_kernel   per tile: T = Q P_q^T -> silu + rotary -> q~ (bf16, shared memory) ->
 //                       Y = q~ C (MMA, C as bf16 in shared memory; Y overwrites T in TMEM) ->
-//                       per row RMSNorm, RMS of the sparse output row, gate, add, store.
+//                       per row RMSNorm, RMS of the sparse output row (a TMA tile in the slot the
+//                       Q tile used), gate, add in place, TMA store.
 // The MMA warp polls for whichever product is ready next (projection of a new tile, or the second
 // product of the oldest tile whose features are written), so the three warpgroups, the loads and
 // the tensor pipe overlap.  Every wait is bounded; rows past N are zero tiles (TMA fill) and are
@@ -333,26 +334,45 @@ __global__ void comp_reduce_kernel(const float* __restrict__ partial, float* __r
   }
 }
 
+// TMA store of a [128 rows x 64 columns] bf16 slab from shared memory (rows past the tensor's end are clipped)
+__device__ __forceinline__ void tma_store_4d(const void* tmap, const void* smem_src, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+      ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// A ring slot of the apply kernel lives through: Q tile (TMA) -> projection MMAs -> sparse-branch
+// tile O_s (TMA into the same bytes) -> fused output written in place by the warpgroup -> TMA
+// store -> free.  Slot = warpgroup = tile % 3, so all global traffic of the tile is bulk copies.
 __global__ void __launch_bounds__(kCompThreads, 1)
 comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_p,
+                  const __grid_constant__ CUtensorMap tmap_os, const __grid_constant__ CUtensorMap tmap_out,
                   const CompParams p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* sP = smem;
   unsigned char* sC = smem + kApplyOffC;           // C as bf16, [64 r rows][128 d], two 64-column slabs of 8 KB
-  unsigned char* sQ = smem + kApplyOffQ;           // ring of 3, stage = tile % 3
+  unsigned char* sQ = smem + kApplyOffQ;           // ring of 3 slots (Q, then O_s / O), slot = tile % 3
   unsigned char* sF = smem + kApplyOffF;           // q~ tiles, one per warpgroup
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kApplyOffBar);
   uint64_t* bar_p_full = bars + 0;
   uint64_t* bar_c_full = bars + 1;                 // C staged (128 arrivals)
-  uint64_t* bar_q_full = bars + 2;                 // [3]
-  uint64_t* bar_q_empty = bars + 5;                // [3] projection MMAs done
-  uint64_t* bar_t_full = bars + 8;                 // [3]
-  uint64_t* bar_f_full = bars + 11;                // [3] q~ tile written (128 arrivals)
-  uint64_t* bar_y_full = bars + 14;                // [3] Y = q~ C done
-  uint64_t* bar_y_empty = bars + 17;               // [3] epilogue has read Y (128 arrivals)
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 20);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 21);
+  uint64_t* bar_q_full = bars + 2;                 // [3] Q tile landed
+  uint64_t* bar_q_empty = bars + 5;                // [3] projection MMAs done: slot may take O_s
+  uint64_t* bar_os_full = bars + 8;                // [3] O_s tile landed
+  uint64_t* bar_t_full = bars + 11;                // [3]
+  uint64_t* bar_f_full = bars + 14;                // [3] q~ tile written (128 arrivals)
+  uint64_t* bar_y_full = bars + 17;                // [3] Y = q~ C done
+  uint64_t* bar_slot_free = bars + 20;             // [3] output store has read the slot; Y has been read
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 24);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(bars + 25);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int bh = blockIdx.y;
@@ -364,8 +384,9 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     mbar_init(bar_p_full, 1);
     mbar_init(bar_c_full, 128);
     for (int g = 0; g < kFeatWGs; ++g) {
-      mbar_init(bar_q_full + g, 1); mbar_init(bar_q_empty + g, 1); mbar_init(bar_t_full + g, 1);
-      mbar_init(bar_f_full + g, 128); mbar_init(bar_y_full + g, 1); mbar_init(bar_y_empty + g, 128);
+      mbar_init(bar_q_full + g, 1); mbar_init(bar_q_empty + g, 1); mbar_init(bar_os_full + g, 1);
+      mbar_init(bar_t_full + g, 1); mbar_init(bar_f_full + g, 128); mbar_init(bar_y_full + g, 1);
+      mbar_init(bar_slot_free + g, 1);
     }
     *s_abort = 0;
     mbar_fence_init();
@@ -385,12 +406,36 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       mbar_expect_tx(bar_p_full, 16384);
       tma_load_4d(sP, &tmap_p, bar_p_full, 0, 0, h, 0);
       tma_load_4d(sP + 8192, &tmap_p, bar_p_full, 64, 0, h, 0);
-      for (int i = 0; i < ntiles; ++i) {
-        const int row = (tile0 + i) * kTileTok, st = i % kFeatWGs, n = i / kFeatWGs;
-        if (n > 0 && !mbar_wait(bar_q_empty + st, (n - 1) & 1, s_abort, p.status, 60)) break;
-        mbar_expect_tx(bar_q_full + st, 32768);
-        tma_load_4d(sQ + st * 32768, &tmap_q, bar_q_full + st, 0, row, h, b);
-        tma_load_4d(sQ + st * 32768 + 16384, &tmap_q, bar_q_full + st, 64, row, h, b);
+      int iq = 0, io = 0;                          // next Q tile / next O_s tile to request
+      bool ok = true;
+      IdleGuard guard;
+      guard.reset();
+      while (ok && io < ntiles) {
+        bool progressed = false;
+        if (iq < ntiles) {
+          const int g = iq % kFeatWGs, n = iq / kFeatWGs;
+          if (n == 0 || mbar_try_wait(bar_slot_free + g, (n - 1) & 1)) {
+            const int row = (tile0 + iq) * kTileTok;
+            mbar_expect_tx(bar_q_full + g, 32768);
+            tma_load_4d(sQ + g * 32768, &tmap_q, bar_q_full + g, 0, row, h, b);
+            tma_load_4d(sQ + g * 32768 + 16384, &tmap_q, bar_q_full + g, 64, row, h, b);
+            ++iq;
+            progressed = true;
+          }
+        }
+        if (io < iq) {
+          const int g = io % kFeatWGs;
+          if (mbar_try_wait(bar_q_empty + g, (io / kFeatWGs) & 1)) {
+            const int row = (tile0 + io) * kTileTok;
+            mbar_expect_tx(bar_os_full + g, 32768);
+            tma_load_4d(sQ + g * 32768, &tmap_os, bar_os_full + g, 0, row, h, b);
+            tma_load_4d(sQ + g * 32768 + 16384, &tmap_os, bar_os_full + g, 64, row, h, b);
+            ++io;
+            progressed = true;
+          }
+        }
+        if (progressed) guard.reset();
+        else ok = guard.idle(s_abort, p.status, 60);
       }
     }
   } else if (warp == kMmaWarp) {
@@ -405,10 +450,9 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       guard.reset();
       while (ok && s2 < ntiles) {
         bool progressed = false;
-        const int g1 = s1 % kFeatWGs, n1 = s1 / kFeatWGs;
-        // the projection of tile s1 overwrites the Y columns of tile s1 - 3: its epilogue must be done
-        if (s1 < ntiles && mbar_try_wait(bar_q_full + g1, n1 & 1) &&
-            (n1 == 0 || mbar_try_wait(bar_y_empty + g1, (n1 - 1) & 1))) {
+        const int g1 = s1 % kFeatWGs;
+        // a landed Q tile implies its slot (and with it the TMEM columns of the warpgroup) was released
+        if (s1 < ntiles && mbar_try_wait(bar_q_full + g1, (s1 / kFeatWGs) & 1)) {
           tc_fence_after();
           issue_projection(tmem + g1 * 128, smem_u32(sQ + g1 * 32768), smem_u32(sP));
           tc_commit(bar_t_full + g1);
@@ -439,6 +483,7 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     const int row = threadIdx.x & 127;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     unsigned char* tileF = sF + g * 16384;
+    unsigned char* slot = sQ + g * 32768;
     const uint32_t tmem_g = tmem + g * 128 + lane_off;
     if (g == 0) {
       if (ntiles > 0) {
@@ -461,29 +506,26 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     }
     bool ok = true;
     for (int i = g, u = 0; ok && i < ntiles; i += kFeatWGs, ++u) {
-      const int token = (tile0 + i) * kTileTok + row;
-      const bool valid = token < p.N;
-      const int tok_c = min(token, p.N - 1);
+      const int tile_row = (tile0 + i) * kTileTok;
+      const int token = tile_row + row;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full + g, u & 1, s_abort, p.status, 64));
       if (!ok) break;
       tc_fence_after();
       // the previous tile of this warpgroup has passed its Y wait, so the q~ tile is free
-      feature_row(tmem_g, tileF, row, p.rope, p.rope_table, p.rope_stride, tok_c);
+      feature_row(tmem_g, tileF, row, p.rope, p.rope_table, p.rope_stride, min(token, p.N - 1));
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar_f_full + g);
 
-      // sparse-branch row and gate, loaded while the second product runs
-      const int64_t off = b * p.stride_b + h * p.stride_h + (int64_t)tok_c * p.stride_n;
-      uint4 os[16];
+      const float gte = token < p.N ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
+      // sum of squares of the sparse-branch row (rows past N are zero tiles)
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_os_full + g, u & 1, s_abort, p.status, 66));
+      if (!ok) break;
       float so = 0.0f;
 #pragma unroll
-      for (int c = 0; c < 16; ++c)
-        os[c] = valid ? __ldg(reinterpret_cast<const uint4*>(p.o_sparse + off) + c) : make_uint4(0u, 0u, 0u, 0u);
-      const float gte = valid ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
-#pragma unroll
       for (int c = 0; c < 16; ++c) {
-        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&os[c]);
+        const uint4 q4 = *reinterpret_cast<const uint4*>(slot + (c >> 3) * 16384 + row * 128 + (((c & 7) ^ (row & 7)) << 4));
+        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&q4);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const float2 f = __bfloat1622float2(h2[j]);
@@ -493,7 +535,7 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       ok = __all_sync(0xffffffffu, mbar_wait(bar_y_full + g, u & 1, s_abort, p.status, 65));
       if (!ok) break;
       tc_fence_after();
-      // two passes over Y in TMEM: sum of squares, then the fused output
+      // two passes over Y in TMEM: sum of squares, then the fused output written over O_s in the slot
       float ss = 0.0f;
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
@@ -509,25 +551,35 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         uint32_t r[32];
         tmem_ld32(tmem_g + ch * 32, r);
         tc_wait_ld();
-        if (valid) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&os[ch * 4 + c]);
-            uint32_t w[4];
+        for (int c = 0; c < 4; ++c) {
+          uint4* cell = reinterpret_cast<uint4*>(slot + (ch >> 1) * 16384 + row * 128 +
+                                                 ((((ch & 1) * 4 + c) ^ (row & 7)) << 4));
+          const uint4 q4 = *cell;
+          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&q4);
+          uint32_t w[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float2 f = __bfloat1622float2(h2[j]);
-              const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(coef, __uint_as_float(r[8 * c + 2 * j]), f.x),
-                                                              fmaf(coef, __uint_as_float(r[8 * c + 2 * j + 1]), f.y));
-              w[j] = *reinterpret_cast<const uint32_t*>(&o2);
-            }
-            reinterpret_cast<uint4*>(p.out + off)[ch * 4 + c] = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int j = 0; j < 4; ++j) {
+            const float2 f = __bfloat1622float2(h2[j]);
+            const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(coef, __uint_as_float(r[8 * c + 2 * j]), f.x),
+                                                            fmaf(coef, __uint_as_float(r[8 * c + 2 * j + 1]), f.y));
+            w[j] = *reinterpret_cast<const uint32_t*>(&o2);
           }
+          *cell = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
+      fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(bar_y_empty + g);
+      named_bar_sync(1 + g, 128);
+      if (row == 0) {
+        tma_store_4d(&tmap_out, slot, 0, tile_row, h, b);
+        tma_store_4d(&tmap_out, slot + 16384, 64, tile_row, h, b);
+        bulk_commit();
+        bulk_wait_read0();
+        mbar_arrive(bar_slot_free + g);
+      }
     }
+    if (row == 0) bulk_wait0();
   }
   tc_fence_before();
   __syncthreads();
@@ -648,9 +700,11 @@ int launch_comp_state(const sparkattn_shape_t& s, const void* k, const void* v, 
 int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq, const int32_t* grid,
                       const int32_t* axis, const float* freq, const float* state, const float* gate,
                       const void* o_sparse, void* out, float eps, void* workspace, cudaStream_t stream) {
-  CUtensorMap mq, mp;
+  CUtensorMap mq, mp, mos, mout;
   int rc;
   if ((rc = comp_map(&mq, q, s.d, s.N, s.H, s.B, s.stride_n, s.stride_h, s.stride_b, kTileTok)) != SPARKATTN_OK) return rc;
+  if ((rc = comp_map(&mos, o_sparse, s.d, s.N, s.H, s.B, s.stride_n, s.stride_h, s.stride_b, kTileTok)) != SPARKATTN_OK) return rc;
+  if ((rc = comp_map(&mout, out, s.d, s.N, s.H, s.B, s.stride_n, s.stride_h, s.stride_b, kTileTok)) != SPARKATTN_OK) return rc;
   if ((rc = comp_map(&mp, pq, kCD, kRank, s.H, 1, kCD, (cuuint64_t)kRank * kCD, (cuuint64_t)s.H * kRank * kCD, kRank)) != SPARKATTN_OK)
     return rc;
   CompParams prm{};
@@ -667,7 +721,7 @@ int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq,
   if (cudaFuncSetAttribute(comp_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kApplySmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const dim3 grid_dim((unsigned)prm.nchunks, (unsigned)(s.B * s.H));
-  comp_apply_kernel<<<grid_dim, kCompThreads, kApplySmem, stream>>>(mq, mp, prm);
+  comp_apply_kernel<<<grid_dim, kCompThreads, kApplySmem, stream>>>(mq, mp, mos, mout, prm);
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
