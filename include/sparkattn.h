@@ -198,7 +198,7 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
  * eps               : RMSNorm epsilon (> 0)
  * workspace         : >= sparkattn_comp_workspace_bytes(shape, grid_host) bytes, 256-byte aligned
  *                     (sized for the state pass; the apply pass needs only its first
- *                     256 + 16 * rank * max(T, Hg, Wg) bytes); first word = device status
+ *                     512 + 4 * rank * (T + Hg + Wg) bytes); first word = device status
  * The host arrays are read during the call only.
  */
 size_t sparkattn_comp_workspace_bytes(const sparkattn_shape_t* shape, const int32_t* grid_host);

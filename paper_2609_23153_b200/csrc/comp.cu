@@ -53,38 +53,48 @@ struct CompParams {
   const __nv_bfloat16* o_sparse;      // apply
   __nv_bfloat16* out;                 // apply
   float eps;
-  const float2* rope_table;           // [rank/2][rope_stride] (cos, sin)
-  int rope_stride;
+  const float2* rope_table;           // [T + Hg + Wg][rank/2] (cos, sin)
   int32_t* status;
 };
 
-// cos/sin of every (rotary pair, coordinate) the grid can produce: table[m * stride + e] =
-// (cos, sin)(e * freq[m]) for e < extent(axis[m]).  A few thousand entries; the feature loops read
-// it through L1 instead of running a full-range sincosf per (token, pair).
-__global__ void rope_table_kernel(const RopeTable rope, float2* __restrict__ table, int stride) {
-  const int m = blockIdx.x;
+// cos/sin of every (coordinate, rotary pair) the grid can produce, position-major so that a token's
+// pairs of one axis sit in one 256-byte row: table[(base(axis) + e) * 32 + m] = (cos, sin)(e * freq[m])
+// with base(t) = 0, base(y) = T, base(x) = T + Hg (entries of pairs that rotate by another axis are
+// unused).  A few thousand entries; the feature loops read it through L1 instead of running a
+// full-range sincosf per (token, pair).
+__global__ void rope_table_kernel(const RopeTable rope, float2* __restrict__ table) {
+  const int m = threadIdx.x;                         // rank/2 threads
   const int ax = rope.axis[m];
-  const int extent = ax == 0 ? rope.T : (ax == 1 ? rope.Hg : rope.Wg);
-  for (int e = threadIdx.x; e < extent; e += blockDim.x) {
-    float sn, cs;
-    sincosf((float)e * rope.freq[m], &sn, &cs);
-    table[m * stride + e] = make_float2(cs, sn);
-  }
+  const int e = blockIdx.x;                          // T + Hg + Wg blocks
+  const int lo = ax == 0 ? 0 : (ax == 1 ? rope.T : rope.T + rope.Hg);
+  const int hi = ax == 0 ? rope.T : (ax == 1 ? rope.T + rope.Hg : rope.T + rope.Hg + rope.Wg);
+  float sn = 0.0f, cs = 1.0f;
+  if (e >= lo && e < hi) sincosf((float)(e - lo) * rope.freq[m], &sn, &cs);
+  table[e * (kRank / 2) + m] = make_float2(cs, sn);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+__device__ __forceinline__ float fast_rcp(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // One token row of T (64 fp32 columns at `taddr`) -> silu -> rank-truncated rotary rotation of the
 // adjacent pairs -> bf16 -> row `row` of a [128 rows x 128 B] tile with 128-byte swizzle.
 // Done in two halves of 32 columns to bound the live registers.
 __device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile, int row, const RopeTable& rope,
-                                            const float2* __restrict__ table, int stride, int token) {
+                                            const float2* __restrict__ table, int token) {
   const int x = token % rope.Wg;
   const int yy = token / rope.Wg;
   const int y = yy % rope.Hg;
   const int t = yy / rope.Hg;
+  const float2* row_t = table + t * (kRank / 2);
+  const float2* row_y = table + (rope.T + y) * (kRank / 2);
+  const float2* row_x = table + (rope.T + rope.Hg + x) * (kRank / 2);
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
     uint32_t r[32];
@@ -94,7 +104,7 @@ __device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile,
     for (int j = 0; j < 16; ++j) {
       const int m = half * 16 + j;
       const int ax = rope.axis[m];
-      cs[j] = __ldg(table + m * stride + (ax == 0 ? t : (ax == 1 ? y : x)));
+      cs[j] = __ldg((ax == 0 ? row_t : (ax == 1 ? row_y : row_x)) + m);
     }
     tc_wait_ld();
     uint32_t w[16];
@@ -103,7 +113,7 @@ __device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile,
       const float u0 = __uint_as_float(r[2 * j]), u1 = __uint_as_float(r[2 * j + 1]);
       const float2 e = unpack_f32x2(fadd2(pack_f32x2(fast_exp2(u0 * -1.4426950408889634f), fast_exp2(u1 * -1.4426950408889634f)),
                                           pack_f32x2(1.0f, 1.0f)));
-      const float z0 = __fdividef(u0, e.x), z1 = __fdividef(u1, e.y);
+      const float z0 = u0 * fast_rcp(e.x), z1 = u1 * fast_rcp(e.y);
       const float o0 = fmaf(z0, cs[j].x, -z1 * cs[j].y);
       const float o1 = fmaf(z0, cs[j].y, z1 * cs[j].x);
       const __nv_bfloat162 h2 = __floats2bfloat162_rn(o0, o1);
@@ -221,16 +231,30 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
       mbar_expect_tx(bar_p_full, 16384);
       tma_load_4d(sP, &tmap_p, bar_p_full, 0, 0, h, 0);
       tma_load_4d(sP + 8192, &tmap_p, bar_p_full, 64, 0, h, 0);
-      for (int i = 0; i < ntiles; ++i) {
-        const int row = (tile0 + i) * kTileTok, st = i & 1, n = i >> 1;
-        if (n > 0 && !mbar_wait(bar_k_empty + st, (n - 1) & 1, s_abort, p.status, 50)) break;
-        mbar_expect_tx(bar_k_full + st, 32768);
-        tma_load_4d(sK + st * 32768, &tmap_k, bar_k_full + st, 0, row, h, b);
-        tma_load_4d(sK + st * 32768 + 16384, &tmap_k, bar_k_full + st, 64, row, h, b);
-        if (n > 0 && !mbar_wait(bar_v_empty + st, (n - 1) & 1, s_abort, p.status, 51)) break;
-        mbar_expect_tx(bar_v_full + st, 32768);
-        tma_load_4d(sV + st * 32768, &tmap_v, bar_v_full + st, 0, row, h, b);
-        tma_load_4d(sV + st * 32768 + 16384, &tmap_v, bar_v_full + st, 64, row, h, b);
+      int ik = 0, iv = 0;                          // next K tile / next V tile to request
+      bool ok = true;
+      IdleGuard guard;
+      guard.reset();
+      while (ok && iv < ntiles) {
+        bool progressed = false;
+        if (ik < ntiles && (ik < 2 || mbar_try_wait(bar_k_empty + (ik & 1), ((ik >> 1) - 1) & 1))) {
+          const int row = (tile0 + ik) * kTileTok, st = ik & 1;
+          mbar_expect_tx(bar_k_full + st, 32768);
+          tma_load_4d(sK + st * 32768, &tmap_k, bar_k_full + st, 0, row, h, b);
+          tma_load_4d(sK + st * 32768 + 16384, &tmap_k, bar_k_full + st, 64, row, h, b);
+          ++ik;
+          progressed = true;
+        }
+        if (iv < 2 || mbar_try_wait(bar_v_empty + (iv & 1), ((iv >> 1) - 1) & 1)) {
+          const int row = (tile0 + iv) * kTileTok, st = iv & 1;
+          mbar_expect_tx(bar_v_full + st, 32768);
+          tma_load_4d(sV + st * 32768, &tmap_v, bar_v_full + st, 0, row, h, b);
+          tma_load_4d(sV + st * 32768 + 16384, &tmap_v, bar_v_full + st, 64, row, h, b);
+          ++iv;
+          progressed = true;
+        }
+        if (progressed) guard.reset();
+        else ok = guard.idle(s_abort, p.status, 50);
       }
     }
   } else if (warp == kMmaWarp) {
@@ -288,7 +312,7 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         if (!ok) break;
       }
       tc_fence_after();
-      feature_row(tmem + g * 64 + lane_off, tileF, row, p.rope, p.rope_table, p.rope_stride,
+      feature_row(tmem + g * 64 + lane_off, tileF, row, p.rope, p.rope_table,
                   min((tile0 + i) * kTileTok + row, p.N - 1));       // rows past N are zero anyway
       fence_proxy_async_smem();
       tc_fence_before();
@@ -512,7 +536,7 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       if (!ok) break;
       tc_fence_after();
       // the previous tile of this warpgroup has passed its Y wait, so the q~ tile is free
-      feature_row(tmem_g, tileF, row, p.rope, p.rope_table, p.rope_stride, min(token, p.N - 1));
+      feature_row(tmem_g, tileF, row, p.rope, p.rope_table, min(token, p.N - 1));
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar_f_full + g);
@@ -641,13 +665,8 @@ static int comp_chunks(const sparkattn_shape_t& s) {
   return best;
 }
 
-static int rope_stride(const int32_t* grid) {
-  int e = grid[0] > grid[1] ? grid[0] : grid[1];
-  if (grid[2] > e) e = grid[2];
-  return (e + 3) / 4 * 4;
-}
 static size_t rope_table_bytes(const int32_t* grid) {
-  return ((size_t)(kRank / 2) * rope_stride(grid) * sizeof(float2) + 255) / 256 * 256;
+  return ((size_t)(kRank / 2) * ((size_t)grid[0] + grid[1] + grid[2]) * sizeof(float2) + 255) / 256 * 256;
 }
 
 size_t comp_workspace_bytes(const sparkattn_shape_t& s, const int32_t* grid, bool with_state) {
@@ -662,10 +681,9 @@ static int prepare_workspace(CompParams& prm, const int32_t* grid, void* workspa
   prm.status = reinterpret_cast<int32_t*>(base);
   float2* table = reinterpret_cast<float2*>(base + kWorkspaceHeaderBytes);
   prm.rope_table = table;
-  prm.rope_stride = rope_stride(grid);
   prm.partial = reinterpret_cast<float*>(base + kWorkspaceHeaderBytes + rope_table_bytes(grid));
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
-  rope_table_kernel<<<kRank / 2, 128, 0, stream>>>(prm.rope, table, prm.rope_stride);
+  rope_table_kernel<<<(unsigned)(grid[0] + grid[1] + grid[2]), kRank / 2, 0, stream>>>(prm.rope, table);
   return SPARKATTN_OK;
 }
 
