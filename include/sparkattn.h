@@ -13,7 +13,9 @@
  *   sparkattn_select     pooled block scores + top-k -> kept-block index lists
  *   sparkattn_quant_fp8  per-(head, token-block) absmax scale + E4M3 encode
  *   sparkattn_fwd        block-sparse flash-attention forward (bf16 or FP8)
- * plus one host-buffer convenience call that chains them with the copies.
+ * plus one host-buffer convenience call that chains them with the copies, and
+ * the low-rank compensation branch with the gate fusion that completes the
+ * paper's attention module (sparkattn_comp_state, sparkattn_comp_apply).
  *
  * Conventions shared by all calls
  *   - Every data pointer is DEVICE memory owned by the caller unless a
