@@ -265,7 +265,7 @@ def run_ours(args, w):
     topk, nb = w.topk, w.nb
     shape = sa.make_shape(q, w.block)
     ws_sel = sa.alloc_workspace(shape, 0, topk, dev)
-    ws_fwd = sa.alloc_workspace(shape, 1, topk, dev)
+    ws_fwd = sa.alloc_workspace(shape, 1, nb if args.sweep else topk, dev)
     kept_idx = torch.empty((w.B, w.H, nb, topk), dtype=torch.int32, device=dev)
     kept_cnt = torch.empty((w.B, w.H, nb), dtype=torch.int32, device=dev)
     out = torch.empty_like(q)

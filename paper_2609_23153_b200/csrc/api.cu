@@ -52,10 +52,10 @@ const char* sparkattn_status_string(int status) {
   }
 }
 
-size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t /*topk_or_kmax*/) {
+size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t topk_or_kmax) {
   if (check_shape(shape) != SPARKATTN_OK) return 0;
   if (which == 0) return select_workspace_bytes(*shape);
-  if (which == 1) return fwd_workspace_bytes(*shape);
+  if (which == 1) return topk_or_kmax >= 1 ? fwd_workspace_bytes(*shape, topk_or_kmax) : 0;
   return 0;
 }
 
@@ -109,7 +109,7 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
   }
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out_bf16) || !aligned256(workspace))
     return SPARKATTN_E_MISALIGNED;
-  if (workspace_bytes < fwd_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < fwd_workspace_bytes(*shape, kmax)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   return launch_fwd(*shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, out_bf16, lse,
                     workspace, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -196,7 +196,7 @@ Arena plan_arena(const sparkattn_shape_t& s, int dtype, int topk) {
   sparkattn_shape_t c = s;
   c.stride_n = s.d; c.stride_h = (int64_t)s.N * s.d; c.stride_b = (int64_t)s.H * s.N * s.d;
   a.ws_sel = take(select_workspace_bytes(c));
-  a.ws_fwd = take(fwd_workspace_bytes(c));
+  a.ws_fwd = take(fwd_workspace_bytes(c, topk));
   a.cq = a.ck = a.cv = a.sq = a.sk = a.sv = 0;
   if (dtype == SPARKATTN_FP8_E4M3) {
     a.cq = take(elems); a.ck = take(elems); a.cv = take(elems);
@@ -253,7 +253,7 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
     sv = reinterpret_cast<const float*>(base + a.sv);
   }
   rc = sparkattn_fwd(&s, dtype, fq, fk, fv, sq, sk, sv, idx, cnt, topk, base + a.out, nullptr, base + a.ws_fwd,
-                     fwd_workspace_bytes(s), cuda_stream);
+                     fwd_workspace_bytes(s, topk), cuda_stream);
   if (rc != SPARKATTN_OK) return rc;
   if (cudaMemcpyAsync(out_host, base + a.out, bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
     return SPARKATTN_E_CUDA;

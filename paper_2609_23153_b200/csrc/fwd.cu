@@ -491,7 +491,11 @@ static int make_tile_map(CUtensorMap* map, const void* base, int elt_bytes, cons
   return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
-size_t fwd_workspace_bytes(const sparkattn_shape_t&) { return kWorkspaceHeaderBytes; }
+size_t fwd_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
+  // the pipelined kernel keeps range-checked, compacted copies of the kept lists behind the header
+  if (s.d == 128 && s.block == 128) return fwd_pipe_workspace_bytes(s, kmax);
+  return kWorkspaceHeaderBytes;
+}
 
 template <int D, int BLK, bool FP8>
 static int launch_fwd_t(const sparkattn_shape_t& s, const CUtensorMap& mq, const CUtensorMap& mk,
@@ -512,6 +516,10 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
+#ifndef SPARKATTN_FWD_NO_PIPE
+  if (!fp8 && s.d == 128 && s.block == 128)
+    return launch_fwd_pipe(s, q, k, v, kept_idx, kept_cnt, kmax, out, lse, workspace, stream);
+#endif
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;
   int rc;

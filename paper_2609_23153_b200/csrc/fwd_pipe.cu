@@ -1,0 +1,619 @@
+// sparkattn_fwd, bf16, d = 128, 128-token blocks: persistent pipelined block-sparse forward.
+//
+// Same arithmetic as fwd.cu (Sec. 2 softmax attention restricted to the kept tiles, Sec. 4.1 sparse
+// branch); different schedule.  Measured on the one-item-per-CTA kernel: a tile's chain
+// S-MMA -> softmax -> PV-MMA is ~3300 clocks long even with the SM to itself, so two independent
+// chains per SM leave the tensor pipe ~45 % busy.  Here one CTA per SM keeps THREE S tiles of the
+// same work item in flight (TMEM: S0 | S1 | S2 | O, 128 columns each):
+//   warps 0-3 / 4-7  two softmax warpgroups; the tiles of the CTA's item stream alternate between
+//                    them (global tile counter parity), thread r owns query row r.  The running
+//                    reference maximum of a row travels from the warpgroup of tile t-1 to the
+//                    warpgroup of tile t through shared memory (token barrier); it only moves
+//                    when a tile maximum exceeds it by more than 2^8 (lazy rescale), and the
+//                    warpgroup that moves it rescales O before it passes the token on.  Each
+//                    warpgroup keeps its own partial row sum relative to the last reference it
+//                    saw; the warpgroup of the item's last tile combines them, normalises O into
+//                    the item's (now dead) Q slot and stores it with one TMA copy.
+//   warp 8           TMA producer: Q (2 slots), K ring (2), V ring (3), across item boundaries.
+//   warp 9           MMA issuer, polling: O += P V of the oldest tile whose P is written, else
+//                    S = Q K^T of the next tile whose K has landed and whose S buffer is free.
+//   warps 10-11      idle (complete the third warpgroup for the register hand-over).
+// Work items (batch, head, query block) go to CTA c as c, c + grid, ... in head-major order, so
+// the CTAs running together read K/V of one head from L2.  Kept lists are range-checked and
+// compacted by a small pre-pass into the workspace; every role reads the clean lists from there.
+// Every wait is bounded; nothing here waits on another CTA.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "launch.h"
+
+namespace sparkattn {
+
+constexpr int kPipeThreads = 384;
+constexpr int kPipeSoftmaxRegs = 216, kPipeCtrlRegs = 64;   // 2*128*216 + 128*64 <= 384*168
+constexpr int kPD = 128, kPBLK = 128;
+constexpr float kPipeLazyLog2 = 8.0f;
+constexpr int kTile = 32768;                               // bytes of one 128 x 128 bf16 tile (two 64-column slabs)
+constexpr int kOffQ = 0, kOffK = 2 * kTile, kOffV = 4 * kTile, kOffMisc = 7 * kTile;
+constexpr int kPipeSmem = kOffMisc + 256 /*barriers*/ + 2 * 128 * 4 /*reference maxima*/ + 128 * 8 /*row sums*/ + 64;
+
+struct PipeParams {
+  const int32_t* clean_cnt;    // [items] valid kept blocks per item
+  const int32_t* clean_list;   // [items][kmax] their indices, compacted in list order
+  __nv_bfloat16* out;
+  float* lse;
+  int32_t* status;
+  int H, N, nb, kmax, items;
+  int64_t stride_b, stride_h, stride_n;
+  float scale_log2;
+};
+
+// one warp per item: drop (and report) kept indices outside [0, nb), clamp the count
+__global__ void compact_lists_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ kept_cnt,
+                                     int32_t* __restrict__ clean_cnt, int32_t* __restrict__ clean_list, int items,
+                                     int nb, int kmax, int32_t* status) {
+  const int item = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (item >= items) return;
+  const int cnt = kept_cnt ? min(max(__ldg(kept_cnt + item), 0), kmax) : kmax;
+  const int32_t* src = kept_idx + (int64_t)item * kmax;
+  int32_t* dst = clean_list + (int64_t)item * kmax;
+  int out = 0;
+  for (int base = 0; base < cnt; base += 32) {
+    const int t = base + lane;
+    const int kb = (t < cnt) ? __ldg(src + t) : 0;
+    const bool valid = (t < cnt) && kb >= 0 && kb < nb;
+    if (t < cnt && !valid) report_status(status, SPARKATTN_E_BAD_INDEX, kb);
+    const uint32_t ballot = __ballot_sync(0xffffffffu, valid);
+    if (valid) dst[out + __popc(ballot & ((1u << lane) - 1u))] = kb;
+    out += __popc(ballot);
+  }
+  if (lane == 0) clean_cnt[item] = out;
+}
+
+__device__ __forceinline__ void pipe_tma_store_4d(const void* tmap, const void* smem_src, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+      ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+struct PipeIdle {
+  uint64_t t0;
+  uint32_t polls;
+  __device__ __forceinline__ void reset() { polls = 0; }
+  // Nothing was ready: yield the issue slots to the softmax warps of this scheduler for a moment.
+  __device__ __forceinline__ bool idle(volatile int* abort_flag, int32_t* status, int wait_id) {
+    if (polls == 0) t0 = global_timer_ns();
+    __nanosleep(32);
+    if ((++polls & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        report_status(status, SPARKATTN_E_DEVICE_TIMEOUT, wait_id);
+        return false;
+      }
+    }
+    return true;
+  }
+};
+
+__global__ void __launch_bounds__(kPipeThreads, 1)
+fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                const PipeParams p) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* sQ = smem + kOffQ;
+  unsigned char* sK = smem + kOffK;
+  unsigned char* sV = smem + kOffV;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffMisc);
+  uint64_t* bar_q_full = bars + 0;     // [2]
+  uint64_t* bar_q_free = bars + 2;     // [2] the item's output store has read the slot (or the item was empty)
+  uint64_t* bar_k_full = bars + 4;     // [2]
+  uint64_t* bar_k_free = bars + 6;     // [2] S MMAs that read the slot are complete
+  uint64_t* bar_v_full = bars + 8;     // [3]
+  uint64_t* bar_v_free = bars + 11;    // [3] PV MMAs that read the slot are complete
+  uint64_t* bar_s_full = bars + 14;    // [3]
+  uint64_t* bar_p_full = bars + 17;    // [3] 128 arrivals
+  uint64_t* bar_pv_done = bars + 20;   // [3] S buffer free again
+  uint64_t* bar_o_free = bars + 23;    // 128 arrivals: the closing warpgroup has read O
+  uint64_t* bar_tok = bars + 24;       // [2] 128 arrivals: warpgroup g has published its reference maxima
+  uint64_t* bar_lsum = bars + 26;      // 128 arrivals: the non-closing warpgroup has published its row sums
+  uint64_t* bar_lsum_ack = bars + 27;  // 128 arrivals: they have been read
+  float* s_mref = reinterpret_cast<float*>(bars + 32);           // [2][128]
+  float2* s_lsum = reinterpret_cast<float2*>(s_mref + 2 * 128);  // [128] (partial row sum, reference it is relative to)
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_lsum + 128);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_q_full + i, 1); mbar_init(bar_q_free + i, 1);
+      mbar_init(bar_k_full + i, 1); mbar_init(bar_k_free + i, 1);
+      mbar_init(bar_tok + i, 128);
+    }
+    for (int i = 0; i < 3; ++i) {
+      mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1);
+      mbar_init(bar_s_full + i, 1); mbar_init(bar_p_full + i, 128); mbar_init(bar_pv_done + i, 1);
+    }
+    mbar_init(bar_o_free, 128); mbar_init(bar_lsum, 128); mbar_init(bar_lsum_ack, 128);
+    int dead = (*reinterpret_cast<volatile int32_t*>(p.status) == SPARKATTN_E_DEVICE_TIMEOUT) ? 1 : 0;
+    if ((smem_u32(smem) & 1023u) != 0u) {       // the swizzled tiles need a 1024-byte aligned base
+      report_status(p.status, SPARKATTN_E_MISALIGNED, (int)(smem_u32(smem) & 1023u));
+      dead = 1;
+    }
+    *s_abort = dead;
+    mbar_fence_init();
+  }
+  if (warp == 8) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); tma_prefetch_desc(&tmap_o);
+    }
+    __syncwarp();
+    tmem_alloc(s_tmem, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+  const uint32_t tmem_O = tmem + 3 * kPBLK;
+  const bool dead = *s_abort != 0;
+  const int first_item = blockIdx.x, item_step = gridDim.x;
+
+  if (warp >= 8) reg_dec<kPipeCtrlRegs>();
+  if (dead) {
+    // fall through to the teardown
+  } else if (warp == 8) {
+    // ------------------------------------------------------------ TMA producer (warp converged, lane 0 issues)
+    // K cursor (also loads Q at the start of an item) and V cursor walk the same tile stream.
+    int ki = 0, k_item = first_item, k_n = 0, k_cnt = 0, k_t = 0, k_chunk = 0;   // item ordinal, item, tile, count, global tile, list registers
+    int vi = 0, v_item = first_item, v_n = 0, v_cnt = 0, v_t = 0, v_chunk = 0;
+    bool k_open = false, v_open = false;   // item header processed?
+    bool ok = true;
+    PipeIdle guard;
+    guard.reset();
+    // lane 0 polls, the warp follows: keeps the warp converged for the shuffles below
+    auto uwait = [&](uint64_t* bar, uint32_t parity) {
+      const int r = (lane == 0 && mbar_try_wait(bar, parity)) ? 1 : 0;
+      return __shfl_sync(0xffffffffu, r, 0) != 0;
+    };
+    while (ok && (k_item < p.items || v_item < p.items)) {
+      bool progressed = false;
+      if (k_item < p.items) {
+        if (!k_open) {
+          const int slot = ki & 1;
+          if (ki < 2 || uwait(bar_q_free + slot, ((ki >> 1) - 1) & 1)) {
+            k_cnt = __ldg(p.clean_cnt + k_item);
+            if (lane == 0) {
+              if (k_cnt > 0) {
+                const int qb = k_item % p.nb, bh = k_item / p.nb;
+                mbar_expect_tx(bar_q_full + slot, kTile);
+                tma_load_4d(sQ + slot * kTile, &tmap_q, bar_q_full + slot, 0, qb * kPBLK, bh % p.H, bh / p.H);
+                tma_load_4d(sQ + slot * kTile + kTile / 2, &tmap_q, bar_q_full + slot, 64, qb * kPBLK, bh % p.H, bh / p.H);
+              } else {
+                mbar_arrive(bar_q_full + slot);      // empty item: nothing to load, consumers still step through it
+              }
+            }
+            k_open = true;
+            k_n = 0;
+            progressed = true;
+          }
+        }
+        if (k_open) {
+          if (k_n >= k_cnt) {
+            k_item += item_step; ++ki; k_open = false;
+            progressed = true;
+          } else {
+            const int slot = k_t & 1;
+            if (k_t < 2 || uwait(bar_k_free + slot, ((k_t >> 1) - 1) & 1)) {
+              if ((k_n & 31) == 0) k_chunk = (k_n + lane < k_cnt) ? __ldg(p.clean_list + (int64_t)k_item * p.kmax + k_n + lane) : 0;
+              const int kb = __shfl_sync(0xffffffffu, k_chunk, k_n & 31);
+              if (lane == 0) {
+                const int bh = k_item / p.nb;
+                mbar_expect_tx(bar_k_full + slot, kTile);
+                tma_load_4d(sK + slot * kTile, &tmap_k, bar_k_full + slot, 0, kb * kPBLK, bh % p.H, bh / p.H);
+                tma_load_4d(sK + slot * kTile + kTile / 2, &tmap_k, bar_k_full + slot, 64, kb * kPBLK, bh % p.H, bh / p.H);
+              }
+              ++k_n; ++k_t;
+              progressed = true;
+            }
+          }
+        }
+      }
+      if (v_item < p.items) {
+        if (!v_open) {
+          // the V cursor never passes the K cursor's item header (it needs no header work of its own)
+          if (vi < ki || (vi == ki && k_open)) {
+            v_cnt = __ldg(p.clean_cnt + v_item);
+            v_open = true;
+            v_n = 0;
+            progressed = true;
+          }
+        }
+        if (v_open) {
+          if (v_n >= v_cnt) {
+            v_item += item_step; ++vi; v_open = false;
+            progressed = true;
+          } else if (v_t < k_t) {
+            const int slot = v_t % 3;
+            if (v_t < 3 || uwait(bar_v_free + slot, ((v_t / 3) - 1) & 1)) {
+              if ((v_n & 31) == 0) v_chunk = (v_n + lane < v_cnt) ? __ldg(p.clean_list + (int64_t)v_item * p.kmax + v_n + lane) : 0;
+              const int kb = __shfl_sync(0xffffffffu, v_chunk, v_n & 31);
+              if (lane == 0) {
+                const int bh = v_item / p.nb;
+                mbar_expect_tx(bar_v_full + slot, kTile);
+                tma_load_4d(sV + slot * kTile, &tmap_v, bar_v_full + slot, 0, kb * kPBLK, bh % p.H, bh / p.H);
+                tma_load_4d(sV + slot * kTile + kTile / 2, &tmap_v, bar_v_full + slot, 64, kb * kPBLK, bh % p.H, bh / p.H);
+              }
+              ++v_n; ++v_t;
+              progressed = true;
+            }
+          }
+        }
+      }
+      if (progressed) guard.reset();
+      else ok = __shfl_sync(0xffffffffu, (lane == 0 && !guard.idle(s_abort, p.status, 1)) ? 0 : 1, 0) != 0;
+    }
+  } else if (warp == 9) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc(1u, 128, kPBLK, false);
+      constexpr uint32_t idesc_pv = make_idesc(1u, 128, kPD, true);
+      // S cursor and PV cursor over the same tile stream
+      int si = 0, s_item = first_item, s_n = 0, s_cnt = -1, s_t = 0;
+      int pi = 0, p_item = first_item, p_n = 0, p_cnt = -1, p_t = 0, p_nonempty = 0;
+      bool ok = true;
+      PipeIdle guard;
+      guard.reset();
+      while (ok && p_item < p.items) {
+        bool progressed = false;
+        // step both cursors over finished and empty items (no shared-memory traffic)
+        if (p_cnt < 0) p_cnt = __ldg(p.clean_cnt + p_item);
+        if (p_n >= p_cnt) {
+          if (p_cnt > 0) ++p_nonempty;
+          p_item += item_step; ++pi; p_n = 0; p_cnt = -1;
+          guard.reset();
+          continue;
+        }
+        if (s_item < p.items) {
+          if (s_cnt < 0) s_cnt = __ldg(p.clean_cnt + s_item);
+          if (s_n >= s_cnt) {
+            s_item += item_step; ++si; s_n = 0; s_cnt = -1;
+            guard.reset();
+            continue;
+          }
+        }
+        // Every barrier either product may need is polled up front, back to back: a poll is a
+        // shared-memory round trip (~100 clocks), and chained polls would add up to the length of
+        // an MMA group per step.
+        const int pbuf = p_t % 3, sbuf = s_t % 3, kslot = s_t & 1, qslot = si & 1;
+        const bool pf = mbar_test(bar_p_full + pbuf, (p_t / 3) & 1);
+        const bool vf = mbar_test(bar_v_full + pbuf, (p_t / 3) & 1);
+        const bool pd = mbar_test(bar_pv_done + sbuf, ((s_t / 3) - 1) & 1);
+        const bool kf = mbar_test(bar_k_full + kslot, (s_t >> 1) & 1);
+        // first tile of an item only: O of the previous item read by its closer; Q of this item landed
+        const bool of = (p_n > 0 || p_nonempty == 0) ? true : mbar_test(bar_o_free, (p_nonempty - 1) & 1);
+        const bool qf = s_n > 0 ? true : mbar_test(bar_q_full + qslot, (si >> 1) & 1);
+        // ---- O += P V of the oldest pending tile
+        if (p_t < s_t && pf && vf && of) {
+          tc_fence_after();
+          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + pbuf * kTile), kTile / 2);
+          const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts<false>(tmem_O, tmem + pbuf * kPBLK + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), v_hi), idesc_pv,
+                          (p_n == 0 && kk == 0) ? 0u : 1u);
+          tc_commit(bar_pv_done + pbuf);
+          tc_commit(bar_v_free + pbuf);
+          ++p_n; ++p_t;
+          progressed = true;
+        }
+        // ---- S = Q K^T of the next tile (its S buffer is free once PV of tile s_t - 3 is complete)
+        if (s_item < p.items && (s_t < 3 || pd) && kf && qf) {
+          tc_fence_after();
+          const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ + qslot * kTile), 16);
+          const uint64_t dK = make_smem_desc_sw128(smem_u32(sK + kslot * kTile), 16);
+          const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32), k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              mma_ss<false>(tmem + sbuf * kPBLK, make_desc(q_lo + ((sl * (kTile / 2) + kk * 32) >> 4), q_hi),
+                            make_desc(k_lo + ((sl * (kTile / 2) + kk * 32) >> 4), k_hi), idesc_qk, (sl | kk) != 0 ? 1u : 0u);
+          tc_commit(bar_s_full + sbuf);
+          tc_commit(bar_k_free + kslot);
+          ++s_n; ++s_t;
+          progressed = true;
+        }
+        if (progressed) guard.reset();
+        else ok = guard.idle(s_abort, p.status, 2);
+      }
+    }
+  } else if (warp < 8) {
+    // ----------------------------------------------------------------- softmax
+    reg_inc<kPipeSoftmaxRegs>();
+    const int g = warp >> 2;                          // warpgroup: takes the tiles with (global tile counter & 1) == g
+    const int row = threadIdx.x & 127;                // query row inside the block = TMEM lane
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const float c = p.scale_log2;
+    float m_used = 0.0f, l = 0.0f;                    // reference maximum this warpgroup last used; its partial row sum
+    int t = 0;                                        // global tile counter at the start of the item
+    int nonempty = 0;                                 // non-empty items finished so far
+    bool ok = true;
+    int io = 0;
+    for (int item = first_item; ok && item < p.items; item += item_step, ++io) {
+      const int qslot = io & 1;
+      const int cnt = __ldg(p.clean_cnt + item);
+      const int qb = item % p.nb, bh = item / p.nb;
+      const int h = bh % p.H, b = bh / p.H;
+      const int q_row = qb * kPBLK + row;
+      const bool row_valid = q_row < p.N;
+      if (cnt == 0) {
+        if (g == 0) {
+          // empty kept list: zero output, lse = -inf; release the item's Q slot
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_q_full + qslot, (io >> 1) & 1, s_abort, p.status, 3));
+          if (!ok) break;
+          if (row_valid) {
+            __nv_bfloat16* orow = p.out + b * p.stride_b + h * p.stride_h + (int64_t)q_row * p.stride_n;
+#pragma unroll
+            for (int ch = 0; ch < kPD / 8; ++ch) reinterpret_cast<uint4*>(orow)[ch] = make_uint4(0u, 0u, 0u, 0u);
+            if (p.lse) p.lse[(int64_t)bh * p.N + q_row] = -INFINITY;
+          }
+          if (row == 0) mbar_arrive(bar_q_free + qslot);
+        }
+        continue;
+      }
+      l = 0.0f;
+      for (int n = 0; ok && n < cnt; ++n) {
+        const int tt = t + n;
+        if ((tt & 1) != g) continue;
+        const int buf = tt % 3;
+        const int kb = __ldg(p.clean_list + (int64_t)item * p.kmax + n);
+        const int ncols = min(kPBLK, p.N - kb * kPBLK);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt / 3) & 1, s_abort, p.status, 4));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tS = tmem + buf * kPBLK + lane_off;
+        uint32_t sr[kPBLK];
+#pragma unroll
+        for (int ch = 0; ch < kPBLK / 32; ++ch) tmem_ld32(tS + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
+        tc_wait_ld();
+        if (ncols < kPBLK) {          // ragged last key block: keys >= N get weight 0
+#pragma unroll
+          for (int i = 0; i < kPBLK; ++i)
+            if (i >= ncols) sr[i] = 0xff800000u;
+        }
+        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
+        float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
+#pragma unroll
+        for (int i = 4; i < kPBLK; i += 8) {
+          mx0 = fmax3(mx0, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+          mx1 = fmax3(mx1, __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+          if (i + 4 < kPBLK) {
+            mx2 = fmax3(mx2, __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+            mx3 = fmax3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
+          }
+        }
+        const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
+
+        // reference maximum: token from the warpgroup of tile tt-1 (also orders the reuse of s_mref[g])
+        if (tt > 0) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_tok + (g ^ 1), ((tt - 1) >> 1) & 1, s_abort, p.status, 5));
+          if (!ok) break;
+        }
+        float m_new;
+        bool need = false;
+        float alpha = 1.0f;
+        if (n == 0) {
+          m_new = m_tile;
+        } else {
+          const float m_prev = s_mref[(g ^ 1) * 128 + row];
+          if (m_tile > m_prev + kPipeLazyLog2) {
+            m_new = m_tile;
+            alpha = fast_exp2(m_prev - m_tile);
+            need = true;
+          } else {
+            m_new = m_prev;
+          }
+        }
+        if (l != 0.0f && m_new != m_used) l *= fast_exp2(m_used - m_new);   // own partial sum to the new reference
+        m_used = m_new;
+        if (__any_sync(0xffffffffu, need)) {
+          // every PV issued so far must be complete before O is rescaled: the last one is tile tt-1's
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + (tt - 1) % 3, ((tt - 1) / 3) & 1, s_abort, p.status, 6));
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t a2 = pack_f32x2(alpha, alpha);
+#pragma unroll 1
+          for (int ch = 0; ch < kPD / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_O + lane_off + ch * 32, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float2 o2 = unpack_f32x2(fmul2(pack_f32x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), a2));
+              r[i] = __float_as_uint(o2.x);
+              r[i + 1] = __float_as_uint(o2.y);
+            }
+            tmem_st32(tmem_O + lane_off + ch * 32, r);
+          }
+          tc_wait_st();
+          tc_fence_before();
+        }
+        s_mref[g * 128 + row] = m_used;
+        mbar_arrive(bar_tok + g);
+
+        // P = exp2(S*c - m) as bf16 over the first 64 columns of this S buffer
+        const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used, -m_used);
+        uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
+#pragma unroll
+        for (int ch = 0; ch < kPBLK / 32; ++ch) {
+          uint32_t w[16];
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float2 x = unpack_f32x2(
+                ffma2(pack_f32x2(__uint_as_float(sr[ch * 32 + i]), __uint_as_float(sr[ch * 32 + i + 1])), c2, nm2));
+            const float e0 = fast_exp2(x.x), e1 = fast_exp2(x.y);
+            if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e0, e1));
+            else lsum0 = fadd2(lsum0, pack_f32x2(e0, e1));
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e0, e1);
+            w[i >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          tmem_st16(tS + ch * 16, w);
+        }
+        const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
+        l += ls.x + ls.y;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar_p_full + buf);
+      }
+      if (!ok) break;
+
+      // ------------------------------------------------------------ end of the item
+      const int t_last = t + cnt - 1;
+      if ((t_last & 1) != g) {
+        // not the closer: hand the partial row sum over (after the previous hand-over was read)
+        if (nonempty > 0) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum_ack, (nonempty - 1) & 1, s_abort, p.status, 7));
+          if (!ok) break;
+        }
+        s_lsum[row] = make_float2(l, m_used);
+        mbar_arrive(bar_lsum);
+      } else {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum, nonempty & 1, s_abort, p.status, 8));
+        if (!ok) break;
+        const float2 other = s_lsum[row];
+        mbar_arrive(bar_lsum_ack);
+        if (other.x != 0.0f) l += other.x * fast_exp2(other.y - m_used);
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + t_last % 3, (t_last / 3) & 1, s_abort, p.status, 9));
+        if (!ok) break;
+        tc_fence_after();
+        // normalised O row as bf16 into the item's Q slot (all S MMAs of the item are complete), 128-byte swizzle
+        const float inv = 1.0f / l;
+        unsigned char* slot = sQ + qslot * kTile;
+#pragma unroll 1
+        for (int ch = 0; ch < kPD / 32; ++ch) {
+          uint32_t r[32];
+          tmem_ld32(tmem_O + lane_off + ch * 32, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            uint32_t ww[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[8 * cc + 2 * j]) * inv,
+                                                              __uint_as_float(r[8 * cc + 2 * j + 1]) * inv);
+              ww[j] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(slot + (ch >> 1) * (kTile / 2) + row * 128 + ((((ch & 1) * 4 + cc) ^ (row & 7)) << 4)) =
+                make_uint4(ww[0], ww[1], ww[2], ww[3]);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_o_free);
+        if (row_valid && p.lse) p.lse[(int64_t)bh * p.N + q_row] = (m_used + log2f(l)) * 0.6931471805599453f;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");
+        if (row == 0) {
+          pipe_tma_store_4d(&tmap_o, slot, 0, qb * kPBLK, h, b);
+          pipe_tma_store_4d(&tmap_o, slot + kTile / 2, 64, qb * kPBLK, h, b);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          mbar_arrive(bar_q_free + qslot);
+        }
+      }
+      t += cnt;
+      ++nonempty;
+    }
+    if (row == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    if (*s_abort) __nanosleep(200000);  // let copies / MMAs in flight land before the CTA's resources go
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*PipeEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static PipeEncodeFn pipe_encode_fn() {
+  static PipeEncodeFn fn = nullptr;
+  if (fn) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<PipeEncodeFn>(ptr);
+  return fn;
+}
+
+static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t& s) {
+  PipeEncodeFn enc = pipe_encode_fn();
+  if (!enc) return SPARKATTN_E_NO_DEVICE;
+  const cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.H, (cuuint64_t)s.B};
+  const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * 2, (cuuint64_t)s.stride_h * 2, (cuuint64_t)s.stride_b * 2};
+  const cuuint32_t box[4] = {64u, (cuuint32_t)kPBLK, 1u, 1u};
+  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
+  const size_t items = (size_t)s.B * s.H * ((s.N + s.block - 1) / s.block);
+  return kWorkspaceHeaderBytes + (items * 4 + 255) / 256 * 256 + items * (size_t)kmax * 4;
+}
+
+int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, const void* v, const int32_t* kept_idx,
+                    const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream) {
+  CUtensorMap mq, mk, mv, mo;
+  int rc;
+  if ((rc = pipe_map(&mq, q, s)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mk, k, s)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mv, v, s)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mo, out, s)) != SPARKATTN_OK) return rc;
+  const int nb = (s.N + s.block - 1) / s.block;
+  const long long items = (long long)s.B * s.H * nb;
+  if (items > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  char* base = static_cast<char*>(workspace);
+  int32_t* clean_cnt = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes);
+  int32_t* clean_list = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256);
+  PipeParams prm;
+  prm.clean_cnt = clean_cnt;
+  prm.clean_list = clean_list;
+  prm.out = static_cast<__nv_bfloat16*>(out);
+  prm.lse = lse;
+  prm.status = static_cast<int32_t*>(workspace);
+  prm.H = s.H; prm.N = s.N; prm.nb = nb; prm.kmax = kmax; prm.items = (int)items;
+  prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
+  const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
+  prm.scale_log2 = sc * 1.4426950408889634f;
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
+      return SPARKATTN_E_CUDA;
+  }
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  compact_lists_kernel<<<(unsigned)((items + 7) / 8), 256, 0, stream>>>(kept_idx, kept_cnt, clean_cnt, clean_list, (int)items,
+                                                                      nb, kmax, prm.status);
+  if (cudaFuncSetAttribute(fwd_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
+  fwd_pipe_kernel<<<grid, kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, prm);
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+}  // namespace sparkattn

@@ -110,7 +110,7 @@ def test_bad_index_is_reported_and_skipped():
     w = _small(37, 1, 128, (2, 8, 16), 128, 0.0)   # N=256, nb=2
     q, k, v = workloads.structured_qkv(w)
     idx = torch.tensor([[[[0, 7], [-1, 1]]]], dtype=torch.int32)
-    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    ws = torch.zeros(sa.workspace_bytes(sa.make_shape(q, w.block), 1, 2), dtype=torch.uint8, device=DEV)
     out = sa.fwd(q.to(DEV), k.to(DEV), v.to(DEV), idx.to(DEV), None, w.block, workspace=ws)
     assert sa.read_status(ws) == sa.E_BAD_INDEX
     good = torch.tensor([[[0, 0], [1, 0]]], dtype=torch.int32)
