@@ -5,7 +5,7 @@
 // S-MMA -> softmax -> PV-MMA is ~3300 clocks long even with the SM to itself, so two independent
 // chains per SM leave the tensor pipe ~45 % busy.  Here one CTA per SM keeps THREE S tiles of the
 // same work item in flight (TMEM: S0 | S1 | S2 | O, 128 columns each):
-//   warps 0-3 / 4-7  two softmax warpgroups; the tiles of the CTA's item stream alternate between
+//   warps 4-7 / 8-11 two softmax warpgroups; the tiles of the CTA's item stream alternate between
 //                    them (global tile counter parity), thread r owns query row r.  The running
 //                    reference maximum of a row travels from the warpgroup of tile t-1 to the
 //                    warpgroup of tile t through shared memory (token barrier); it only moves
@@ -14,10 +14,14 @@
 //                    warpgroup keeps its own partial row sum relative to the last reference it
 //                    saw; the warpgroup of the item's last tile combines them, normalises O into
 //                    the item's (now dead) Q slot and stores it with one TMA copy.
-//   warp 8           TMA producer: Q (2 slots), K ring (2), V ring (3), across item boundaries.
-//   warp 9           MMA issuer, polling: O += P V of the oldest tile whose P is written, else
-//                    S = Q K^T of the next tile whose K has landed and whose S buffer is free.
-//   warps 10-11      idle (complete the third warpgroup for the register hand-over).
+//   warp 0           TMA producer: Q (2 slots), K ring (2), V ring (3), across item boundaries.
+//   warp 1           S issuer, polling: S = Q K^T of the next tile whose K has landed and whose S
+//                    buffer is free (PV of the tile three back complete).
+//   warp 2           PV issuer, polling: O += P V of the oldest tile whose P is written.
+//                    Two issuing warps on two schedulers: an issuing thread shares its scheduler
+//                    with two softmax warps that are almost always ready and only gets an issue
+//                    slot when they stall, so its instruction count per tile is what matters.
+//   warp 3           idle (completes the first warpgroup for the register hand-over).
 // Work items (batch, head, query block) go to CTA c as c, c + grid, ... in head-major order, so
 // the CTAs running together read K/V of one head from L2.  Kept lists are range-checked and
 // compacted by a small pre-pass into the workspace; every role reads the clean lists from there.
@@ -146,7 +150,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     *s_abort = dead;
     mbar_fence_init();
   }
-  if (warp == 8) {
+  if (warp == 0) {
     if (lane == 0) {
       tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); tma_prefetch_desc(&tmap_o);
     }
@@ -162,10 +166,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   const bool dead = *s_abort != 0;
   const int first_item = blockIdx.x, item_step = gridDim.x;
 
-  if (warp >= 8) reg_dec<kPipeCtrlRegs>();
+  if (warp < 4) reg_dec<kPipeCtrlRegs>();
   if (dead) {
     // fall through to the teardown
-  } else if (warp == 8) {
+  } else if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (warp converged, lane 0 issues)
     // K cursor (also loads Q at the start of an item) and V cursor walk the same tile stream.
     int ki = 0, k_item = first_item, k_n = 0, k_cnt = 0, k_t = 0, k_chunk = 0;   // item ordinal, item, tile, count, global tile, list registers
@@ -256,62 +260,26 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       if (progressed) guard.reset();
       else ok = __shfl_sync(0xffffffffu, (lane == 0 && !guard.idle(s_abort, p.status, 1)) ? 0 : 1, 0) != 0;
     }
-  } else if (warp == 9) {
-    // -------------------------------------------------------------- MMA issuer
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- S issuer: S = Q K^T of the next tile
     if (lane == 0) {
       constexpr uint32_t idesc_qk = make_idesc(1u, 128, kPBLK, false);
-      constexpr uint32_t idesc_pv = make_idesc(1u, 128, kPD, true);
-      // S cursor and PV cursor over the same tile stream
       int si = 0, s_item = first_item, s_n = 0, s_cnt = -1, s_t = 0;
-      int pi = 0, p_item = first_item, p_n = 0, p_cnt = -1, p_t = 0, p_nonempty = 0;
       bool ok = true;
       PipeIdle guard;
       guard.reset();
-      while (ok && p_item < p.items) {
-        bool progressed = false;
-        // step both cursors over finished and empty items (no shared-memory traffic)
-        if (p_cnt < 0) p_cnt = __ldg(p.clean_cnt + p_item);
-        if (p_n >= p_cnt) {
-          if (p_cnt > 0) ++p_nonempty;
-          p_item += item_step; ++pi; p_n = 0; p_cnt = -1;
-          guard.reset();
+      while (ok && s_item < p.items) {
+        if (s_cnt < 0) s_cnt = __ldg(p.clean_cnt + s_item);
+        if (s_n >= s_cnt) {
+          s_item += item_step; ++si; s_n = 0; s_cnt = -1;
           continue;
         }
-        if (s_item < p.items) {
-          if (s_cnt < 0) s_cnt = __ldg(p.clean_cnt + s_item);
-          if (s_n >= s_cnt) {
-            s_item += item_step; ++si; s_n = 0; s_cnt = -1;
-            guard.reset();
-            continue;
-          }
-        }
-        // Every barrier either product may need is polled up front, back to back: a poll is a
-        // shared-memory round trip (~100 clocks), and chained polls would add up to the length of
-        // an MMA group per step.
-        const int pbuf = p_t % 3, sbuf = s_t % 3, kslot = s_t & 1, qslot = si & 1;
-        const bool pf = mbar_test(bar_p_full + pbuf, (p_t / 3) & 1);
-        const bool vf = mbar_test(bar_v_full + pbuf, (p_t / 3) & 1);
-        const bool pd = mbar_test(bar_pv_done + sbuf, ((s_t / 3) - 1) & 1);
+        // polled back to back: a poll is a shared-memory round trip
+        const int sbuf = s_t % 3, kslot = s_t & 1, qslot = si & 1;
+        const bool pd = s_t < 3 ? true : mbar_test(bar_pv_done + sbuf, ((s_t / 3) - 1) & 1);   // S buffer free: PV of tile s_t - 3 complete
         const bool kf = mbar_test(bar_k_full + kslot, (s_t >> 1) & 1);
-        // first tile of an item only: O of the previous item read by its closer; Q of this item landed
-        const bool of = (p_n > 0 || p_nonempty == 0) ? true : mbar_test(bar_o_free, (p_nonempty - 1) & 1);
         const bool qf = s_n > 0 ? true : mbar_test(bar_q_full + qslot, (si >> 1) & 1);
-        // ---- O += P V of the oldest pending tile
-        if (p_t < s_t && pf && vf && of) {
-          tc_fence_after();
-          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + pbuf * kTile), kTile / 2);
-          const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts<false>(tmem_O, tmem + pbuf * kPBLK + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), v_hi), idesc_pv,
-                          (p_n == 0 && kk == 0) ? 0u : 1u);
-          tc_commit(bar_pv_done + pbuf);
-          tc_commit(bar_v_free + pbuf);
-          ++p_n; ++p_t;
-          progressed = true;
-        }
-        // ---- S = Q K^T of the next tile (its S buffer is free once PV of tile s_t - 3 is complete)
-        if (s_item < p.items && (s_t < 3 || pd) && kf && qf) {
+        if (pd && kf && qf) {
           tc_fence_after();
           const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ + qslot * kTile), 16);
           const uint64_t dK = make_smem_desc_sw128(smem_u32(sK + kslot * kTile), 16);
@@ -325,16 +293,55 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           tc_commit(bar_s_full + sbuf);
           tc_commit(bar_k_free + kslot);
           ++s_n; ++s_t;
-          progressed = true;
+          guard.reset();
+        } else {
+          ok = guard.idle(s_abort, p.status, 2);
         }
-        if (progressed) guard.reset();
-        else ok = guard.idle(s_abort, p.status, 2);
       }
     }
-  } else if (warp < 8) {
+  } else if (warp == 2) {
+    // -------------------------------------------------------------- PV issuer: O += P V of the oldest pending tile
+    // (its own warp on another scheduler: an issuing thread shares its scheduler with two softmax
+    // warps that are almost always ready, and gets an issue slot only when they stall)
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = make_idesc(1u, 128, kPD, true);
+      int p_item = first_item, p_n = 0, p_cnt = -1, p_t = 0, p_nonempty = 0;
+      bool ok = true;
+      PipeIdle guard;
+      guard.reset();
+      while (ok && p_item < p.items) {
+        if (p_cnt < 0) p_cnt = __ldg(p.clean_cnt + p_item);
+        if (p_n >= p_cnt) {
+          if (p_cnt > 0) ++p_nonempty;
+          p_item += item_step; p_n = 0; p_cnt = -1;
+          continue;
+        }
+        const int pbuf = p_t % 3;
+        const bool pf = mbar_test(bar_p_full + pbuf, (p_t / 3) & 1);
+        const bool vf = mbar_test(bar_v_full + pbuf, (p_t / 3) & 1);
+        // first tile of an item only: O of the previous item must have been read by its closer
+        const bool of = (p_n > 0 || p_nonempty == 0) ? true : mbar_test(bar_o_free, (p_nonempty - 1) & 1);
+        if (pf && vf && of) {
+          tc_fence_after();
+          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + pbuf * kTile), kTile / 2);
+          const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts<false>(tmem_O, tmem + pbuf * kPBLK + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), v_hi), idesc_pv,
+                          (p_n == 0 && kk == 0) ? 0u : 1u);
+          tc_commit(bar_pv_done + pbuf);
+          tc_commit(bar_v_free + pbuf);
+          ++p_n; ++p_t;
+          guard.reset();
+        } else {
+          ok = guard.idle(s_abort, p.status, 10);
+        }
+      }
+    }
+  } else if (warp >= 4) {
     // ----------------------------------------------------------------- softmax
     reg_inc<kPipeSoftmaxRegs>();
-    const int g = warp >> 2;                          // warpgroup: takes the tiles with (global tile counter & 1) == g
+    const int g = (warp >> 2) - 1;                    // warpgroup: takes the tiles with (global tile counter & 1) == g
     const int row = threadIdx.x & 127;                // query row inside the block = TMEM lane
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
     const float c = p.scale_log2;
@@ -533,7 +540,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 0) {
     if (*s_abort) __nanosleep(200000);  // let copies / MMAs in flight land before the CTA's resources go
     tc_fence_after();
     tmem_dealloc(tmem, 512);
