@@ -3,8 +3,10 @@
 // Same arithmetic as fwd.cu (Sec. 2 softmax attention restricted to the kept tiles, Sec. 4.1 sparse
 // branch); different schedule.  Measured on the one-item-per-CTA kernel: a tile's chain
 // S-MMA -> softmax -> PV-MMA is ~3300 clocks long even with the SM to itself, so two independent
-// chains per SM leave the tensor pipe ~45 % busy.  Here one CTA per SM keeps THREE S tiles of the
-// same work item in flight (TMEM: S0 | S1 | S2 | O, 128 columns each):
+// chains per SM leave the tensor pipe ~45 % busy.  Here one CTA per SM keeps the chain open: each
+// softmax warpgroup owns an S buffer and a separate P buffer in TMEM (S0 | S1 | P0 | P1 | O =
+// 128 + 128 + 64 + 64 + 128 columns), so its S buffer is free again as soon as the S row sits in
+// registers and the next-but-one S product runs while the warpgroup is still busy with this tile:
 //   warps 4-7 / 8-11 two softmax warpgroups; the tiles of the CTA's item stream alternate between
 //                    them (global tile counter parity), thread r owns query row r.  The running
 //                    reference maximum of a row travels from the warpgroup of tile t-1 to the
@@ -117,13 +119,14 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   uint64_t* bar_k_free = bars + 6;     // [2] S MMAs that read the slot are complete
   uint64_t* bar_v_full = bars + 8;     // [3]
   uint64_t* bar_v_free = bars + 11;    // [3] PV MMAs that read the slot are complete
-  uint64_t* bar_s_full = bars + 14;    // [3]
-  uint64_t* bar_p_full = bars + 17;    // [3] 128 arrivals
-  uint64_t* bar_pv_done = bars + 20;   // [3] S buffer free again
-  uint64_t* bar_o_free = bars + 23;    // 128 arrivals: the closing warpgroup has read O
-  uint64_t* bar_tok = bars + 24;       // [2] 128 arrivals: warpgroup g has published its reference maxima
-  uint64_t* bar_lsum = bars + 26;      // 128 arrivals: the non-closing warpgroup has published its row sums
-  uint64_t* bar_lsum_ack = bars + 27;  // 128 arrivals: they have been read
+  uint64_t* bar_s_full = bars + 14;    // [2] S of a tile complete in S buffer (tile & 1)
+  uint64_t* bar_s_free = bars + 16;    // [2] 128 arrivals: the warpgroup holds that S row in registers
+  uint64_t* bar_p_full = bars + 18;    // [2] 128 arrivals: P written to P buffer (tile & 1)
+  uint64_t* bar_pv_done = bars + 20;   // [2] PV of a tile complete: P buffer free again
+  uint64_t* bar_o_free = bars + 22;    // 128 arrivals: the closing warpgroup has read O
+  uint64_t* bar_tok = bars + 23;       // [2] 128 arrivals: warpgroup g has published its reference maxima
+  uint64_t* bar_lsum = bars + 25;      // 128 arrivals: the non-closing warpgroup has published its row sums
+  uint64_t* bar_lsum_ack = bars + 26;  // 128 arrivals: they have been read
   float* s_mref = reinterpret_cast<float*>(bars + 32);           // [2][128]
   float2* s_lsum = reinterpret_cast<float2*>(s_mref + 2 * 128);  // [128] (partial row sum, reference it is relative to)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_lsum + 128);
@@ -136,10 +139,11 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       mbar_init(bar_q_full + i, 1); mbar_init(bar_q_free + i, 1);
       mbar_init(bar_k_full + i, 1); mbar_init(bar_k_free + i, 1);
       mbar_init(bar_tok + i, 128);
+      mbar_init(bar_s_full + i, 1); mbar_init(bar_s_free + i, 128);
+      mbar_init(bar_p_full + i, 128); mbar_init(bar_pv_done + i, 1);
     }
     for (int i = 0; i < 3; ++i) {
       mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1);
-      mbar_init(bar_s_full + i, 1); mbar_init(bar_p_full + i, 128); mbar_init(bar_pv_done + i, 1);
     }
     mbar_init(bar_o_free, 128); mbar_init(bar_lsum, 128); mbar_init(bar_lsum_ack, 128);
     int dead = (*reinterpret_cast<volatile int32_t*>(p.status) == SPARKATTN_E_DEVICE_TIMEOUT) ? 1 : 0;
@@ -162,6 +166,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  const uint32_t tmem_P = tmem + 2 * kPBLK;          // P buffer g at columns [256 + 64 g, +64)
   const uint32_t tmem_O = tmem + 3 * kPBLK;
   const bool dead = *s_abort != 0;
   const int first_item = blockIdx.x, item_step = gridDim.x;
@@ -275,8 +280,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           continue;
         }
         // polled back to back: a poll is a shared-memory round trip
-        const int sbuf = s_t % 3, kslot = s_t & 1, qslot = si & 1;
-        const bool pd = s_t < 3 ? true : mbar_test(bar_pv_done + sbuf, ((s_t / 3) - 1) & 1);   // S buffer free: PV of tile s_t - 3 complete
+        const int sbuf = s_t & 1, kslot = s_t & 1, qslot = si & 1;
+        const bool pd = s_t < 2 ? true : mbar_test(bar_s_free + sbuf, ((s_t >> 1) - 1) & 1);   // S buffer free: row of tile s_t - 2 is in registers
         const bool kf = mbar_test(bar_k_full + kslot, (s_t >> 1) & 1);
         const bool qf = s_n > 0 ? true : mbar_test(bar_q_full + qslot, (si >> 1) & 1);
         if (pd && kf && qf) {
@@ -316,21 +321,21 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           p_item += item_step; p_n = 0; p_cnt = -1;
           continue;
         }
-        const int pbuf = p_t % 3;
-        const bool pf = mbar_test(bar_p_full + pbuf, (p_t / 3) & 1);
-        const bool vf = mbar_test(bar_v_full + pbuf, (p_t / 3) & 1);
+        const int pbuf = p_t & 1, vslot = p_t % 3;
+        const bool pf = mbar_test(bar_p_full + pbuf, (p_t >> 1) & 1);
+        const bool vf = mbar_test(bar_v_full + vslot, (p_t / 3) & 1);
         // first tile of an item only: O of the previous item must have been read by its closer
         const bool of = (p_n > 0 || p_nonempty == 0) ? true : mbar_test(bar_o_free, (p_nonempty - 1) & 1);
         if (pf && vf && of) {
           tc_fence_after();
-          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + pbuf * kTile), kTile / 2);
+          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + vslot * kTile), kTile / 2);
           const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
-            mma_ts<false>(tmem_O, tmem + pbuf * kPBLK + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), v_hi), idesc_pv,
+            mma_ts<false>(tmem_O, tmem_P + pbuf * 64 + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), v_hi), idesc_pv,
                           (p_n == 0 && kk == 0) ? 0u : 1u);
           tc_commit(bar_pv_done + pbuf);
-          tc_commit(bar_v_free + pbuf);
+          tc_commit(bar_v_free + vslot);
           ++p_n; ++p_t;
           guard.reset();
         } else {
@@ -376,10 +381,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       for (int n = 0; ok && n < cnt; ++n) {
         const int tt = t + n;
         if ((tt & 1) != g) continue;
-        const int buf = tt % 3;
+        const int buf = g;                          // (tt & 1) == g: this warpgroup's S and P buffers
         const int kb = __ldg(p.clean_list + (int64_t)item * p.kmax + n);
         const int ncols = min(kPBLK, p.N - kb * kPBLK);
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt / 3) & 1, s_abort, p.status, 4));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt >> 1) & 1, s_abort, p.status, 4));
         if (!ok) break;
         tc_fence_after();
         const uint32_t tS = tmem + buf * kPBLK + lane_off;
@@ -387,6 +392,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 #pragma unroll
         for (int ch = 0; ch < kPBLK / 32; ++ch) tmem_ld32(tS + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
         tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_s_free + buf);    // the S buffer can take the next-but-one tile
         if (ncols < kPBLK) {          // ragged last key block: keys >= N get weight 0
 #pragma unroll
           for (int i = 0; i < kPBLK; ++i)
@@ -429,7 +436,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         m_used = m_new;
         if (__any_sync(0xffffffffu, need)) {
           // every PV issued so far must be complete before O is rescaled: the last one is tile tt-1's
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + (tt - 1) % 3, ((tt - 1) / 3) & 1, s_abort, p.status, 6));
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + ((tt - 1) & 1), ((tt - 1) >> 1) & 1, s_abort, p.status, 6));
           if (!ok) break;
           tc_fence_after();
           const uint64_t a2 = pack_f32x2(alpha, alpha);
@@ -449,10 +456,19 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           tc_wait_st();
           tc_fence_before();
         }
+        // This warpgroup's P buffer is free once PV of tile tt-2 is complete.  Waited for BEFORE the
+        // token is passed on: a parity wait is only sound while the barrier is at most one completion
+        // behind the one waited for, and the next warpgroup's rescale path waits on this barrier for
+        // PV of tile tt-1 as soon as it holds the token.
+        if (tt >= 2) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + buf, ((tt >> 1) - 1) & 1, s_abort, p.status, 11));
+          if (!ok) break;
+        }
         s_mref[g * 128 + row] = m_used;
         mbar_arrive(bar_tok + g);
 
-        // P = exp2(S*c - m) as bf16 over the first 64 columns of this S buffer
+        // P = exp2(S*c - m) as bf16 into this warpgroup's P buffer
+        const uint32_t tP = tmem_P + buf * 64 + lane_off;
         const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used, -m_used);
         uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
 #pragma unroll
@@ -468,7 +484,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(e0, e1);
             w[i >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
           }
-          tmem_st16(tS + ch * 16, w);
+          tmem_st16(tP + ch * 16, w);
         }
         const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
         l += ls.x + ls.y;
@@ -494,7 +510,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const float2 other = s_lsum[row];
         mbar_arrive(bar_lsum_ack);
         if (other.x != 0.0f) l += other.x * fast_exp2(other.y - m_used);
-        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + t_last % 3, (t_last / 3) & 1, s_abort, p.status, 9));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + (t_last & 1), (t_last >> 1) & 1, s_abort, p.status, 9));
         if (!ok) break;
         tc_fence_after();
         // normalised O row as bf16 into the item's Q slot (all S MMAs of the item are complete), 128-byte swizzle
