@@ -175,95 +175,91 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   if (dead) {
     // fall through to the teardown
   } else if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (warp converged, lane 0 issues)
-    // K cursor (also loads Q at the start of an item) and V cursor walk the same tile stream.
-    int ki = 0, k_item = first_item, k_n = 0, k_cnt = 0, k_t = 0, k_chunk = 0;   // item ordinal, item, tile, count, global tile, list registers
-    int vi = 0, v_item = first_item, v_n = 0, v_cnt = 0, v_t = 0, v_chunk = 0;
-    bool k_open = false, v_open = false;   // item header processed?
-    bool ok = true;
-    PipeIdle guard;
-    guard.reset();
-    // lane 0 polls, the warp follows: keeps the warp converged for the shuffles below
-    auto uwait = [&](uint64_t* bar, uint32_t parity) {
-      const int r = (lane == 0 && mbar_try_wait(bar, parity)) ? 1 : 0;
-      return __shfl_sync(0xffffffffu, r, 0) != 0;
-    };
-    while (ok && (k_item < p.items || v_item < p.items)) {
-      bool progressed = false;
-      if (k_item < p.items) {
-        if (!k_open) {
-          const int slot = ki & 1;
-          if (ki < 2 || uwait(bar_q_free + slot, ((ki >> 1) - 1) & 1)) {
-            k_cnt = __ldg(p.clean_cnt + k_item);
-            if (lane == 0) {
-              if (k_cnt > 0) {
-                const int qb = k_item % p.nb, bh = k_item / p.nb;
-                mbar_expect_tx(bar_q_full + slot, kTile);
-                tma_load_4d(sQ + slot * kTile, &tmap_q, bar_q_full + slot, 0, qb * kPBLK, bh % p.H, bh / p.H);
-                tma_load_4d(sQ + slot * kTile + kTile / 2, &tmap_q, bar_q_full + slot, 64, qb * kPBLK, bh % p.H, bh / p.H);
+    // ------------------------------------------------------------ TMA producer (one thread)
+    // A K cursor (which also loads Q at the start of an item) and a V cursor walk the same tile
+    // stream; each step tests the barriers both may need back to back and then issues what is
+    // ready.  List entries and item counts are fetched one step ahead of their use.
+    if (lane == 0) {
+      struct Cursor {
+        int ord, item, n, cnt, t;       // item ordinal, item, tile within the item, valid tiles, global tile counter
+        int kb, cnt_next, kb_next_item; // prefetched: this tile's block, next item's count and first block
+        bool open;
+      };
+      auto prefetch_item = [&](Cursor& c) {
+        const int nxt = c.item + item_step;
+        c.cnt_next = nxt < p.items ? __ldg(p.clean_cnt + nxt) : 0;
+        c.kb_next_item = nxt < p.items ? __ldg(p.clean_list + (int64_t)nxt * p.kmax) : 0;
+      };
+      auto init = [&](Cursor& c) {
+        c.ord = 0; c.item = first_item; c.n = 0; c.t = 0; c.open = false;
+        c.cnt = c.item < p.items ? __ldg(p.clean_cnt + c.item) : 0;
+        c.kb = c.item < p.items ? __ldg(p.clean_list + (int64_t)c.item * p.kmax) : 0;
+        prefetch_item(c);
+      };
+      auto next_item = [&](Cursor& c) {
+        c.item += item_step; ++c.ord; c.n = 0; c.open = false;
+        c.cnt = c.cnt_next; c.kb = c.kb_next_item;
+        if (c.item < p.items) prefetch_item(c);
+      };
+      auto next_tile = [&](Cursor& c) {
+        ++c.n; ++c.t;
+        if (c.n < c.cnt) c.kb = __ldg(p.clean_list + (int64_t)c.item * p.kmax + c.n);   // used one step later
+      };
+      Cursor kc, vc;
+      init(kc);
+      init(vc);
+      bool ok = true;
+      PipeIdle guard;
+      guard.reset();
+      while (ok && (kc.item < p.items || vc.item < p.items)) {
+        bool progressed = false;
+        const int qslot = kc.ord & 1, kslot = kc.t & 1, vslot = vc.t % 3;
+        const bool qf = kc.ord < 2 ? true : mbar_test(bar_q_free + qslot, ((kc.ord >> 1) - 1) & 1);
+        const bool kf = kc.t < 2 ? true : mbar_test(bar_k_free + kslot, ((kc.t >> 1) - 1) & 1);
+        const bool vf = vc.t < 3 ? true : mbar_test(bar_v_free + vslot, ((vc.t / 3) - 1) & 1);
+        if (kc.item < p.items) {
+          if (!kc.open) {
+            if (qf) {
+              if (kc.cnt > 0) {
+                const int qb = kc.item % p.nb, bh = kc.item / p.nb;
+                mbar_expect_tx(bar_q_full + qslot, kTile);
+                tma_load_4d(sQ + qslot * kTile, &tmap_q, bar_q_full + qslot, 0, qb * kPBLK, bh % p.H, bh / p.H);
+                tma_load_4d(sQ + qslot * kTile + kTile / 2, &tmap_q, bar_q_full + qslot, 64, qb * kPBLK, bh % p.H, bh / p.H);
+                kc.open = true;
               } else {
-                mbar_arrive(bar_q_full + slot);      // empty item: nothing to load, consumers still step through it
+                mbar_arrive(bar_q_full + qslot);      // empty item: nothing to load, consumers still step through it
+                next_item(kc);
               }
-            }
-            k_open = true;
-            k_n = 0;
-            progressed = true;
-          }
-        }
-        if (k_open) {
-          if (k_n >= k_cnt) {
-            k_item += item_step; ++ki; k_open = false;
-            progressed = true;
-          } else {
-            const int slot = k_t & 1;
-            if (k_t < 2 || uwait(bar_k_free + slot, ((k_t >> 1) - 1) & 1)) {
-              if ((k_n & 31) == 0) k_chunk = (k_n + lane < k_cnt) ? __ldg(p.clean_list + (int64_t)k_item * p.kmax + k_n + lane) : 0;
-              const int kb = __shfl_sync(0xffffffffu, k_chunk, k_n & 31);
-              if (lane == 0) {
-                const int bh = k_item / p.nb;
-                mbar_expect_tx(bar_k_full + slot, kTile);
-                tma_load_4d(sK + slot * kTile, &tmap_k, bar_k_full + slot, 0, kb * kPBLK, bh % p.H, bh / p.H);
-                tma_load_4d(sK + slot * kTile + kTile / 2, &tmap_k, bar_k_full + slot, 64, kb * kPBLK, bh % p.H, bh / p.H);
-              }
-              ++k_n; ++k_t;
               progressed = true;
             }
-          }
-        }
-      }
-      if (v_item < p.items) {
-        if (!v_open) {
-          // the V cursor never passes the K cursor's item header (it needs no header work of its own)
-          if (vi < ki || (vi == ki && k_open)) {
-            v_cnt = __ldg(p.clean_cnt + v_item);
-            v_open = true;
-            v_n = 0;
+          } else if (kc.n >= kc.cnt) {
+            next_item(kc);
+            progressed = true;
+          } else if (kf) {
+            const int bh = kc.item / p.nb;
+            mbar_expect_tx(bar_k_full + kslot, kTile);
+            tma_load_4d(sK + kslot * kTile, &tmap_k, bar_k_full + kslot, 0, kc.kb * kPBLK, bh % p.H, bh / p.H);
+            tma_load_4d(sK + kslot * kTile + kTile / 2, &tmap_k, bar_k_full + kslot, 64, kc.kb * kPBLK, bh % p.H, bh / p.H);
+            next_tile(kc);
             progressed = true;
           }
         }
-        if (v_open) {
-          if (v_n >= v_cnt) {
-            v_item += item_step; ++vi; v_open = false;
+        if (vc.item < p.items) {
+          if (vc.n >= vc.cnt) {
+            // the V cursor never passes the K cursor's item
+            if (vc.ord < kc.ord) { next_item(vc); progressed = true; }
+          } else if (vc.t < kc.t && vf) {
+            const int bh = vc.item / p.nb;
+            mbar_expect_tx(bar_v_full + vslot, kTile);
+            tma_load_4d(sV + vslot * kTile, &tmap_v, bar_v_full + vslot, 0, vc.kb * kPBLK, bh % p.H, bh / p.H);
+            tma_load_4d(sV + vslot * kTile + kTile / 2, &tmap_v, bar_v_full + vslot, 64, vc.kb * kPBLK, bh % p.H, bh / p.H);
+            next_tile(vc);
             progressed = true;
-          } else if (v_t < k_t) {
-            const int slot = v_t % 3;
-            if (v_t < 3 || uwait(bar_v_free + slot, ((v_t / 3) - 1) & 1)) {
-              if ((v_n & 31) == 0) v_chunk = (v_n + lane < v_cnt) ? __ldg(p.clean_list + (int64_t)v_item * p.kmax + v_n + lane) : 0;
-              const int kb = __shfl_sync(0xffffffffu, v_chunk, v_n & 31);
-              if (lane == 0) {
-                const int bh = v_item / p.nb;
-                mbar_expect_tx(bar_v_full + slot, kTile);
-                tma_load_4d(sV + slot * kTile, &tmap_v, bar_v_full + slot, 0, kb * kPBLK, bh % p.H, bh / p.H);
-                tma_load_4d(sV + slot * kTile + kTile / 2, &tmap_v, bar_v_full + slot, 64, kb * kPBLK, bh % p.H, bh / p.H);
-              }
-              ++v_n; ++v_t;
-              progressed = true;
-            }
           }
         }
+        if (progressed) guard.reset();
+        else ok = guard.idle(s_abort, p.status, 1);
       }
-      if (progressed) guard.reset();
-      else ok = __shfl_sync(0xffffffffu, (lane == 0 && !guard.idle(s_abort, p.status, 1)) ? 0 : 1, 0) != 0;
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- S issuer: S = Q K^T of the next tile
@@ -435,7 +431,15 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (l != 0.0f && m_new != m_used) l *= fast_exp2(m_used - m_new);   // own partial sum to the new reference
         m_used = m_new;
         if (__any_sync(0xffffffffu, need)) {
-          // every PV issued so far must be complete before O is rescaled: the last one is tile tt-1's
+          // Every PV issued so far must be complete before O is rescaled: the last one is tile tt-1's,
+          // tracked by the other warpgroup's barrier.  A parity wait is only sound while the barrier is
+          // at most one completion behind the one waited for, and the other warpgroup may not have
+          // waited for PV of tile tt-3 yet; PVs complete in order, so PV of tile tt-2 (this warpgroup's
+          // own barrier, whose previous completion it has already seen) is waited for first.
+          if (tt >= 2) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + buf, ((tt >> 1) - 1) & 1, s_abort, p.status, 12));
+            if (!ok) break;
+          }
           ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + ((tt - 1) & 1), ((tt - 1) >> 1) & 1, s_abort, p.status, 6));
           if (!ok) break;
           tc_fence_after();
@@ -456,14 +460,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           tc_wait_st();
           tc_fence_before();
         }
-        // This warpgroup's P buffer is free once PV of tile tt-2 is complete.  Waited for BEFORE the
-        // token is passed on: a parity wait is only sound while the barrier is at most one completion
-        // behind the one waited for, and the next warpgroup's rescale path waits on this barrier for
-        // PV of tile tt-1 as soon as it holds the token.
-        if (tt >= 2) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + buf, ((tt >> 1) - 1) & 1, s_abort, p.status, 11));
-          if (!ok) break;
-        }
         s_mref[g * 128 + row] = m_used;
         mbar_arrive(bar_tok + g);
 
@@ -483,6 +479,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             else lsum0 = fadd2(lsum0, pack_f32x2(e0, e1));
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(e0, e1);
             w[i >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          if (ch == 0 && tt >= 2) {
+            // this warpgroup's P buffer is free once PV of tile tt-2 is complete (normally long ago)
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + buf, ((tt >> 1) - 1) & 1, s_abort, p.status, 11));
           }
           tmem_st16(tP + ch * 16, w);
         }
