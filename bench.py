@@ -42,7 +42,7 @@ METRIC = "block-sparse attn effective TFLOP/s (kept FLOPs), select+fwd, 97% spar
 UNIT = "TFLOP/s"
 # DRAM bytes (read + write) of one bf16 forward launch on the default workload (wan14b, 97 %),
 # from the one-pass ncu capture summarised in profiles/launch_list_wan14b_s97.md.
-FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2406387968 + 757543424}
+FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2580123136 + 761104384}   # ncu one-pass capture of the full-size fwd_pipe_kernel launch
 
 
 def load_peaks():
@@ -303,9 +303,10 @@ def run_ours(args, w):
     kernels = {
         "select": {"ms": ms_sel, "launches_per_step": 2, "algorithmic_bytes": sel_bytes,
                    "GBps": sel_bytes / (ms_sel * 1e-3) / 1e9, "frac_of_hbm_peak": sel_bytes / (ms_sel * 1e-3) / 1e9 / peaks["hbm"]},
-        "fwd_bf16": {"ms": ms_fwd, "launches_per_step": 1, "TFLOPs": fwd_tflops},
+        "fwd_bf16": {"ms": ms_fwd, "launches_per_step": 2 if (w.d == 128 and w.block == 128) else 1, "TFLOPs": fwd_tflops},
     }
-    roofline = {"kernel": "fwd_kernel<128,128,bf16>", "bound": "tensor", "achieved": fwd_tflops, "peak": peaks["bf16"],
+    pipelined = w.d == 128 and w.block == 128   # bf16 at this tile shape runs the persistent pipelined kernel (+ list pre-pass)
+    roofline = {"kernel": "fwd_pipe_kernel (bf16, d=128, 128x128)" if pipelined else f"fwd_kernel<{w.d},{w.block},bf16>", "bound": "tensor", "achieved": fwd_tflops, "peak": peaks["bf16"],
                 "unit": "TFLOP/s", "frac": fwd_tflops / peaks["bf16"], "traffic": FWD_DRAM_TRAFFIC_BYTES.get(w.name) if w.sparsity == 0.97 else None,
                 "peak_source": f"{peaks['source']} bf16 burst (sustained {peaks['bf16_sustained']})",
                 "flops_per_launch": flops, "ms_per_launch": ms_fwd}
@@ -428,7 +429,7 @@ def run_ours(args, w):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": config_dict(w, "bf16"),
-            "kept_flops_per_step_per_gpu": flops, "clocks": clocks, "gpu_launches": 3 * K,
+            "kept_flops_per_step_per_gpu": flops, "clocks": clocks, "gpu_launches": (4 if pipelined else 3) * K,
             "kernels": kernels, "roofline": roofline, "fp8": fp8, "compensation": comp, "e2e": e2e, "cpu_baseline": cpu,
         }
         if sweep is not None:
