@@ -504,11 +504,17 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
         s_lsum[row] = make_float2(l, m_used);
         mbar_arrive(bar_lsum);
+        // The two hand-over barriers are waited on by whichever warpgroup closes (or does not close) the
+        // next item, with a phase parity counted in items; that is only sound if no thread of this
+        // warpgroup runs ahead while the phase its own warpgroup completes is still open (items of one
+        // or two tiles make that possible).  So the warpgroup lines up after arriving.
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");
       } else {
         ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum, nonempty & 1, s_abort, p.status, 8));
         if (!ok) break;
         const float2 other = s_lsum[row];
         mbar_arrive(bar_lsum_ack);
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");     // see the note at the hand-over above
         if (other.x != 0.0f) l += other.x * fast_exp2(other.y - m_used);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + (t_last & 1), (t_last >> 1) & 1, s_abort, p.status, 9));
         if (!ok) break;

@@ -165,3 +165,31 @@ def test_small_structured_full_parity_fp8(w):
                                         scales=tuple(s[0].cpu() for s in scales))
     items = [(h, i) for h in range(w.H) for i in range(w.nb)]
     _compare_items(out[0], lse[0], ref_out, ref_lse, items, w.block, w.N, FP8_RELRMS, None, lse_tol=2e-2)
+
+
+@pytest.mark.parametrize("seed,kmax", [(0, 3), (1, 6)])
+def test_persistent_path_short_and_empty_lists(seed, kmax):
+    """bf16, d = 128, 128-token blocks with more work items than SMs: every CTA of the persistent kernel
+    walks several items whose kept lists have 0, 1, 2, ... blocks (item boundaries, hand-over of the row
+    sums between the two softmax warpgroups, empty items), ragged last block included.  Compared in full
+    against the oracle, and two runs must agree bitwise."""
+    w = _small(41 + seed, 3, 128, (5, 18, 18), 128, 0.0)   # N = 1620: nb = 13 (ragged), 39 items per head
+    w = workloads.Workload(w.name, w.cfg_id, 1, 12, w.d, w.grid, w.block, w.sparsity)   # 156 items > 148 SMs
+    q, k, v = workloads.structured_qkv(w)
+    g = torch.Generator().manual_seed(100 + seed)
+    idx = torch.stack([torch.stack([torch.randperm(w.nb, generator=g)[:kmax] for _ in range(w.nb)]) for _ in range(w.H)]).to(torch.int32)
+    cnt = torch.randint(0, kmax + 1, (w.H, w.nb), generator=g, dtype=torch.int32)
+    cnt[0, 0] = 0; cnt[0, 1] = 1; cnt[0, 2] = 1; cnt[0, 3] = 2; cnt[0, 4] = 0; cnt[0, 5] = 0; cnt[0, 6] = kmax
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    out, lse = sa.fwd(qd, kd, vd, idx[None].to(DEV), cnt[None].to(DEV), w.block, return_lse=True, check_status=True)
+    out2, lse2 = sa.fwd(qd, kd, vd, idx[None].to(DEV), cnt[None].to(DEV), w.block, return_lse=True, check_status=True)
+    assert torch.equal(out, out2) and torch.equal(lse.view(torch.int32), lse2.view(torch.int32))
+    ref_out, ref_lse = oracle.attention(q[0], k[0], v[0], idx, cnt, w.block)
+    items = [(h, i) for h in range(w.H) for i in range(w.nb) if cnt[h, i] > 0]
+    sel = [n for n, (h, i) in enumerate((h, i) for h in range(w.H) for i in range(w.nb)) if cnt[h, i] > 0]
+    _compare_items(out[0], lse[0], ref_out[sel], ref_lse[sel], items, w.block, w.N, BF16_RELRMS, BF16_MAXABS)
+    for h in range(w.H):
+        for i in range(w.nb):
+            if cnt[h, i] == 0:
+                rows = slice(i * w.block, min(w.N, (i + 1) * w.block))
+                assert torch.all(out[0, h, rows] == 0) and torch.all(torch.isneginf(lse[0, h, rows]))
