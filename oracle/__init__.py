@@ -98,12 +98,16 @@ def attention(
     items: Optional[Sequence[Tuple[int, int]]] = None,
     scales: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
     softmax_scale: float = 0.0,
+    frame_tokens: int = 0,
+    window: int = 0,
 ):
     """ATT-0.  q, k, v: [H, N, d] bf16, or uint8 E4M3 codes with
     ``scales = (q_scale, k_scale, v_scale)`` each fp32 [H, nb].
     kept_idx int32 [H, nb, kmax], kept_cnt int32 [H, nb].
     Returns (out fp64 [n_items, block, d], lse fp64 [n_items, block]) for the
-    (head, query-block) pairs in ``items`` (default: all, head-major)."""
+    (head, query-block) pairs in ``items`` (default: all, head-major).
+    WIN-0: with ``frame_tokens`` = F > 0, key j counts for query i only if its frame j // F lies in
+    (i // F - window, i // F]; a row with no such kept key gives out = 0, lse = -inf."""
     L = _load()
     H, N, d = q.shape
     nb = (N + block - 1) // block
@@ -130,7 +134,7 @@ def attention(
         ctypes.c_int(dtype), _ptr(qq), _ptr(kk), _ptr(vv), _ptr(sq), _ptr(sk), _ptr(sv),
         ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d), ctypes.c_int(block),
         _ptr(ki), _ptr(kc), ctypes.c_int(kmax), ctypes.c_double(softmax_scale),
-        _ptr(it), ctypes.c_int(n_items), _ptr(out), _ptr(lse))
+        _ptr(it), ctypes.c_int(n_items), ctypes.c_int(frame_tokens), ctypes.c_int(window), _ptr(out), _ptr(lse))
     if rc != 0:
         raise ValueError("kept_idx holds a block index outside [0, nb)")
     return out, lse
@@ -147,9 +151,12 @@ def pool(x: torch.Tensor, block: int) -> torch.Tensor:
     return out
 
 
-def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, return_scores: bool = False):
+def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, return_scores: bool = False,
+           frame_tokens: int = 0, window: int = 0):
     """SEL-1.  q, k: [H, N, d] bf16.  Returns kept_idx int32 [H, nb, topk]
-    (ascending), kept_cnt int32 [H, nb] (and the fp32 scores [H, nb, nb])."""
+    (ascending), kept_cnt int32 [H, nb] (and the fp32 scores [H, nb, nb]).
+    WIN-0: with ``frame_tokens`` > 0 only key blocks inside the causal frame window of the query
+    block are candidates; kept_cnt = min(topk, candidates), unused list entries are -1."""
     L = _load()
     H, N, d = q.shape
     nb = (N + block - 1) // block
@@ -158,7 +165,7 @@ def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, return_score
     scores = torch.empty((H, nb, nb), dtype=torch.float32) if return_scores else None
     rc = L.oracle_select(_ptr(_raw16(q)), _ptr(_raw16(k)), ctypes.c_int(H), ctypes.c_int(N),
                          ctypes.c_int(d), ctypes.c_int(block), ctypes.c_int(topk),
-                         _ptr(idx), _ptr(cnt), _ptr(scores))
+                         ctypes.c_int(frame_tokens), ctypes.c_int(window), _ptr(idx), _ptr(cnt), _ptr(scores))
     if rc != 0:
         raise ValueError("topk must be in [1, nb]")
     return (idx, cnt, scores) if return_scores else (idx, cnt)

@@ -25,6 +25,15 @@
  *          oracle_quant_fp8_per_token   the same with one scale per token.
  *   CMP-0  oracle_comp_state / oracle_comp_apply   low-rank compensation branch and
  *                             token-wise gate fusion (Sec. 4.1), fp64.
+ *   WIN-0  frame_tokens / window arguments of oracle_attention and oracle_select:
+ *                             the causal window of the auto-regressive extension
+ *                             (Sec. 1, "Extension to auto-regressive video diffusion":
+ *                             the attention "can be restricted to a causal window";
+ *                             no formula is given).  Reading: tokens come in frames of
+ *                             F = frame_tokens; key j counts for query i iff
+ *                             j / F lies in (i / F - window, i / F].  Selection only
+ *                             ranks the key blocks that hold such a key for some row
+ *                             of the query block.
  *
  * OpenMP only distributes independent work items (one (head, query block) or
  * one (head, block) each); inside an item everything is a scalar loop in the
@@ -110,7 +119,7 @@ static inline double load_elem(const void* x, const float* scale, int dtype, int
 int oracle_attention(int dtype, const void* q, const void* k, const void* v, const float* q_scale,
                      const float* k_scale, const float* v_scale, int H, int N, int d, int blk,
                      const int32_t* kept_idx, const int32_t* kept_cnt, int kmax, double scale,
-                     const int32_t* items, int n_items, double* out, double* lse) {
+                     const int32_t* items, int n_items, int frame_tokens, int window, double* out, double* lse) {
   const int64_t nb = ((int64_t)N + blk - 1) / blk;
   if (scale == 0.0) scale = 1.0 / sqrt((double)d);
   int bad = 0;
@@ -135,6 +144,11 @@ int oracle_attention(int dtype, const void* q, const void* k, const void* v, con
         const int64_t kb = list[t];
         if (kb < 0 || kb >= nb) { bad = 1; continue; }
         for (int64_t j = kb * blk; j < (kb + 1) * blk && j < N; ++j) {
+          /* causal window over frames (WIN-0): key frame in (query frame - window, query frame] */
+          if (frame_tokens > 0) {
+            const int64_t fi = i / frame_tokens, fj = j / frame_tokens;
+            if (fj > fi || fj <= fi - window) continue;
+          }
           double acc = 0.0;
           for (int c = 0; c < d; ++c) acc += qrow[c] * load_elem(k, k_scale, dtype, N, d, blk, nb, h, j, c);
           s[nk] = scale * acc;
@@ -201,6 +215,7 @@ static int int_cmp(const void* a, const void* b) {
 
 /* scores_out (optional, may be NULL): [H][nb][nb] fp32 scores, for inspection in tests. */
 int oracle_select(const uint16_t* q, const uint16_t* k, int H, int N, int d, int blk, int topk,
+                  int frame_tokens, int window,
                   int32_t* kept_idx /* [H][nb][topk] */, int32_t* kept_cnt /* [H][nb] or NULL */,
                   float* scores_out) {
   const int64_t nb = ((int64_t)N + blk - 1) / blk;
@@ -220,11 +235,27 @@ int oracle_select(const uint16_t* q, const uint16_t* k, int H, int N, int d, int
       sc[j].j = (int32_t)j;
       if (scores_out) scores_out[hi * nb + j] = a;
     }
-    qsort(sc, nb, sizeof(scored_t), scored_cmp);
+    /* WIN-0: with a causal window only the key blocks that hold at least one key some row of the
+     * query block may attend to are candidates: a contiguous run [jlo, jhi] of block indices. */
+    int64_t jlo = 0, jhi = nb - 1;
+    if (frame_tokens > 0) {
+      const int64_t qb = hi % nb;
+      const int64_t r0 = qb * blk, r1 = ((qb + 1) * blk < N ? (qb + 1) * blk : N) - 1;
+      int64_t f0 = r0 / frame_tokens - window + 1;
+      if (f0 < 0) f0 = 0;
+      int64_t kend = (r1 / frame_tokens + 1) * frame_tokens;
+      if (kend > N) kend = N;
+      jlo = f0 * frame_tokens / blk;
+      jhi = (kend - 1) / blk;
+    }
+    const int64_t ncand = jhi - jlo + 1;
+    qsort(sc + jlo, ncand, sizeof(scored_t), scored_cmp);
+    const int cnt = topk < ncand ? topk : (int)ncand;
     int32_t* dst = kept_idx + hi * topk;
-    for (int t = 0; t < topk; ++t) dst[t] = sc[t].j;
-    qsort(dst, topk, sizeof(int32_t), int_cmp);
-    if (kept_cnt) kept_cnt[hi] = topk;
+    for (int t = 0; t < cnt; ++t) dst[t] = sc[jlo + t].j;
+    qsort(dst, cnt, sizeof(int32_t), int_cmp);
+    for (int t = cnt; t < topk; ++t) dst[t] = -1;     /* unused tail of the list */
+    if (kept_cnt) kept_cnt[hi] = cnt;
     free(sc);
   }
   free(pq); free(pk);
