@@ -157,6 +157,29 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
                   const int32_t* kept_cnt, int32_t kmax, void* out_bf16, float* lse, void* workspace,
                   size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * Causal frame window (Sec. 1, "Extension to auto-regressive video diffusion":
+ * the compensated sparse attention "can be restricted to a causal window"; the
+ * paper gives no formula, so the reading is:)  tokens come in frames of
+ * `frame_tokens` consecutive tokens; key token j counts for query token i iff
+ *     i / frame_tokens - window_frames  <  j / frame_tokens  <=  i / frame_tokens.
+ * sparkattn_select_window ranks only the key blocks that hold such a key for
+ * some row of the query block (a contiguous run of blocks): kept_cnt =
+ * min(topk, candidates) (kept_cnt must not be NULL) and the unused tail of a
+ * list is -1.  sparkattn_fwd_window evaluates the same softmax attention as
+ * sparkattn_fwd over the kept blocks with the token-exact window mask; a query
+ * row without any admissible kept key gives a zero output row and lse = -inf.
+ * All other arguments, layouts and errors are those of sparkattn_select /
+ * sparkattn_fwd; frame_tokens < 1 or window_frames < 1 is SPARKATTN_E_INVALID_ARG.
+ */
+int sparkattn_select_window(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                            int32_t frame_tokens, int32_t window_frames, int32_t* kept_idx, int32_t* kept_cnt,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+int sparkattn_fwd_window(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+                         const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                         const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window_frames,
+                         void* out_bf16, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Synchronises the stream and returns the device status word of a workspace
  * (SPARKATTN_OK, SPARKATTN_E_BAD_INDEX or SPARKATTN_E_DEVICE_TIMEOUT). */
 int sparkattn_read_status(void* workspace, void* cuda_stream);

@@ -36,7 +36,7 @@ EXPORTS = (
     "sparkattn_quant_fp8", "sparkattn_quant_fp8_per_token", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
     "sparkattn_attention_host", "sparkattn_select_noalloc", "sparkattn_select_noalloc_max_bytes",
     "sparkattn_select_noalloc_status", "sparkattn_comp_workspace_bytes", "sparkattn_comp_state",
-    "sparkattn_comp_apply",
+    "sparkattn_comp_apply", "sparkattn_select_window", "sparkattn_fwd_window",
 )
 
 
@@ -95,6 +95,10 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_select_noalloc_max_bytes.restype = sz
         L.sparkattn_select_noalloc_status.restype = ctypes.c_int
         L.sparkattn_select_noalloc_status.argtypes = [vp]
+        L.sparkattn_select_window.restype = ctypes.c_int
+        L.sparkattn_select_window.argtypes = [sp, vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.sparkattn_fwd_window.restype = ctypes.c_int
+        L.sparkattn_fwd_window.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, sz, vp]
         L.sparkattn_comp_workspace_bytes.restype = sz
         L.sparkattn_comp_workspace_bytes.argtypes = [sp, vp]
         L.sparkattn_comp_state.restype = ctypes.c_int
@@ -156,9 +160,9 @@ def read_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = N
 def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, *,
            kept_idx: Optional[torch.Tensor] = None, kept_cnt: Optional[torch.Tensor] = None,
            workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-           ) -> Tuple[torch.Tensor, torch.Tensor]:
-    """``sparkattn_select``: q, k bf16 [B,H,N,d] on the device -> (kept_idx int32
-    [B,H,nb,topk] ascending, kept_cnt int32 [B,H,nb])."""
+           frame_tokens: int = 0, window: int = 0) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_select`` (``sparkattn_select_window`` when ``frame_tokens`` > 0): q, k bf16
+    [B,H,N,d] on the device -> (kept_idx int32 [B,H,nb,topk] ascending, kept_cnt int32 [B,H,nb])."""
     _same_layout(q, k)
     shape = make_shape(q, block)
     B, H, N, _ = q.shape
@@ -169,6 +173,12 @@ def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, *,
         kept_cnt = torch.empty((B, H, nb), dtype=torch.int32, device=q.device)
     if workspace is None:
         workspace = alloc_workspace(shape, 0, topk, q.device)
+    if frame_tokens > 0:
+        rc = lib().sparkattn_select_window(ctypes.byref(shape), _ptr(q), _ptr(k), topk, frame_tokens, window,
+                                           _ptr(kept_idx), _ptr(kept_cnt), _ptr(workspace), workspace.numel(),
+                                           _stream_ptr(stream))
+        _check(rc, "sparkattn_select_window")
+        return kept_idx, kept_cnt
     rc = lib().sparkattn_select(ctypes.byref(shape), _ptr(q), _ptr(k), topk, _ptr(kept_idx), _ptr(kept_cnt),
                                 _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     _check(rc, "sparkattn_select")
@@ -225,9 +235,10 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tenso
         scales: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
         softmax_scale: float = 0.0, out: Optional[torch.Tensor] = None, return_lse: bool = False,
         workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-        check_status: bool = False):
-    """``sparkattn_fwd``.  bf16 q,k,v, or uint8 E4M3 codes with ``scales=(q_scale,
-    k_scale, v_scale)``.  Returns out bf16 [B,H,N,d] (and lse fp32 [B,H,N])."""
+        check_status: bool = False, frame_tokens: int = 0, window: int = 0):
+    """``sparkattn_fwd`` (``sparkattn_fwd_window`` when ``frame_tokens`` > 0).  bf16 q,k,v, or uint8
+    E4M3 codes with ``scales=(q_scale, k_scale, v_scale)``.  Returns out bf16 [B,H,N,d] (and lse
+    fp32 [B,H,N])."""
     _same_layout(q, k, v)
     shape = make_shape(q, block, softmax_scale)
     B, H, N, _ = q.shape
@@ -239,9 +250,14 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tenso
     if workspace is None:
         workspace = alloc_workspace(shape, 1, kmax, q.device)
     sq, sk, sv = scales if scales is not None else (None, None, None)
-    rc = lib().sparkattn_fwd(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(sq), _ptr(sk), _ptr(sv),
-                             _ptr(kept_idx), _ptr(kept_cnt), kmax, _ptr(out), _ptr(lse), _ptr(workspace),
-                             workspace.numel(), _stream_ptr(stream))
+    if frame_tokens > 0:
+        rc = lib().sparkattn_fwd_window(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(sq), _ptr(sk),
+                                        _ptr(sv), _ptr(kept_idx), _ptr(kept_cnt), kmax, frame_tokens, window,
+                                        _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    else:
+        rc = lib().sparkattn_fwd(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(sq), _ptr(sk), _ptr(sv),
+                                 _ptr(kept_idx), _ptr(kept_cnt), kmax, _ptr(out), _ptr(lse), _ptr(workspace),
+                                 workspace.numel(), _stream_ptr(stream))
     _check(rc, "sparkattn_fwd")
     if check_status:
         _check(read_status(workspace, stream), "sparkattn_fwd (device status)")

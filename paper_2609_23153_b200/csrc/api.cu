@@ -59,9 +59,30 @@ size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, 
   return 0;
 }
 
+namespace {
+int select_impl(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                int32_t frame_tokens, int32_t window, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                size_t workspace_bytes, void* cuda_stream);
+}  // namespace
+
 int sparkattn_select(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
                      int32_t* kept_idx, int32_t* kept_cnt, void* workspace, size_t workspace_bytes,
                      void* cuda_stream) {
+  return select_impl(shape, q_bf16, k_bf16, topk, 0, 0, kept_idx, kept_cnt, workspace, workspace_bytes, cuda_stream);
+}
+
+int sparkattn_select_window(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                            int32_t frame_tokens, int32_t window_frames, int32_t* kept_idx, int32_t* kept_cnt,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (frame_tokens < 1 || window_frames < 1 || kept_cnt == nullptr) return SPARKATTN_E_INVALID_ARG;
+  return select_impl(shape, q_bf16, k_bf16, topk, frame_tokens, window_frames, kept_idx, kept_cnt, workspace,
+                     workspace_bytes, cuda_stream);
+}
+
+namespace {
+int select_impl(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                int32_t frame_tokens, int32_t window, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                size_t workspace_bytes, void* cuda_stream) {
   int rc = check_shape(shape);
   if (rc != SPARKATTN_OK) return rc;
   if (!q_bf16 || !k_bf16 || !kept_idx || !workspace) return SPARKATTN_E_INVALID_ARG;
@@ -72,8 +93,9 @@ int sparkattn_select(const sparkattn_shape_t* shape, const void* q_bf16, const v
   if (workspace_bytes < select_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
-  return launch_select(*shape, q_bf16, k_bf16, topk, kept_idx, kept_cnt, workspace, stream);
+  return launch_select(*shape, q_bf16, k_bf16, topk, frame_tokens, window, kept_idx, kept_cnt, workspace, stream);
 }
+}  // namespace
 
 int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes, float* scales,
                         uint32_t flags, void* cuda_stream) {
@@ -93,10 +115,35 @@ int sparkattn_quant_fp8_per_token(const sparkattn_shape_t* shape, const void* x_
   return launch_quant_fp8_per_token(*shape, x_bf16, codes, scales, static_cast<cudaStream_t>(cuda_stream));
 }
 
+namespace {
+int fwd_impl(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+             const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+             const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window, void* out_bf16, float* lse,
+             void* workspace, size_t workspace_bytes, void* cuda_stream);
+}  // namespace
+
 int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
                   const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                   const int32_t* kept_cnt, int32_t kmax, void* out_bf16, float* lse, void* workspace,
                   size_t workspace_bytes, void* cuda_stream) {
+  return fwd_impl(shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, 0, 0, out_bf16, lse,
+                  workspace, workspace_bytes, cuda_stream);
+}
+
+int sparkattn_fwd_window(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+                         const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                         const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window_frames,
+                         void* out_bf16, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (frame_tokens < 1 || window_frames < 1) return SPARKATTN_E_INVALID_ARG;
+  return fwd_impl(shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens,
+                  window_frames, out_bf16, lse, workspace, workspace_bytes, cuda_stream);
+}
+
+namespace {
+int fwd_impl(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+             const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+             const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window, void* out_bf16, float* lse,
+             void* workspace, size_t workspace_bytes, void* cuda_stream) {
   int rc = check_shape(shape);
   if (rc != SPARKATTN_OK) return rc;
   if (dtype != SPARKATTN_BF16 && dtype != SPARKATTN_FP8_E4M3) return SPARKATTN_E_INVALID_ARG;
@@ -110,9 +157,10 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out_bf16) || !aligned256(workspace))
     return SPARKATTN_E_MISALIGNED;
   if (workspace_bytes < fwd_workspace_bytes(*shape, kmax)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
-  return launch_fwd(*shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, out_bf16, lse,
-                    workspace, static_cast<cudaStream_t>(cuda_stream));
+  return launch_fwd(*shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
+                    out_bf16, lse, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
+}  // namespace
 
 namespace {
 int check_comp(const sparkattn_shape_t* s, int32_t rank, const int32_t* grid, const int32_t* axis, const float* freq) {

@@ -78,6 +78,7 @@ struct FwdParams {
   float* lse;
   int32_t* status;
   int H, N, nb, kmax;
+  int frame_tokens, window;  // causal frame window (0 = none): key frame in (query frame - window, query frame]
   int64_t stride_b, stride_h, stride_n;
   float scale_log2;  // softmax_scale * log2(e)
 };
@@ -275,6 +276,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
     const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
     const int q_row = qb * BLK + row;
     const bool row_valid = row < BLK && q_row < p.N;
+    // keys this row may attend to: [klo, khi) (everything up to N without a causal window)
+    int klo = 0, khi = p.N;
+    if (p.frame_tokens > 0) {
+      const int fi = min(q_row, p.N - 1) / p.frame_tokens;
+      klo = max(fi - p.window + 1, 0) * p.frame_tokens;
+      khi = (int)min((long long)(fi + 1) * p.frame_tokens, (long long)p.N);
+    }
     float m_used = 0.0f, l = 0.0f;
     float q_sc = 1.0f, v_max = 1.0f;
     if constexpr (FP8) {
@@ -286,7 +294,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
     bool ok = true;
     for (int n = 0; ok && n < ntiles; ++n) {
       const int kb = s_list[n];
-      const int ncols = min(BLK, p.N - kb * BLK);    // valid keys in this block
+      const int c_lo_tile = klo - kb * BLK, c_hi_tile = khi - kb * BLK;   // this row's valid columns of the tile
       float c = p.scale_log2;                        // logit -> log2 units
       float p_off = 0.0f;                            // log2 of the factor folded into P
       if constexpr (FP8) {
@@ -295,7 +303,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       }
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
-        const int nc = ncols - hf * HALF;            // valid keys in this half (may be <= 0)
+        const int c_lo = c_lo_tile - hf * HALF, c_hi = c_hi_tile - hf * HALF;   // valid columns of this half: [c_lo, c_hi)
         ok = mbar_wait(bar_s_full + hf, n & 1, s_abort, p.status, 8);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -307,10 +315,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         for (int ch = 0; ch < HALF / 32; ++ch)
           tmem_ld32(tmem_S + lane_off + hf * HALF + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
         tc_wait_ld();
-        if (nc < HALF) {  // ragged last key block: keys >= N get weight 0
+        if (c_lo > 0 || c_hi < HALF) {  // ragged last key block / keys outside the causal window get weight 0
 #pragma unroll
           for (int i = 0; i < HALF; ++i)
-            if (i >= nc) sr[i] = 0xff800000u;
+            if (i < c_lo || i >= c_hi) sr[i] = 0xff800000u;
         }
         float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
         float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
@@ -326,8 +334,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         const float m_new = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
         float alpha = 1.0f;
         bool need = false;
-        if (n == 0 && hf == 0) {
-          m_used = m_new;
+        if ((n == 0 && hf == 0) || m_used == -INFINITY) {
+          m_used = m_new;               // first half, or nothing accumulated for this row yet (all keys so far masked)
         } else if (m_new > m_used + (FP8 ? 0.0f : kLazyRescaleLog2)) {
           alpha = fast_exp2(m_used - m_new);
           m_used = m_new;
@@ -360,7 +368,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         }
 
         // P = exp2(S*c - m) in the input precision, written over the start of this S half
-        const float neg_m = p_off - m_used;
+        const float neg_m = m_used == -INFINITY ? 0.0f : p_off - m_used;   // a fully masked row: exp2(-inf) = 0, not NaN
         const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
         uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
         constexpr int kWordsPerChunk = FP8 ? 8 : 16;   // P words produced from 32 S columns
@@ -420,7 +428,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
-        float inv = 1.0f / l;
+        float inv = l > 0.0f ? 1.0f / l : 0.0f;     // no admissible key at all: zero row, lse = -inf
         if constexpr (FP8) inv *= v_max * fast_exp2(-kFp8PScaleLog2);
 #pragma unroll
         for (int ch = 0; ch < D / 32; ++ch) {
@@ -514,11 +522,12 @@ static int launch_fwd_t(const sparkattn_shape_t& s, const CUtensorMap& mq, const
 
 int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void* k, const void* v,
                const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
-               const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream) {
+               const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse, void* workspace,
+               cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
 #ifndef SPARKATTN_FWD_NO_PIPE
   if (!fp8 && s.d == 128 && s.block == 128)
-    return launch_fwd_pipe(s, q, k, v, kept_idx, kept_cnt, kmax, out, lse, workspace, stream);
+    return launch_fwd_pipe(s, q, k, v, kept_idx, kept_cnt, kmax, frame_tokens, window, out, lse, workspace, stream);
 #endif
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;
@@ -539,6 +548,8 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
   prm.N = s.N;
   prm.nb = (s.N + s.block - 1) / s.block;
   prm.kmax = kmax;
+  prm.frame_tokens = frame_tokens;
+  prm.window = window;
   prm.stride_b = s.stride_b;
   prm.stride_h = s.stride_h;
   prm.stride_n = s.stride_n;

@@ -50,6 +50,7 @@ struct PipeParams {
   float* lse;
   int32_t* status;
   int H, N, nb, kmax, items;
+  int frame_tokens, window;    // causal frame window (0 = none): key frame in (query frame - window, query frame]
   int64_t stride_b, stride_h, stride_n;
   float scale_log2;
 };
@@ -358,6 +359,13 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       const int h = bh % p.H, b = bh / p.H;
       const int q_row = qb * kPBLK + row;
       const bool row_valid = q_row < p.N;
+      // keys this row may attend to: [klo, khi) (everything up to N without a causal window)
+      int klo = 0, khi = p.N;
+      if (p.frame_tokens > 0) {
+        const int fi = min(q_row, p.N - 1) / p.frame_tokens;
+        klo = max(fi - p.window + 1, 0) * p.frame_tokens;
+        khi = (int)min((long long)(fi + 1) * p.frame_tokens, (long long)p.N);
+      }
       if (cnt == 0) {
         if (g == 0) {
           // empty kept list: zero output, lse = -inf; release the item's Q slot
@@ -379,7 +387,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if ((tt & 1) != g) continue;
         const int buf = g;                          // (tt & 1) == g: this warpgroup's S and P buffers
         const int kb = __ldg(p.clean_list + (int64_t)item * p.kmax + n);
-        const int ncols = min(kPBLK, p.N - kb * kPBLK);
+        const int c_lo = klo - kb * kPBLK, c_hi = khi - kb * kPBLK;   // this row's valid columns of the tile: [c_lo, c_hi)
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt >> 1) & 1, s_abort, p.status, 4));
         if (!ok) break;
         tc_fence_after();
@@ -390,10 +398,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + buf);    // the S buffer can take the next-but-one tile
-        if (ncols < kPBLK) {          // ragged last key block: keys >= N get weight 0
+        if (c_lo > 0 || c_hi < kPBLK) {   // ragged last key block / keys outside the causal window get weight 0
 #pragma unroll
           for (int i = 0; i < kPBLK; ++i)
-            if (i >= ncols) sr[i] = 0xff800000u;
+            if (i < c_lo || i >= c_hi) sr[i] = 0xff800000u;
         }
         float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
         float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
@@ -420,7 +428,9 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           m_new = m_tile;
         } else {
           const float m_prev = s_mref[(g ^ 1) * 128 + row];
-          if (m_tile > m_prev + kPipeLazyLog2) {
+          if (m_prev == -INFINITY) {
+            m_new = m_tile;             // nothing accumulated for this row yet (all keys so far masked): O row and l are 0
+          } else if (m_tile > m_prev + kPipeLazyLog2) {
             m_new = m_tile;
             alpha = fast_exp2(m_prev - m_tile);
             need = true;
@@ -465,7 +475,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
         // P = exp2(S*c - m) as bf16 into this warpgroup's P buffer
         const uint32_t tP = tmem_P + buf * 64 + lane_off;
-        const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(-m_used, -m_used);
+        const float neg_m = m_used == -INFINITY ? 0.0f : -m_used;     // a fully masked row: exp2(-inf) = 0, not NaN
+        const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
         uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
 #pragma unroll
         for (int ch = 0; ch < kPBLK / 32; ++ch) {
@@ -520,7 +531,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (!ok) break;
         tc_fence_after();
         // normalised O row as bf16 into the item's Q slot (all S MMAs of the item are complete), 128-byte swizzle
-        const float inv = 1.0f / l;
+        const float inv = l > 0.0f ? 1.0f / l : 0.0f;     // no admissible key at all: zero row, lse = -inf
         unsigned char* slot = sQ + qslot * kTile;
 #pragma unroll 1
         for (int ch = 0; ch < kPD / 32; ++ch) {
@@ -605,7 +616,8 @@ size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
 }
 
 int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, const void* v, const int32_t* kept_idx,
-                    const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream) {
+                    const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse,
+                    void* workspace, cudaStream_t stream) {
   CUtensorMap mq, mk, mv, mo;
   int rc;
   if ((rc = pipe_map(&mq, q, s)) != SPARKATTN_OK) return rc;
@@ -625,6 +637,7 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, co
   prm.lse = lse;
   prm.status = static_cast<int32_t*>(workspace);
   prm.H = s.H; prm.N = s.N; prm.nb = nb; prm.kmax = kmax; prm.items = (int)items;
+  prm.frame_tokens = frame_tokens; prm.window = window;
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
   const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
   prm.scale_log2 = sc * 1.4426950408889634f;

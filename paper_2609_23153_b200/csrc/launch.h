@@ -20,20 +20,23 @@ int launch_quant_fp8_per_token(const sparkattn_shape_t& s, const void* x, uint8_
 // select.cu
 constexpr int kSelectMaxBlocks = 4096;  // largest nb the selection kernel holds in shared memory
 size_t select_workspace_bytes(const sparkattn_shape_t& s);
-int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int32_t* kept_idx,
-                  int32_t* kept_cnt, void* workspace, cudaStream_t stream);
+// frame_tokens = 0: no causal window; otherwise window >= 1 frames of frame_tokens tokens
+int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int frame_tokens, int window,
+                  int32_t* kept_idx, int32_t* kept_cnt, void* workspace, cudaStream_t stream);
 
 // fwd.cu
 constexpr int kFwdMaxKept = 2048;  // longest kept list (kmax) the forward kernel stages in shared memory
 size_t fwd_workspace_bytes(const sparkattn_shape_t& s, int kmax);
 int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void* k, const void* v,
                const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
-               const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream);
+               const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse, void* workspace,
+               cudaStream_t stream);
 
 // fwd_pipe.cu: persistent pipelined forward for bf16, d = 128, block = 128
 size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax);
 int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, const void* v, const int32_t* kept_idx,
-                    const int32_t* kept_cnt, int kmax, void* out, float* lse, void* workspace, cudaStream_t stream);
+                    const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse,
+                    void* workspace, cudaStream_t stream);
 
 // comp.cu
 constexpr int kCompRank = 64;  // rank of the compensation branch the kernels are built for

@@ -103,12 +103,15 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 
 // Exact selection of the topk largest keys of one row by one warp (ties: lowest index first),
 // written in ascending index order.  KeyAt(j) returns key j; the keys are visited several times.
+// Only the key blocks jlo..jhi are candidates (the whole row without a causal window); the caller
+// passes topk <= jhi - jlo + 1 and key_at returns 0 (below every real key) outside that range.
 template <typename KeyAt>
-__device__ __forceinline__ void select_row(KeyAt key_at, int nb, int topk, int lane, int32_t* __restrict__ dst) {
+__device__ __forceinline__ void select_row(KeyAt key_at, int nb, int jlo, int jhi, int topk, int lane,
+                                           int32_t* __restrict__ dst) {
   // value of the topk-th largest key, one bit per pass from the top; bits above the highest bit in
   // which the row's keys differ are common to all keys and need no pass
   uint32_t kmin = 0xffffffffu, kmaxv = 0u;
-  for (int j = lane; j < nb; j += 32) {
+  for (int j = jlo + lane; j <= jhi; j += 32) {
     const uint32_t kj = key_at(j);
     kmin = min(kmin, kj);
     kmaxv = max(kmaxv, kj);
@@ -134,7 +137,7 @@ __device__ __forceinline__ void select_row(KeyAt key_at, int nb, int topk, int l
   const uint32_t lt_mask = (1u << lane) - 1u;
   for (int base = 0; base < nb; base += 32) {
     const int j = base + lane;
-    const bool valid = j < nb;
+    const bool valid = j >= jlo && j <= jhi;
     const uint32_t kj = valid ? key_at(j) : 0u;
     const bool tie = valid && (kj == thr);
     const uint32_t tie_ballot = __ballot_sync(0xffffffffu, tie);
@@ -152,7 +155,8 @@ constexpr int kKeysInRegs = 24;   // rows with nb <= 32 * 24 keep their keys in 
 template <int D>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
-            int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh) {
+            int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh, int N, int blk_size,
+            int frame_tokens, int window) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // pooled Q of the CTA's 8 query blocks, channel-major: s_pq[c][r], so that one 16-byte load
   // yields four rows of one channel as two packed fp32x2 operands
@@ -225,16 +229,31 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
   if (warp >= nrows) return;   // (warps beyond the 8 rows of the CTA have no row)
   const uint32_t* key = s_key + warp * nbp;
   int32_t* dst = kept_idx + (bh * nb + i0 + warp) * (int64_t)topk;
+  // Causal frame window (Sec. 1, auto-regressive extension): only the key blocks that hold a key some
+  // row of this query block may attend to are candidates, a contiguous run jlo..jhi.
+  int jlo = 0, jhi = nb - 1;
+  if (frame_tokens > 0) {
+    const int r0 = (i0 + warp) * blk_size, r1 = min((i0 + warp + 1) * blk_size, N) - 1;
+    const int f0 = max(r0 / frame_tokens - window + 1, 0);
+    const int kend = (int)min((long long)(r1 / frame_tokens + 1) * frame_tokens, (long long)N);
+    jlo = (int)((long long)f0 * frame_tokens / blk_size);
+    jhi = (kend - 1) / blk_size;
+  }
+  const int topk_all = topk;
+  topk = min(topk, jhi - jlo + 1);
   if (nb <= 32 * kKeysInRegs) {
     uint32_t kr[kKeysInRegs];
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u) kr[u] = (lane + 32 * u < nb) ? key[lane + 32 * u] : 0u;
+    for (int u = 0; u < kKeysInRegs; ++u) {
+      const int j = lane + 32 * u;
+      kr[u] = (j >= jlo && j <= jhi) ? key[j] : 0u;
+    }
     // same algorithm as select_row, with the key loops unrolled over registers; a padding key
     // of 0 is below every candidate (candidates are >= 1) and is excluded by index where needed
     uint32_t kmin = 0xffffffffu, kmaxv = 0u;
 #pragma unroll
     for (int u = 0; u < kKeysInRegs; ++u)
-      if (lane + 32 * u < nb) { kmin = min(kmin, kr[u]); kmaxv = max(kmaxv, kr[u]); }
+      if (lane + 32 * u >= jlo && lane + 32 * u <= jhi) { kmin = min(kmin, kr[u]); kmaxv = max(kmaxv, kr[u]); }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmaxv = __reduce_max_sync(0xffffffffu, kmaxv);
     const int top_bit = 31 - __clz(kmin ^ kmaxv);
@@ -250,7 +269,7 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
     }
     int ngreater = 0;
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u) ngreater += (lane + 32 * u < nb) && (kr[u] > thr);
+    for (int u = 0; u < kKeysInRegs; ++u) ngreater += (lane + 32 * u >= jlo) && (lane + 32 * u <= jhi) && (kr[u] > thr);
     ngreater = __reduce_add_sync(0xffffffffu, ngreater);
     const int ties_allowed = topk - ngreater;
     int out = 0, ties_seen = 0;
@@ -259,7 +278,7 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
     for (int u = 0; u < kKeysInRegs; ++u) {
       if (32 * u < nb) {
         const int j = lane + 32 * u;
-        const bool valid = j < nb;
+        const bool valid = j >= jlo && j <= jhi;
         const bool tie = valid && (kr[u] == thr);
         const uint32_t tie_ballot = __ballot_sync(0xffffffffu, tie);
         const int tie_rank = ties_seen + __popc(tie_ballot & lt_mask);
@@ -271,13 +290,14 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
       }
     }
   } else {
-    select_row([&](int j) { return key[j]; }, nb, topk, lane, dst);
+    select_row([&](int j) { return (j >= jlo && j <= jhi) ? key[j] : 0u; }, nb, jlo, jhi, topk, lane, dst);
   }
+  for (int t = topk + lane; t < topk_all; t += 32) dst[t] = -1;      // unused tail of a list cut short by the window
   if (lane == 0 && kept_cnt != nullptr) kept_cnt[bh * nb + i0 + warp] = topk;
 }
 
-int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int32_t* kept_idx,
-                  int32_t* kept_cnt, void* workspace, cudaStream_t stream) {
+int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int frame_tokens, int window,
+                  int32_t* kept_idx, int32_t* kept_cnt, void* workspace, cudaStream_t stream) {
   const int nb = (s.N + s.block - 1) / s.block;
   const int nbp = round_up(nb, 32);
   if (nb > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
@@ -301,7 +321,7 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
         cudaSuccess)
       return SPARKATTN_E_CUDA;
     topk_kernel<128><<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp,
-                                                                          topk, groups);
+                                                                          topk, groups, s.N, s.block, frame_tokens, window);
   } else if (s.d == 64) {
     pool_kernel<64><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
@@ -309,7 +329,7 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
         cudaSuccess)
       return SPARKATTN_E_CUDA;
     topk_kernel<64><<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp,
-                                                                         topk, groups);
+                                                                         topk, groups, s.N, s.block, frame_tokens, window);
   } else {
     return SPARKATTN_E_UNSUPPORTED_SHAPE;
   }
