@@ -83,7 +83,7 @@ struct FwdParams {
   float scale_log2;  // softmax_scale * log2(e)
 };
 
-template <int D, int BLK, bool FP8>
+template <int D, int BLK, bool FP8, bool WINDOW>
 __global__ void __launch_bounds__(kFwdThreads, 2)
 fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
            const __grid_constant__ CUtensorMap tmap_v, const FwdParams p) {
@@ -278,7 +278,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
     const bool row_valid = row < BLK && q_row < p.N;
     // keys this row may attend to: [klo, khi) (everything up to N without a causal window)
     int klo = 0, khi = p.N;
-    if (p.frame_tokens > 0) {
+    if constexpr (WINDOW) {
       const int fi = min(q_row, p.N - 1) / p.frame_tokens;
       klo = max(fi - p.window + 1, 0) * p.frame_tokens;
       khi = (int)min((long long)(fi + 1) * p.frame_tokens, (long long)p.N);
@@ -315,10 +315,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
         for (int ch = 0; ch < HALF / 32; ++ch)
           tmem_ld32(tmem_S + lane_off + hf * HALF + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[ch * 32]));
         tc_wait_ld();
-        if (c_lo > 0 || c_hi < HALF) {  // ragged last key block / keys outside the causal window get weight 0
+        if ((WINDOW && c_lo > 0) || c_hi < HALF) {  // ragged last key block / keys outside the causal window get weight 0
 #pragma unroll
           for (int i = 0; i < HALF; ++i)
-            if (i < c_lo || i >= c_hi) sr[i] = 0xff800000u;
+            if ((WINDOW && i < c_lo) || i >= c_hi) sr[i] = 0xff800000u;
         }
         float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
         float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
@@ -511,7 +511,7 @@ static int launch_fwd_t(const sparkattn_shape_t& s, const CUtensorMap& mq, const
   using Cfg = FwdCfg<D, BLK, FP8>;
   // at least 100 KB so that no more than two CTAs (2 x <=256 TMEM columns) share an SM
   const int smem = Cfg::kSmemBytes < 100 * 1024 ? 100 * 1024 : Cfg::kSmemBytes;
-  auto kern = fwd_kernel<D, BLK, FP8>;
+  auto kern = prm.frame_tokens > 0 ? fwd_kernel<D, BLK, FP8, true> : fwd_kernel<D, BLK, FP8, false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const long long ctas = (long long)s.B * s.H * prm.nb;

@@ -105,6 +105,7 @@ struct PipeIdle {
   }
 };
 
+template <bool WINDOW>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -361,7 +362,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       const bool row_valid = q_row < p.N;
       // keys this row may attend to: [klo, khi) (everything up to N without a causal window)
       int klo = 0, khi = p.N;
-      if (p.frame_tokens > 0) {
+      if constexpr (WINDOW) {
         const int fi = min(q_row, p.N - 1) / p.frame_tokens;
         klo = max(fi - p.window + 1, 0) * p.frame_tokens;
         khi = (int)min((long long)(fi + 1) * p.frame_tokens, (long long)p.N);
@@ -398,10 +399,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + buf);    // the S buffer can take the next-but-one tile
-        if (c_lo > 0 || c_hi < kPBLK) {   // ragged last key block / keys outside the causal window get weight 0
+        if ((WINDOW && c_lo > 0) || c_hi < kPBLK) {   // ragged last key block / keys outside the causal window get weight 0
 #pragma unroll
           for (int i = 0; i < kPBLK; ++i)
-            if (i < c_lo || i >= c_hi) sr[i] = 0xff800000u;
+            if ((WINDOW && i < c_lo) || i >= c_hi) sr[i] = 0xff800000u;
         }
         float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
         float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
@@ -651,10 +652,11 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, co
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
   compact_lists_kernel<<<(unsigned)((items + 7) / 8), 256, 0, stream>>>(kept_idx, kept_cnt, clean_cnt, clean_list, (int)items,
                                                                       nb, kmax, prm.status);
-  if (cudaFuncSetAttribute(fwd_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
+  auto kern = frame_tokens > 0 ? fwd_pipe_kernel<true> : fwd_pipe_kernel<false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
-  fwd_pipe_kernel<<<grid, kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, prm);
+  kern<<<grid, kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, prm);
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 

@@ -152,7 +152,7 @@ __device__ __forceinline__ void select_row(KeyAt key_at, int nb, int jlo, int jh
 
 constexpr int kKeysInRegs = 24;   // rows with nb <= 32 * 24 keep their keys in registers during the selection
 
-template <int D>
+template <int D, bool WINDOW>
 __global__ void __launch_bounds__(kTopkThreads)
 topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
             int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh, int N, int blk_size,
@@ -232,7 +232,7 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
   // Causal frame window (Sec. 1, auto-regressive extension): only the key blocks that hold a key some
   // row of this query block may attend to are candidates, a contiguous run jlo..jhi.
   int jlo = 0, jhi = nb - 1;
-  if (frame_tokens > 0) {
+  if constexpr (WINDOW) {
     const int r0 = (i0 + warp) * blk_size, r1 = min((i0 + warp + 1) * blk_size, N) - 1;
     const int f0 = max(r0 / frame_tokens - window + 1, 0);
     const int kend = (int)min((long long)(r1 / frame_tokens + 1) * frame_tokens, (long long)N);
@@ -241,19 +241,20 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
   }
   const int topk_all = topk;
   topk = min(topk, jhi - jlo + 1);
+  auto in_range = [&](int j) { return WINDOW ? (j >= jlo && j <= jhi) : (j < nb); };
   if (nb <= 32 * kKeysInRegs) {
     uint32_t kr[kKeysInRegs];
 #pragma unroll
     for (int u = 0; u < kKeysInRegs; ++u) {
       const int j = lane + 32 * u;
-      kr[u] = (j >= jlo && j <= jhi) ? key[j] : 0u;
+      kr[u] = in_range(j) ? key[j] : 0u;
     }
     // same algorithm as select_row, with the key loops unrolled over registers; a padding key
     // of 0 is below every candidate (candidates are >= 1) and is excluded by index where needed
     uint32_t kmin = 0xffffffffu, kmaxv = 0u;
 #pragma unroll
     for (int u = 0; u < kKeysInRegs; ++u)
-      if (lane + 32 * u >= jlo && lane + 32 * u <= jhi) { kmin = min(kmin, kr[u]); kmaxv = max(kmaxv, kr[u]); }
+      if (in_range(lane + 32 * u)) { kmin = min(kmin, kr[u]); kmaxv = max(kmaxv, kr[u]); }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmaxv = __reduce_max_sync(0xffffffffu, kmaxv);
     const int top_bit = 31 - __clz(kmin ^ kmaxv);
@@ -269,7 +270,7 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
     }
     int ngreater = 0;
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u) ngreater += (lane + 32 * u >= jlo) && (lane + 32 * u <= jhi) && (kr[u] > thr);
+    for (int u = 0; u < kKeysInRegs; ++u) ngreater += in_range(lane + 32 * u) && (kr[u] > thr);
     ngreater = __reduce_add_sync(0xffffffffu, ngreater);
     const int ties_allowed = topk - ngreater;
     int out = 0, ties_seen = 0;
@@ -278,7 +279,7 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
     for (int u = 0; u < kKeysInRegs; ++u) {
       if (32 * u < nb) {
         const int j = lane + 32 * u;
-        const bool valid = j >= jlo && j <= jhi;
+        const bool valid = in_range(j);
         const bool tie = valid && (kr[u] == thr);
         const uint32_t tie_ballot = __ballot_sync(0xffffffffu, tie);
         const int tie_rank = ties_seen + __popc(tie_ballot & lt_mask);
@@ -290,9 +291,10 @@ topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t
       }
     }
   } else {
-    select_row([&](int j) { return (j >= jlo && j <= jhi) ? key[j] : 0u; }, nb, jlo, jhi, topk, lane, dst);
+    select_row([&](int j) { return in_range(j) ? key[j] : 0u; }, nb, jlo, jhi, topk, lane, dst);
   }
-  for (int t = topk + lane; t < topk_all; t += 32) dst[t] = -1;      // unused tail of a list cut short by the window
+  if constexpr (WINDOW)
+    for (int t = topk + lane; t < topk_all; t += 32) dst[t] = -1;    // unused tail of a list cut short by the window
   if (lane == 0 && kept_cnt != nullptr) kept_cnt[bh * nb + i0 + warp] = topk;
 }
 
@@ -317,19 +319,19 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
   if (s.d == 128) {
     pool_kernel<128><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
-    if (cudaFuncSetAttribute(topk_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
+    auto kern = frame_tokens > 0 ? topk_kernel<128, true> : topk_kernel<128, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return SPARKATTN_E_CUDA;
-    topk_kernel<128><<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp,
-                                                                          topk, groups, s.N, s.block, frame_tokens, window);
+    kern<<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, groups, s.N,
+                                                             s.block, frame_tokens, window);
   } else if (s.d == 64) {
     pool_kernel<64><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
-    if (cudaFuncSetAttribute(topk_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
+    auto kern = frame_tokens > 0 ? topk_kernel<64, true> : topk_kernel<64, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return SPARKATTN_E_CUDA;
-    topk_kernel<64><<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp,
-                                                                         topk, groups, s.N, s.block, frame_tokens, window);
+    kern<<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, groups, s.N,
+                                                             s.block, frame_tokens, window);
   } else {
     return SPARKATTN_E_UNSUPPORTED_SHAPE;
   }
