@@ -337,7 +337,7 @@ def run_ours(args, w):
         ms_q = statistics.mean(a.elapsed_time(b) for a, b in evq)
         ms_f8 = statistics.mean(a.elapsed_time(b) for a, b in evf)
         qbytes = 3 * (elems * 3 + scales[0].numel() * 4)
-        fp8 = {"ms_per_step_quant_plus_fwd": ms8, "quant_ms_3_tensors": ms_q, "quant_GBps": qbytes / (ms_q * 1e-3) / 1e9,
+        fp8 = {"kernel": "fwd_pipe_kernel (FP8)" if pipelined else f"fwd_kernel<{w.d},{w.block},fp8>", "ms_per_step_quant_plus_fwd": ms8, "quant_ms_3_tensors": ms_q, "quant_GBps": qbytes / (ms_q * 1e-3) / 1e9,
                "quant_frac_of_hbm_peak": qbytes / (ms_q * 1e-3) / 1e9 / peaks["hbm"],
                "fwd_ms": ms_f8, "fwd_TFLOPs": flops / (ms_f8 * 1e-3) / 1e12,
                "fwd_frac_of_nominal_fp8_peak_4500": flops / (ms_f8 * 1e-3) / 1e12 / 4500.0,

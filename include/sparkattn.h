@@ -79,9 +79,9 @@ const char* sparkattn_status_string(int status);
 
 /* Bytes of device workspace a call needs.  which: 0 = sparkattn_select (pass
  * topk), 1 = sparkattn_fwd (pass kmax: for d = 128 with 128-token blocks the
- * forward keeps a range-checked copy of the kept lists behind the status words,
- * 4 * B * H * nb * (kmax + 1) bytes; 256 bytes otherwise).  Returns 0 for an
- * invalid shape or a non-positive topk / kmax. */
+ * forward keeps a range-checked copy of the kept lists and one scale per head
+ * behind the status words, about 4 * B * H * nb * (kmax + 1) bytes; 256 bytes
+ * otherwise).  Returns 0 for an invalid shape or a non-positive topk / kmax. */
 size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t topk_or_kmax);
 
 /*

@@ -526,8 +526,9 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
 #ifndef SPARKATTN_FWD_NO_PIPE
-  if (!fp8 && s.d == 128 && s.block == 128)
-    return launch_fwd_pipe(s, q, k, v, kept_idx, kept_cnt, kmax, frame_tokens, window, out, lse, workspace, stream);
+  if (s.d == 128 && s.block == 128)
+    return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window, out,
+                           lse, workspace, stream);
 #endif
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;

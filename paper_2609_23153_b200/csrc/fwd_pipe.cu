@@ -1,4 +1,4 @@
-// sparkattn_fwd, bf16, d = 128, 128-token blocks: persistent pipelined block-sparse forward.
+// sparkattn_fwd, d = 128, 128-token blocks (bf16 and FP8): persistent pipelined block-sparse forward.
 //
 // Same arithmetic as fwd.cu (Sec. 2 softmax attention restricted to the kept tiles, Sec. 4.1 sparse
 // branch); different schedule.  Measured on the one-item-per-CTA kernel: a tile's chain
@@ -29,6 +29,7 @@
 // compacted by a small pre-pass into the workspace; every role reads the clean lists from there.
 // Every wait is bounded; nothing here waits on another CTA.
 #include <cuda.h>
+#include <cuda_fp8.h>
 
 #include "common.cuh"
 #include "launch.h"
@@ -38,7 +39,10 @@ namespace sparkattn {
 constexpr int kPipeThreads = 384;
 constexpr int kPipeSoftmaxRegs = 216, kPipeCtrlRegs = 64;   // 2*128*216 + 128*64 <= 384*168
 constexpr int kPD = 128, kPBLK = 128;
-constexpr float kPipeLazyLog2 = 8.0f;
+constexpr float kPipeLazyLog2 = 8.0f;        // bf16: P may exceed 1 by up to 2^8 before O is rescaled
+// FP8: P is pre-scaled by 2^4 * (s_v[j] / max s_v) and may grow by another 2^4 before O is rescaled:
+// at most 2^8 = 256 < 448, the E4M3 maximum; values below 2^-13 of the row maximum flush to zero.
+constexpr float kPipeFp8LazyLog2 = 4.0f, kPipeFp8PScaleLog2 = 4.0f;
 constexpr int kTile = 32768;                               // bytes of one 128 x 128 bf16 tile (two 64-column slabs)
 constexpr int kOffQ = 0, kOffK = 2 * kTile, kOffV = 4 * kTile, kOffMisc = 7 * kTile;
 constexpr int kPipeSmem = kOffMisc + 256 /*barriers*/ + 2 * 128 * 4 /*reference maxima*/ + 128 * 8 /*row sums*/ + 64;
@@ -46,6 +50,10 @@ constexpr int kPipeSmem = kOffMisc + 256 /*barriers*/ + 2 * 128 * 4 /*reference 
 struct PipeParams {
   const int32_t* clean_cnt;    // [items] valid kept blocks per item
   const int32_t* clean_list;   // [items][kmax] their indices, compacted in list order
+  const float* q_scale;        // FP8: [B*H*nb] dequantisation scales of the token blocks
+  const float* k_scale;
+  const float* v_scale;
+  const float* v_max;          // FP8: [B*H] largest V scale of the head (pre-pass)
   __nv_bfloat16* out;
   float* lse;
   int32_t* status;
@@ -78,6 +86,18 @@ __global__ void compact_lists_kernel(const int32_t* __restrict__ kept_idx, const
   if (lane == 0) clean_cnt[item] = out;
 }
 
+// FP8: largest V block scale of every (batch, head); one warp each
+__global__ void head_vmax_kernel(const float* __restrict__ v_scale, float* __restrict__ v_max, int bh_count, int nb) {
+  const int bh = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (bh >= bh_count) return;
+  float m = 0.0f;
+  for (int j = lane; j < nb; j += 32) m = fmaxf(m, __ldg(v_scale + (int64_t)bh * nb + j));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) v_max[bh] = m;
+}
+
 __device__ __forceinline__ void pipe_tma_store_4d(const void* tmap, const void* smem_src, int c0, int c1, int c2, int c3) {
   asm volatile(
       "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
@@ -105,7 +125,7 @@ struct PipeIdle {
   }
 };
 
-template <bool WINDOW>
+template <bool FP8, bool WINDOW>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -135,6 +155,9 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // An input tile is 128 rows x 128 channels: two 64-channel slabs of 16 KB in bf16, one slab in FP8
+  // (the slots keep their 32 KB stride).
+  constexpr int kTileTx = FP8 ? kTile / 2 : kTile;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -224,9 +247,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if (qf) {
               if (kc.cnt > 0) {
                 const int qb = kc.item % p.nb, bh = kc.item / p.nb;
-                mbar_expect_tx(bar_q_full + qslot, kTile);
+                mbar_expect_tx(bar_q_full + qslot, kTileTx);
                 tma_load_4d(sQ + qslot * kTile, &tmap_q, bar_q_full + qslot, 0, qb * kPBLK, bh % p.H, bh / p.H);
-                tma_load_4d(sQ + qslot * kTile + kTile / 2, &tmap_q, bar_q_full + qslot, 64, qb * kPBLK, bh % p.H, bh / p.H);
+                if constexpr (!FP8)
+                  tma_load_4d(sQ + qslot * kTile + kTile / 2, &tmap_q, bar_q_full + qslot, 64, qb * kPBLK, bh % p.H, bh / p.H);
                 kc.open = true;
               } else {
                 mbar_arrive(bar_q_full + qslot);      // empty item: nothing to load, consumers still step through it
@@ -239,9 +263,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             progressed = true;
           } else if (kf) {
             const int bh = kc.item / p.nb;
-            mbar_expect_tx(bar_k_full + kslot, kTile);
+            mbar_expect_tx(bar_k_full + kslot, kTileTx);
             tma_load_4d(sK + kslot * kTile, &tmap_k, bar_k_full + kslot, 0, kc.kb * kPBLK, bh % p.H, bh / p.H);
-            tma_load_4d(sK + kslot * kTile + kTile / 2, &tmap_k, bar_k_full + kslot, 64, kc.kb * kPBLK, bh % p.H, bh / p.H);
+            if constexpr (!FP8)
+              tma_load_4d(sK + kslot * kTile + kTile / 2, &tmap_k, bar_k_full + kslot, 64, kc.kb * kPBLK, bh % p.H, bh / p.H);
             next_tile(kc);
             progressed = true;
           }
@@ -252,9 +277,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if (vc.ord < kc.ord) { next_item(vc); progressed = true; }
           } else if (vc.t < kc.t && vf) {
             const int bh = vc.item / p.nb;
-            mbar_expect_tx(bar_v_full + vslot, kTile);
+            mbar_expect_tx(bar_v_full + vslot, kTileTx);
             tma_load_4d(sV + vslot * kTile, &tmap_v, bar_v_full + vslot, 0, vc.kb * kPBLK, bh % p.H, bh / p.H);
-            tma_load_4d(sV + vslot * kTile + kTile / 2, &tmap_v, bar_v_full + vslot, 64, vc.kb * kPBLK, bh % p.H, bh / p.H);
+            if constexpr (!FP8)
+              tma_load_4d(sV + vslot * kTile + kTile / 2, &tmap_v, bar_v_full + vslot, 64, vc.kb * kPBLK, bh % p.H, bh / p.H);
             next_tile(vc);
             progressed = true;
           }
@@ -266,7 +292,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   } else if (warp == 1) {
     // -------------------------------------------------------------- S issuer: S = Q K^T of the next tile
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc(1u, 128, kPBLK, false);
+      constexpr uint32_t idesc_qk = make_idesc(FP8 ? 0u : 1u, 128, kPBLK, false);
       int si = 0, s_item = first_item, s_n = 0, s_cnt = -1, s_t = 0;
       bool ok = true;
       PipeIdle guard;
@@ -287,12 +313,13 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ + qslot * kTile), 16);
           const uint64_t dK = make_smem_desc_sw128(smem_u32(sK + kslot * kTile), 16);
           const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32), k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
+          // 32 bytes of the channel dimension per MMA: 16 bf16 (8 MMAs over two slabs) or 32 E4M3 (4 MMAs)
 #pragma unroll
-          for (int sl = 0; sl < 2; ++sl)
+          for (int sl = 0; sl < (FP8 ? 1 : 2); ++sl)
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-              mma_ss<false>(tmem + sbuf * kPBLK, make_desc(q_lo + ((sl * (kTile / 2) + kk * 32) >> 4), q_hi),
-                            make_desc(k_lo + ((sl * (kTile / 2) + kk * 32) >> 4), k_hi), idesc_qk, (sl | kk) != 0 ? 1u : 0u);
+              mma_ss<FP8>(tmem + sbuf * kPBLK, make_desc(q_lo + ((sl * (kTile / 2) + kk * 32) >> 4), q_hi),
+                          make_desc(k_lo + ((sl * (kTile / 2) + kk * 32) >> 4), k_hi), idesc_qk, (sl | kk) != 0 ? 1u : 0u);
           tc_commit(bar_s_full + sbuf);
           tc_commit(bar_k_free + kslot);
           ++s_n; ++s_t;
@@ -307,7 +334,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     // (its own warp on another scheduler: an issuing thread shares its scheduler with two softmax
     // warps that are almost always ready, and gets an issue slot only when they stall)
     if (lane == 0) {
-      constexpr uint32_t idesc_pv = make_idesc(1u, 128, kPD, true);
+      constexpr uint32_t idesc_pv = make_idesc(FP8 ? 0u : 1u, 128, kPD, true);
+      constexpr int kPvSteps = FP8 ? 4 : 8;          // 32 bytes of P per row per MMA: 16 bf16 or 32 E4M3 keys
       int p_item = first_item, p_n = 0, p_cnt = -1, p_t = 0, p_nonempty = 0;
       bool ok = true;
       PipeIdle guard;
@@ -329,9 +357,9 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + vslot * kTile), kTile / 2);
           const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts<false>(tmem_O, tmem_P + pbuf * 64 + kk * 8, make_desc(v_lo + ((kk * 16 * 128) >> 4), v_hi), idesc_pv,
-                          (p_n == 0 && kk == 0) ? 0u : 1u);
+          for (int kk = 0; kk < kPvSteps; ++kk)
+            mma_ts<FP8>(tmem_O, tmem_P + pbuf * 64 + kk * 8, make_desc(v_lo + ((kk * (128 / kPvSteps) * 128) >> 4), v_hi),
+                        idesc_pv, (p_n == 0 && kk == 0) ? 0u : 1u);
           tc_commit(bar_pv_done + pbuf);
           tc_commit(bar_v_free + vslot);
           ++p_n; ++p_t;
@@ -347,7 +375,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     const int g = (warp >> 2) - 1;                    // warpgroup: takes the tiles with (global tile counter & 1) == g
     const int row = threadIdx.x & 127;                // query row inside the block = TMEM lane
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    const float c = p.scale_log2;
+    constexpr float kLazy = FP8 ? kPipeFp8LazyLog2 : kPipeLazyLog2;
     float m_used = 0.0f, l = 0.0f;                    // reference maximum this warpgroup last used; its partial row sum
     int t = 0;                                        // global tile counter at the start of the item
     int nonempty = 0;                                 // non-empty items finished so far
@@ -383,11 +411,22 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         continue;
       }
       l = 0.0f;
+      float q_sc = 1.0f, v_max = 1.0f;
+      if constexpr (FP8) {
+        q_sc = __ldg(p.q_scale + item);
+        v_max = __ldg(p.v_max + bh);
+      }
       for (int n = 0; ok && n < cnt; ++n) {
         const int tt = t + n;
         if ((tt & 1) != g) continue;
         const int buf = g;                          // (tt & 1) == g: this warpgroup's S and P buffers
         const int kb = __ldg(p.clean_list + (int64_t)item * p.kmax + n);
+        float c = p.scale_log2;                      // logit -> log2 units
+        float p_off = 0.0f;                          // log2 of the factor folded into P
+        if constexpr (FP8) {
+          c *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb);
+          p_off = kPipeFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb) / v_max);
+        }
         const int c_lo = klo - kb * kPBLK, c_hi = khi - kb * kPBLK;   // this row's valid columns of the tile: [c_lo, c_hi)
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt >> 1) & 1, s_abort, p.status, 4));
         if (!ok) break;
@@ -431,7 +470,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           const float m_prev = s_mref[(g ^ 1) * 128 + row];
           if (m_prev == -INFINITY) {
             m_new = m_tile;             // nothing accumulated for this row yet (all keys so far masked): O row and l are 0
-          } else if (m_tile > m_prev + kPipeLazyLog2) {
+          } else if (m_tile > m_prev + kLazy) {
             m_new = m_tile;
             alpha = fast_exp2(m_prev - m_tile);
             need = true;
@@ -476,30 +515,47 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
         // P = exp2(S*c - m) as bf16 into this warpgroup's P buffer
         const uint32_t tP = tmem_P + buf * 64 + lane_off;
-        const float neg_m = m_used == -INFINITY ? 0.0f : -m_used;     // a fully masked row: exp2(-inf) = 0, not NaN
+        const float neg_m = m_used == -INFINITY ? 0.0f : p_off - m_used;     // a fully masked row: exp2(-inf) = 0, not NaN
         const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
         uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
+        constexpr int kWords = FP8 ? 8 : 16;        // 32-bit words of P per 32 S columns
 #pragma unroll
         for (int ch = 0; ch < kPBLK / 32; ++ch) {
-          uint32_t w[16];
+          uint32_t w[kWords];
+          float e[32];
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
             const float2 x = unpack_f32x2(
                 ffma2(pack_f32x2(__uint_as_float(sr[ch * 32 + i]), __uint_as_float(sr[ch * 32 + i + 1])), c2, nm2));
-            const float e0 = fast_exp2(x.x), e1 = fast_exp2(x.y);
-            if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e0, e1));
-            else lsum0 = fadd2(lsum0, pack_f32x2(e0, e1));
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e0, e1);
-            w[i >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+            e[i] = fast_exp2(x.x);
+            e[i + 1] = fast_exp2(x.y);
+            if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e[i], e[i + 1]));
+            else lsum0 = fadd2(lsum0, pack_f32x2(e[i], e[i + 1]));
+          }
+          if constexpr (FP8) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i], e[4 * i + 1]), __NV_SATFINITE, __NV_E4M3);
+              const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(e[4 * i + 2], e[4 * i + 3]), __NV_SATFINITE, __NV_E4M3);
+              w[i] = lo | (hi << 16);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(e[2 * i], e[2 * i + 1]);
+              w[i] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
           }
           if (ch == 0 && tt >= 2) {
             // this warpgroup's P buffer is free once PV of tile tt-2 is complete (normally long ago)
             ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + buf, ((tt >> 1) - 1) & 1, s_abort, p.status, 11));
           }
-          tmem_st16(tP + ch * 16, w);
+          if constexpr (FP8) tmem_st8(tP + ch * 8, w);
+          else tmem_st16(tP + ch * 16, w);
         }
         const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
-        l += ls.x + ls.y;
+        if constexpr (FP8) l += (ls.x + ls.y) * fast_exp2(-p_off);     // the row sum is kept without the folded factor
+        else l += ls.x + ls.y;
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p_full + buf);
@@ -532,7 +588,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (!ok) break;
         tc_fence_after();
         // normalised O row as bf16 into the item's Q slot (all S MMAs of the item are complete), 128-byte swizzle
-        const float inv = l > 0.0f ? 1.0f / l : 0.0f;     // no admissible key at all: zero row, lse = -inf
+        float inv = l > 0.0f ? 1.0f / l : 0.0f;           // no admissible key at all: zero row, lse = -inf
+        if constexpr (FP8) inv *= v_max * 0.0625f;        // undo the 2^4 / max s_v folded into P
         unsigned char* slot = sQ + qslot * kTile;
 #pragma unroll 1
         for (int ch = 0; ch < kPD / 32; ++ch) {
@@ -598,14 +655,15 @@ static PipeEncodeFn pipe_encode_fn() {
   return fn;
 }
 
-static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t& s) {
+// [B,H,N,d] tensor of 2-byte (bf16) or 1-byte (E4M3) elements; box = 128 rows of one 128-byte slab
+static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t& s, int elt = 2) {
   PipeEncodeFn enc = pipe_encode_fn();
   if (!enc) return SPARKATTN_E_NO_DEVICE;
   const cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.H, (cuuint64_t)s.B};
-  const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * 2, (cuuint64_t)s.stride_h * 2, (cuuint64_t)s.stride_b * 2};
-  const cuuint32_t box[4] = {64u, (cuuint32_t)kPBLK, 1u, 1u};
+  const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * elt, (cuuint64_t)s.stride_h * elt, (cuuint64_t)s.stride_b * elt};
+  const cuuint32_t box[4] = {(cuuint32_t)(128 / elt), (cuuint32_t)kPBLK, 1u, 1u};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+  const CUresult r = enc(map, elt == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
@@ -613,17 +671,21 @@ static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t&
 
 size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
   const size_t items = (size_t)s.B * s.H * ((s.N + s.block - 1) / s.block);
-  return kWorkspaceHeaderBytes + (items * 4 + 255) / 256 * 256 + items * (size_t)kmax * 4;
+  // header | valid counts | compacted lists | FP8: largest V scale per (batch, head)
+  return kWorkspaceHeaderBytes + (items * 4 + 255) / 256 * 256 + (items * (size_t)kmax * 4 + 255) / 256 * 256 +
+         (size_t)s.B * s.H * 4;
 }
 
-int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, const void* v, const int32_t* kept_idx,
+int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
+                    const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                     const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse,
                     void* workspace, cudaStream_t stream) {
   CUtensorMap mq, mk, mv, mo;
   int rc;
-  if ((rc = pipe_map(&mq, q, s)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mk, k, s)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mv, v, s)) != SPARKATTN_OK) return rc;
+  const int elt = fp8 ? 1 : 2;
+  if ((rc = pipe_map(&mq, q, s, elt)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mk, k, s, elt)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mv, v, s, elt)) != SPARKATTN_OK) return rc;
   if ((rc = pipe_map(&mo, out, s)) != SPARKATTN_OK) return rc;
   const int nb = (s.N + s.block - 1) / s.block;
   const long long items = (long long)s.B * s.H * nb;
@@ -631,9 +693,12 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, co
   char* base = static_cast<char*>(workspace);
   int32_t* clean_cnt = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes);
   int32_t* clean_list = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256);
+  float* v_max = reinterpret_cast<float*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256 +
+                                          ((size_t)items * kmax * 4 + 255) / 256 * 256);
   PipeParams prm;
   prm.clean_cnt = clean_cnt;
   prm.clean_list = clean_list;
+  prm.q_scale = q_scale; prm.k_scale = k_scale; prm.v_scale = v_scale; prm.v_max = v_max;
   prm.out = static_cast<__nv_bfloat16*>(out);
   prm.lse = lse;
   prm.status = static_cast<int32_t*>(workspace);
@@ -652,7 +717,9 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, co
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
   compact_lists_kernel<<<(unsigned)((items + 7) / 8), 256, 0, stream>>>(kept_idx, kept_cnt, clean_cnt, clean_list, (int)items,
                                                                       nb, kmax, prm.status);
-  auto kern = frame_tokens > 0 ? fwd_pipe_kernel<true> : fwd_pipe_kernel<false>;
+  if (fp8) head_vmax_kernel<<<(unsigned)((s.B * s.H + 7) / 8), 256, 0, stream>>>(v_scale, v_max, s.B * s.H, nb);
+  auto kern = fp8 ? (frame_tokens > 0 ? fwd_pipe_kernel<true, true> : fwd_pipe_kernel<true, false>)
+                  : (frame_tokens > 0 ? fwd_pipe_kernel<false, true> : fwd_pipe_kernel<false, false>);
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);

@@ -32,9 +32,10 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse, void* workspace,
                cudaStream_t stream);
 
-// fwd_pipe.cu: persistent pipelined forward for bf16, d = 128, block = 128
+// fwd_pipe.cu: persistent pipelined forward for d = 128, block = 128 (bf16 and FP8)
 size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax);
-int launch_fwd_pipe(const sparkattn_shape_t& s, const void* q, const void* k, const void* v, const int32_t* kept_idx,
+int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
+                    const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                     const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse,
                     void* workspace, cudaStream_t stream);
 
