@@ -501,7 +501,7 @@ static int make_tile_map(CUtensorMap* map, const void* base, int elt_bytes, cons
 
 size_t fwd_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
   // the pipelined kernel keeps range-checked, compacted copies of the kept lists behind the header
-  if (s.d == 128 && s.block == 128) return fwd_pipe_workspace_bytes(s, kmax);
+  if (fwd_pipe_supported(s)) return fwd_pipe_workspace_bytes(s, kmax);
   return kWorkspaceHeaderBytes;
 }
 
@@ -526,7 +526,7 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
 #ifndef SPARKATTN_FWD_NO_PIPE
-  if (s.d == 128 && s.block == 128)
+  if (fwd_pipe_supported(s))
     return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window, out,
                            lse, workspace, stream);
 #endif

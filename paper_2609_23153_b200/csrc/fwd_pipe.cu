@@ -1,4 +1,5 @@
-// sparkattn_fwd, d = 128, 128-token blocks (bf16 and FP8): persistent pipelined block-sparse forward.
+// sparkattn_fwd, d = 128 (128-token blocks, or 64-token blocks in pairs; bf16 and FP8): persistent pipelined
+// block-sparse forward.
 //
 // Same arithmetic as fwd.cu (Sec. 2 softmax attention restricted to the kept tiles, Sec. 4.1 sparse
 // branch); different schedule.  Measured on the one-item-per-CTA kernel: a tile's chain
@@ -57,7 +58,9 @@ struct PipeParams {
   __nv_bfloat16* out;
   float* lse;
   int32_t* status;
-  int H, N, nb, kmax, items;
+  int H, N, nb, items;
+  int nbq;                     // work items per (batch, head): query blocks, or pairs of 64-token query blocks
+  int lstride;                 // list entries per item in clean_list
   int frame_tokens, window;    // causal frame window (0 = none): key frame in (query frame - window, query frame]
   int64_t stride_b, stride_h, stride_n;
   float scale_log2;
@@ -84,6 +87,55 @@ __global__ void compact_lists_kernel(const int32_t* __restrict__ kept_idx, const
     out += __popc(ballot);
   }
   if (lane == 0) clean_cnt[item] = out;
+}
+
+// 64-token blocks: the kernel works on pairs of adjacent query blocks (128 query rows, the MMA's M) and on
+// tiles of two key blocks.  One warp per pair merges the two kept lists (range-checked, duplicates folded)
+// into one ascending list; an entry is block | in-list-of-first-query-block << 30 | in-list-of-second << 31,
+// two entries per tile (an odd tail repeats its block with both flags clear).  clean_cnt = tiles.
+constexpr int kPairMaxBlocks = 16384;    // key blocks per head the merge can mark in shared memory
+constexpr int kPairWarps = 4;
+__global__ void __launch_bounds__(kPairWarps * 32)
+pair_lists_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ kept_cnt,
+                  int32_t* __restrict__ clean_cnt, int32_t* __restrict__ clean_list, int pairs, int nb, int nbq,
+                  int kmax, int32_t* status) {
+  extern __shared__ uint32_t s_bits[];                      // [kPairWarps][2][words]
+  const int words = (nb + 31) / 32;
+  const int wl = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int pair = blockIdx.x * kPairWarps + wl;
+  if (pair >= pairs) return;
+  uint32_t* bits = s_bits + wl * 2 * words;
+  for (int i = lane; i < 2 * words; i += 32) bits[i] = 0u;
+  __syncwarp();
+  const int bh = pair / nbq, qp = pair % nbq;
+  for (int side = 0; side < 2; ++side) {
+    const int qb = 2 * qp + side;
+    if (qb >= nb) break;
+    const int64_t item = (int64_t)bh * nb + qb;
+    const int cnt = kept_cnt ? min(max(__ldg(kept_cnt + item), 0), kmax) : kmax;
+    const int32_t* src = kept_idx + item * kmax;
+    for (int t = lane; t < cnt; t += 32) {
+      const int kb = __ldg(src + t);
+      if (kb >= 0 && kb < nb) atomicOr(bits + side * words + (kb >> 5), 1u << (kb & 31));
+      else report_status(status, SPARKATTN_E_BAD_INDEX, kb);
+    }
+  }
+  __syncwarp();
+  int32_t* dst = clean_list + (int64_t)pair * (2 * kmax);
+  int out = 0;
+  for (int base = 0; base < nb; base += 32) {
+    const int kb = base + lane;
+    const uint32_t a = bits[base >> 5], bmask = bits[words + (base >> 5)];
+    const bool ina = (a >> lane) & 1u, inb = (bmask >> lane) & 1u;
+    const uint32_t u = a | bmask;
+    if (ina || inb) dst[out + __popc(u & ((1u << lane) - 1u))] = kb | (ina ? (1 << 30) : 0) | (inb ? (int)(1u << 31) : 0);
+    out += __popc(u);
+  }
+  __syncwarp();
+  if (lane == 0) {
+    if (out & 1) { dst[out] = dst[out - 1] & 0x3fffffff; }   // odd tail: second half of the last tile is nobody's
+    clean_cnt[pair] = (out + 1) >> 1;
+  }
 }
 
 // FP8: largest V block scale of every (batch, head); one warp each
@@ -125,7 +177,8 @@ struct PipeIdle {
   }
 };
 
-template <bool FP8, bool WINDOW>
+// PAIR: 64-token blocks; a work item is a pair of query blocks, a tile two key blocks (see pair_lists_kernel).
+template <bool FP8, bool WINDOW, bool PAIR>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -158,6 +211,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   // An input tile is 128 rows x 128 channels: two 64-channel slabs of 16 KB in bf16, one slab in FP8
   // (the slots keep their 32 KB stride).
   constexpr int kTileTx = FP8 ? kTile / 2 : kTile;
+  constexpr int kEnt = PAIR ? 2 : 1;              // list entries per tile
+  constexpr int kKeyBlk = PAIR ? 64 : 128;        // tokens per key block
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -207,28 +262,51 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (lane == 0) {
       struct Cursor {
         int ord, item, n, cnt, t;       // item ordinal, item, tile within the item, valid tiles, global tile counter
-        int kb, cnt_next, kb_next_item; // prefetched: this tile's block, next item's count and first block
+        int kb, kb2, cnt_next, kb_next_item, kb2_next_item; // prefetched: this tile's block(s), next item's count and first block(s)
         bool open;
       };
       auto prefetch_item = [&](Cursor& c) {
         const int nxt = c.item + item_step;
         c.cnt_next = nxt < p.items ? __ldg(p.clean_cnt + nxt) : 0;
-        c.kb_next_item = nxt < p.items ? __ldg(p.clean_list + (int64_t)nxt * p.kmax) : 0;
+        c.kb_next_item = nxt < p.items ? __ldg(p.clean_list + (int64_t)nxt * p.lstride) : 0;
+        c.kb2_next_item = (PAIR && nxt < p.items) ? __ldg(p.clean_list + (int64_t)nxt * p.lstride + 1) : 0;
       };
       auto init = [&](Cursor& c) {
         c.ord = 0; c.item = first_item; c.n = 0; c.t = 0; c.open = false;
         c.cnt = c.item < p.items ? __ldg(p.clean_cnt + c.item) : 0;
-        c.kb = c.item < p.items ? __ldg(p.clean_list + (int64_t)c.item * p.kmax) : 0;
+        c.kb = c.item < p.items ? __ldg(p.clean_list + (int64_t)c.item * p.lstride) : 0;
+        c.kb2 = (PAIR && c.item < p.items) ? __ldg(p.clean_list + (int64_t)c.item * p.lstride + 1) : 0;
         prefetch_item(c);
       };
       auto next_item = [&](Cursor& c) {
         c.item += item_step; ++c.ord; c.n = 0; c.open = false;
-        c.cnt = c.cnt_next; c.kb = c.kb_next_item;
+        c.cnt = c.cnt_next; c.kb = c.kb_next_item; c.kb2 = c.kb2_next_item;
         if (c.item < p.items) prefetch_item(c);
       };
       auto next_tile = [&](Cursor& c) {
         ++c.n; ++c.t;
-        if (c.n < c.cnt) c.kb = __ldg(p.clean_list + (int64_t)c.item * p.kmax + c.n);   // used one step later
+        if (c.n < c.cnt) {             // used one step later
+          c.kb = __ldg(p.clean_list + (int64_t)c.item * p.lstride + c.n * kEnt);
+          if constexpr (PAIR) c.kb2 = __ldg(p.clean_list + (int64_t)c.item * p.lstride + c.n * kEnt + 1);
+        }
+      };
+      // one K or V tile: 128 key rows of one block, or 64 + 64 rows of the tile's two 64-token blocks
+      auto load_kv = [&](unsigned char* slot, const CUtensorMap* map, uint64_t* bar, const Cursor& c) {
+        const int bh = c.item / p.nbq;
+        const int hh = bh % p.H, bb = bh / p.H;
+        mbar_expect_tx(bar, kTileTx);
+        if constexpr (PAIR) {
+          const int r0 = (c.kb & 0x3fffffff) * 64, r1 = (c.kb2 & 0x3fffffff) * 64;
+          tma_load_4d(slot, map, bar, 0, r0, hh, bb);
+          tma_load_4d(slot + 8192, map, bar, 0, r1, hh, bb);
+          if constexpr (!FP8) {
+            tma_load_4d(slot + kTile / 2, map, bar, 64, r0, hh, bb);
+            tma_load_4d(slot + kTile / 2 + 8192, map, bar, 64, r1, hh, bb);
+          }
+        } else {
+          tma_load_4d(slot, map, bar, 0, c.kb * kPBLK, hh, bb);
+          if constexpr (!FP8) tma_load_4d(slot + kTile / 2, map, bar, 64, c.kb * kPBLK, hh, bb);
+        }
       };
       Cursor kc, vc;
       init(kc);
@@ -246,7 +324,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           if (!kc.open) {
             if (qf) {
               if (kc.cnt > 0) {
-                const int qb = kc.item % p.nb, bh = kc.item / p.nb;
+                const int qb = kc.item % p.nbq, bh = kc.item / p.nbq;
                 mbar_expect_tx(bar_q_full + qslot, kTileTx);
                 tma_load_4d(sQ + qslot * kTile, &tmap_q, bar_q_full + qslot, 0, qb * kPBLK, bh % p.H, bh / p.H);
                 if constexpr (!FP8)
@@ -262,11 +340,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             next_item(kc);
             progressed = true;
           } else if (kf) {
-            const int bh = kc.item / p.nb;
-            mbar_expect_tx(bar_k_full + kslot, kTileTx);
-            tma_load_4d(sK + kslot * kTile, &tmap_k, bar_k_full + kslot, 0, kc.kb * kPBLK, bh % p.H, bh / p.H);
-            if constexpr (!FP8)
-              tma_load_4d(sK + kslot * kTile + kTile / 2, &tmap_k, bar_k_full + kslot, 64, kc.kb * kPBLK, bh % p.H, bh / p.H);
+            load_kv(sK + kslot * kTile, &tmap_k, bar_k_full + kslot, kc);
             next_tile(kc);
             progressed = true;
           }
@@ -276,11 +350,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             // the V cursor never passes the K cursor's item
             if (vc.ord < kc.ord) { next_item(vc); progressed = true; }
           } else if (vc.t < kc.t && vf) {
-            const int bh = vc.item / p.nb;
-            mbar_expect_tx(bar_v_full + vslot, kTileTx);
-            tma_load_4d(sV + vslot * kTile, &tmap_v, bar_v_full + vslot, 0, vc.kb * kPBLK, bh % p.H, bh / p.H);
-            if constexpr (!FP8)
-              tma_load_4d(sV + vslot * kTile + kTile / 2, &tmap_v, bar_v_full + vslot, 64, vc.kb * kPBLK, bh % p.H, bh / p.H);
+            load_kv(sV + vslot * kTile, &tmap_v, bar_v_full + vslot, vc);
             next_tile(vc);
             progressed = true;
           }
@@ -384,7 +454,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     for (int item = first_item; ok && item < p.items; item += item_step, ++io) {
       const int qslot = io & 1;
       const int cnt = __ldg(p.clean_cnt + item);
-      const int qb = item % p.nb, bh = item / p.nb;
+      const int qb = item % p.nbq, bh = item / p.nbq;     // PAIR: qb counts pairs of 64-token query blocks
       const int h = bh % p.H, b = bh / p.H;
       const int q_row = qb * kPBLK + row;
       const bool row_valid = q_row < p.N;
@@ -413,21 +483,41 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       l = 0.0f;
       float q_sc = 1.0f, v_max = 1.0f;
       if constexpr (FP8) {
-        q_sc = __ldg(p.q_scale + item);
+        q_sc = PAIR ? __ldg(p.q_scale + (int64_t)bh * p.nb + min(2 * qb + (row >> 6), p.nb - 1)) : __ldg(p.q_scale + item);
         v_max = __ldg(p.v_max + bh);
       }
       for (int n = 0; ok && n < cnt; ++n) {
         const int tt = t + n;
         if ((tt & 1) != g) continue;
         const int buf = g;                          // (tt & 1) == g: this warpgroup's S and P buffers
-        const int kb = __ldg(p.clean_list + (int64_t)item * p.kmax + n);
+        // the tile's key block(s); PAIR: two 64-token blocks, each with a flag per query block of the pair
+        int kb, kb1 = 0;
+        bool mem0 = true, mem1 = true;
+        if constexpr (PAIR) {
+          const int e0 = __ldg(p.clean_list + (int64_t)item * p.lstride + 2 * n);
+          const int e1 = __ldg(p.clean_list + (int64_t)item * p.lstride + 2 * n + 1);
+          kb = e0 & 0x3fffffff;
+          kb1 = e1 & 0x3fffffff;
+          mem0 = (((uint32_t)e0 >> (30 + (row >> 6))) & 1u) != 0u;
+          mem1 = (((uint32_t)e1 >> (30 + (row >> 6))) & 1u) != 0u;
+        } else {
+          kb = __ldg(p.clean_list + (int64_t)item * p.lstride + n);
+        }
         float c = p.scale_log2;                      // logit -> log2 units
         float p_off = 0.0f;                          // log2 of the factor folded into P
+        float c1 = c, p_off1 = 0.0f;                 // PAIR + FP8: the second key block of the tile has its own scales
         if constexpr (FP8) {
           c *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb);
           p_off = kPipeFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb) / v_max);
+          if constexpr (PAIR) {
+            c1 *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb1);
+            p_off1 = kPipeFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb1) / v_max);
+          }
         }
-        const int c_lo = klo - kb * kPBLK, c_hi = khi - kb * kPBLK;   // this row's valid columns of the tile: [c_lo, c_hi)
+        // this row's valid columns: [c_lo, c_hi) of the tile, or (PAIR) [c_lo, c_hi) of its first 64 and
+        // [c_lo1, c_hi1) of its second 64 columns (empty when the block is not in this query block's list)
+        const int c_lo = klo - kb * kKeyBlk, c_hi = PAIR ? (mem0 ? min(khi - kb * 64, 64) : 0) : khi - kb * kPBLK;
+        const int c_lo1 = klo - kb1 * 64, c_hi1 = mem1 ? min(khi - kb1 * 64, 64) : 0;
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt >> 1) & 1, s_abort, p.status, 4));
         if (!ok) break;
         tc_fence_after();
@@ -438,7 +528,15 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         tc_wait_ld();
         tc_fence_before();
         mbar_arrive(bar_s_free + buf);    // the S buffer can take the next-but-one tile
-        if ((WINDOW && c_lo > 0) || c_hi < kPBLK) {   // ragged last key block / keys outside the causal window get weight 0
+        if constexpr (PAIR) {
+          if ((WINDOW && (c_lo > 0 || c_lo1 > 0)) || c_hi < 64 || c_hi1 < 64) {
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+              if ((WINDOW && i < c_lo) || i >= c_hi) sr[i] = 0xff800000u;
+              if ((WINDOW && i < c_lo1) || i >= c_hi1) sr[64 + i] = 0xff800000u;
+            }
+          }
+        } else if ((WINDOW && c_lo > 0) || c_hi < kPBLK) {   // ragged last key block / keys outside the causal window get weight 0
 #pragma unroll
           for (int i = 0; i < kPBLK; ++i)
             if ((WINDOW && i < c_lo) || i >= c_hi) sr[i] = 0xff800000u;
@@ -454,7 +552,16 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mx3 = fmax3(mx3, __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
           }
         }
-        const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
+        float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;
+        if constexpr (PAIR && FP8) {      // two logit scales in one tile: maxima of the two halves separately
+          float ma = __uint_as_float(sr[0]), mb = __uint_as_float(sr[64]);
+#pragma unroll
+          for (int i = 1; i < 64; i += 2) {
+            ma = fmax3(ma, __uint_as_float(sr[i]), __uint_as_float(sr[(i + 1) & 63]));
+            mb = fmax3(mb, __uint_as_float(sr[64 + i]), __uint_as_float(sr[64 + ((i + 1) & 63)]));
+          }
+          m_tile = fmaxf(ma * c, mb * c1);
+        }
 
         // reference maximum: token from the warpgroup of tile tt-1 (also orders the reuse of s_mref[g])
         if (tt > 0) {
@@ -516,20 +623,24 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // P = exp2(S*c - m) as bf16 into this warpgroup's P buffer
         const uint32_t tP = tmem_P + buf * 64 + lane_off;
         const float neg_m = m_used == -INFINITY ? 0.0f : p_off - m_used;     // a fully masked row: exp2(-inf) = 0, not NaN
-        const uint64_t c2 = pack_f32x2(c, c), nm2 = pack_f32x2(neg_m, neg_m);
+        const float neg_m1 = m_used == -INFINITY ? 0.0f : p_off1 - m_used;
+        const uint64_t c2a = pack_f32x2(c, c), nm2a = pack_f32x2(neg_m, neg_m);
+        const uint64_t c2b = pack_f32x2(c1, c1), nm2b = pack_f32x2(neg_m1, neg_m1);
         uint64_t lsum0 = pack_f32x2(0.0f, 0.0f), lsum1 = lsum0;
         constexpr int kWords = FP8 ? 8 : 16;        // 32-bit words of P per 32 S columns
 #pragma unroll
         for (int ch = 0; ch < kPBLK / 32; ++ch) {
           uint32_t w[kWords];
           float e[32];
+          const bool second = PAIR && FP8 && ch >= 2;       // the tile's second key block: its own scales, its own sum
+          const uint64_t c2 = second ? c2b : c2a, nm2 = second ? nm2b : nm2a;
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
             const float2 x = unpack_f32x2(
                 ffma2(pack_f32x2(__uint_as_float(sr[ch * 32 + i]), __uint_as_float(sr[ch * 32 + i + 1])), c2, nm2));
             e[i] = fast_exp2(x.x);
             e[i + 1] = fast_exp2(x.y);
-            if ((i >> 1) & 1) lsum1 = fadd2(lsum1, pack_f32x2(e[i], e[i + 1]));
+            if ((PAIR && FP8) ? second : (((i >> 1) & 1) != 0)) lsum1 = fadd2(lsum1, pack_f32x2(e[i], e[i + 1]));
             else lsum0 = fadd2(lsum0, pack_f32x2(e[i], e[i + 1]));
           }
           if constexpr (FP8) {
@@ -553,9 +664,14 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           if constexpr (FP8) tmem_st8(tP + ch * 8, w);
           else tmem_st16(tP + ch * 16, w);
         }
-        const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
-        if constexpr (FP8) l += (ls.x + ls.y) * fast_exp2(-p_off);     // the row sum is kept without the folded factor
-        else l += ls.x + ls.y;
+        if constexpr (PAIR && FP8) {       // the row sum is kept without the factors folded into P, one per key block
+          const float2 la = unpack_f32x2(lsum0), lb = unpack_f32x2(lsum1);
+          l += (la.x + la.y) * fast_exp2(-p_off) + (lb.x + lb.y) * fast_exp2(-p_off1);
+        } else {
+          const float2 ls = unpack_f32x2(fadd2(lsum0, lsum1));
+          if constexpr (FP8) l += (ls.x + ls.y) * fast_exp2(-p_off);
+          else l += ls.x + ls.y;
+        }
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar_p_full + buf);
@@ -655,13 +771,13 @@ static PipeEncodeFn pipe_encode_fn() {
   return fn;
 }
 
-// [B,H,N,d] tensor of 2-byte (bf16) or 1-byte (E4M3) elements; box = 128 rows of one 128-byte slab
-static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t& s, int elt = 2) {
+// [B,H,N,d] tensor of 2-byte (bf16) or 1-byte (E4M3) elements; box = `rows` rows of one 128-byte slab
+static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t& s, int elt = 2, int rows = kPBLK) {
   PipeEncodeFn enc = pipe_encode_fn();
   if (!enc) return SPARKATTN_E_NO_DEVICE;
   const cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.H, (cuuint64_t)s.B};
   const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * elt, (cuuint64_t)s.stride_h * elt, (cuuint64_t)s.stride_b * elt};
-  const cuuint32_t box[4] = {(cuuint32_t)(128 / elt), (cuuint32_t)kPBLK, 1u, 1u};
+  const cuuint32_t box[4] = {(cuuint32_t)(128 / elt), (cuuint32_t)rows, 1u, 1u};
   const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
   const CUresult r = enc(map, elt == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -669,10 +785,26 @@ static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t&
   return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
+// items (query blocks, or pairs of 64-token query blocks) per (batch, head), and list entries per item
+static void pipe_geometry(const sparkattn_shape_t& s, int kmax, int* nbq, int* lstride) {
+  const int nb = (s.N + s.block - 1) / s.block;
+  const bool pair = s.block == 64;
+  *nbq = pair ? (nb + 1) / 2 : nb;
+  *lstride = pair ? 2 * kmax : kmax;
+}
+
+bool fwd_pipe_supported(const sparkattn_shape_t& s) {
+  if (s.d != 128) return false;
+  if (s.block == 128) return true;
+  return s.block == 64 && (s.N + 63) / 64 <= kPairMaxBlocks;
+}
+
 size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
-  const size_t items = (size_t)s.B * s.H * ((s.N + s.block - 1) / s.block);
-  // header | valid counts | compacted lists | FP8: largest V scale per (batch, head)
-  return kWorkspaceHeaderBytes + (items * 4 + 255) / 256 * 256 + (items * (size_t)kmax * 4 + 255) / 256 * 256 +
+  int nbq, lstride;
+  pipe_geometry(s, kmax, &nbq, &lstride);
+  const size_t items = (size_t)s.B * s.H * nbq;
+  // header | tiles per item | compacted (merged) lists | FP8: largest V scale per (batch, head)
+  return kWorkspaceHeaderBytes + (items * 4 + 255) / 256 * 256 + (items * (size_t)lstride * 4 + 255) / 256 * 256 +
          (size_t)s.B * s.H * 4;
 }
 
@@ -683,18 +815,21 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   CUtensorMap mq, mk, mv, mo;
   int rc;
   const int elt = fp8 ? 1 : 2;
+  const bool pair = s.block == 64;
   if ((rc = pipe_map(&mq, q, s, elt)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mk, k, s, elt)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mv, v, s, elt)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mk, k, s, elt, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
+  if ((rc = pipe_map(&mv, v, s, elt, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
   if ((rc = pipe_map(&mo, out, s)) != SPARKATTN_OK) return rc;
   const int nb = (s.N + s.block - 1) / s.block;
-  const long long items = (long long)s.B * s.H * nb;
+  int nbq, lstride;
+  pipe_geometry(s, kmax, &nbq, &lstride);
+  const long long items = (long long)s.B * s.H * nbq;
   if (items > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   char* base = static_cast<char*>(workspace);
   int32_t* clean_cnt = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes);
   int32_t* clean_list = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256);
   float* v_max = reinterpret_cast<float*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256 +
-                                          ((size_t)items * kmax * 4 + 255) / 256 * 256);
+                                          ((size_t)items * lstride * 4 + 255) / 256 * 256);
   PipeParams prm;
   prm.clean_cnt = clean_cnt;
   prm.clean_list = clean_list;
@@ -702,7 +837,7 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   prm.out = static_cast<__nv_bfloat16*>(out);
   prm.lse = lse;
   prm.status = static_cast<int32_t*>(workspace);
-  prm.H = s.H; prm.N = s.N; prm.nb = nb; prm.kmax = kmax; prm.items = (int)items;
+  prm.H = s.H; prm.N = s.N; prm.nb = nb; prm.items = (int)items; prm.nbq = nbq; prm.lstride = lstride;
   prm.frame_tokens = frame_tokens; prm.window = window;
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
   const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
@@ -715,11 +850,20 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
       return SPARKATTN_E_CUDA;
   }
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
-  compact_lists_kernel<<<(unsigned)((items + 7) / 8), 256, 0, stream>>>(kept_idx, kept_cnt, clean_cnt, clean_list, (int)items,
-                                                                      nb, kmax, prm.status);
+  if (pair) {
+    const size_t bits = (size_t)kPairWarps * 2 * ((nb + 31) / 32) * sizeof(uint32_t);
+    pair_lists_kernel<<<(unsigned)((items + kPairWarps - 1) / kPairWarps), kPairWarps * 32, bits, stream>>>(
+        kept_idx, kept_cnt, clean_cnt, clean_list, (int)items, nb, nbq, kmax, prm.status);
+  } else {
+    compact_lists_kernel<<<(unsigned)((items + 7) / 8), 256, 0, stream>>>(kept_idx, kept_cnt, clean_cnt, clean_list,
+                                                                        (int)items, nb, kmax, prm.status);
+  }
   if (fp8) head_vmax_kernel<<<(unsigned)((s.B * s.H + 7) / 8), 256, 0, stream>>>(v_scale, v_max, s.B * s.H, nb);
-  auto kern = fp8 ? (frame_tokens > 0 ? fwd_pipe_kernel<true, true> : fwd_pipe_kernel<true, false>)
-                  : (frame_tokens > 0 ? fwd_pipe_kernel<false, true> : fwd_pipe_kernel<false, false>);
+  const bool win = frame_tokens > 0;
+  auto kern = pair ? (fp8 ? (win ? fwd_pipe_kernel<true, true, true> : fwd_pipe_kernel<true, false, true>)
+                          : (win ? fwd_pipe_kernel<false, true, true> : fwd_pipe_kernel<false, false, true>))
+                   : (fp8 ? (win ? fwd_pipe_kernel<true, true, false> : fwd_pipe_kernel<true, false, false>)
+                          : (win ? fwd_pipe_kernel<false, true, false> : fwd_pipe_kernel<false, false, false>));
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);

@@ -33,6 +33,7 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                cudaStream_t stream);
 
 // fwd_pipe.cu: persistent pipelined forward for d = 128, block = 128 (bf16 and FP8)
+bool fwd_pipe_supported(const sparkattn_shape_t& s);   // d = 128 with 128-token blocks, or 64-token blocks (paired)
 size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax);
 int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
                     const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,

@@ -167,14 +167,16 @@ def test_small_structured_full_parity_fp8(w):
     _compare_items(out[0], lse[0], ref_out, ref_lse, items, w.block, w.N, FP8_RELRMS, None, lse_tol=2e-2)
 
 
-@pytest.mark.parametrize("seed,kmax", [(0, 3), (1, 6)])
-def test_persistent_path_short_and_empty_lists(seed, kmax):
-    """bf16, d = 128, 128-token blocks with more work items than SMs: every CTA of the persistent kernel
-    walks several items whose kept lists have 0, 1, 2, ... blocks (item boundaries, hand-over of the row
-    sums between the two softmax warpgroups, empty items), ragged last block included.  Compared in full
-    against the oracle, and two runs must agree bitwise."""
-    w = _small(41 + seed, 3, 128, (5, 18, 18), 128, 0.0)   # N = 1620: nb = 13 (ragged), 39 items per head
-    w = workloads.Workload(w.name, w.cfg_id, 1, 12, w.d, w.grid, w.block, w.sparsity)   # 156 items > 148 SMs
+@pytest.mark.parametrize("seed,kmax,block", [(0, 3, 128), (1, 6, 128), (2, 3, 64), (3, 7, 64)])
+def test_persistent_path_short_and_empty_lists(seed, kmax, block):
+    """bf16, d = 128 with more work items than SMs: every CTA of the persistent kernel walks several items
+    whose kept lists have 0, 1, 2, ... blocks (item boundaries, hand-over of the row sums between the two
+    softmax warpgroups, empty items), ragged last block included.  With 64-token blocks the items are
+    pairs of query blocks over the merged lists (one list empty, disjoint lists, odd merged length, an odd
+    number of query blocks).  Compared in full against the oracle, and two runs must agree bitwise."""
+    grid = (5, 18, 19) if seed == 3 else (5, 18, 18)        # N = 1620: 13 (ragged) or 26 blocks; N = 1710: 27 blocks of 64
+    w = _small(41 + seed, 3, 128, grid, block, 0.0)
+    w = workloads.Workload(w.name, w.cfg_id, 1, 12 if block == 128 else 13, w.d, w.grid, w.block, w.sparsity)   # > 148 items
     q, k, v = workloads.structured_qkv(w)
     g = torch.Generator().manual_seed(100 + seed)
     idx = torch.stack([torch.stack([torch.randperm(w.nb, generator=g)[:kmax] for _ in range(w.nb)]) for _ in range(w.H)]).to(torch.int32)
