@@ -95,7 +95,11 @@ def test_argument_errors_are_caught_on_the_host(lib):
     r = lib.sparkattn_fwd(ctypes.byref(s), sa.FP8_E4M3, fake, fake, fake, fake, fake, fake, fake, null, 4, fake,
                           null, fake, 256, st)
     assert r == sa.E_UNSUPPORTED_SHAPE            # FP8 needs d = 128
-    assert sa.workspace_bytes(_shape(d=128, block=64), 1, 4) == 256
+    assert sa.workspace_bytes(_shape(d=64, block=64), 1, 4) == 256
+    # d = 128 keeps checked copies of the kept lists behind the status words: per item, or per pair of 64-token blocks
+    assert sa.workspace_bytes(_shape(d=128, block=128), 1, 4) == 256 + 256 + 2 * 16 * 4 * 4 + 2 * 4
+    assert sa.workspace_bytes(_shape(d=128, block=64), 1, 4) == 256 + 256 + 2 * 16 * 8 * 4 + 2 * 4
+    assert sa.workspace_bytes(_shape(d=128, block=64), 1, 0) == 0
     assert sa.workspace_bytes(_shape(d=64, block=128), 1, 4) == 0
     r = lib.sparkattn_fwd(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 40, fake,
                           null, fake, 256, st)
@@ -106,6 +110,40 @@ def test_argument_errors_are_caught_on_the_host(lib):
     r = lib.sparkattn_fwd(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 4, fake,
                           null, fake, 8, st)
     assert r == sa.E_WORKSPACE_TOO_SMALL
+    # causal window: frame size and window length must be positive; selection with a window needs kept_cnt
+    r = lib.sparkattn_fwd_window(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 4, 0, 1, fake,
+                                 null, fake, 256, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_fwd_window(ctypes.byref(s), sa.BF16, fake, fake, fake, null, null, null, fake, null, 4, 64, 0, fake,
+                                 null, fake, 256, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_select_window(ctypes.byref(s), fake, fake, 4, 64, 1, fake, null, fake, 1 << 20, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_select_window(ctypes.byref(s), fake, fake, 4, 64, 1, fake, fake, fake, 16, st)
+    assert r == sa.E_WORKSPACE_TOO_SMALL
+    # compensation branch: d = 128 and rank 64 only; the grid must cover N; rotary tables checked
+    s128 = _shape(d=128, block=128)
+    grid = (ctypes.c_int32 * 3)(2, 32, 32)
+    axis = (ctypes.c_int32 * 32)(*([0] * 32))
+    freq = (ctypes.c_float * 32)(*([1.0] * 32))
+    r = lib.sparkattn_comp_state(ctypes.byref(s), fake, fake, fake, 64, grid, axis, freq, fake, fake, 1 << 30, st)
+    assert r == sa.E_UNSUPPORTED_SHAPE            # d = 64
+    r = lib.sparkattn_comp_state(ctypes.byref(s128), fake, fake, fake, 32, grid, axis, freq, fake, fake, 1 << 30, st)
+    assert r == sa.E_UNSUPPORTED_SHAPE            # rank 32
+    bad_grid = (ctypes.c_int32 * 3)(2, 32, 31)
+    r = lib.sparkattn_comp_state(ctypes.byref(s128), fake, fake, fake, 64, bad_grid, axis, freq, fake, fake, 1 << 30, st)
+    assert r == sa.E_INVALID_ARG
+    axis[5] = 3
+    r = lib.sparkattn_comp_state(ctypes.byref(s128), fake, fake, fake, 64, grid, axis, freq, fake, fake, 1 << 30, st)
+    assert r == sa.E_INVALID_ARG
+    axis[5] = 0
+    r = lib.sparkattn_comp_state(ctypes.byref(s128), fake, fake, fake, 64, grid, axis, freq, fake, fake, 256, st)
+    assert r == sa.E_WORKSPACE_TOO_SMALL
+    r = lib.sparkattn_comp_apply(ctypes.byref(s128), fake, fake, 64, grid, axis, freq, fake, fake, fake, fake,
+                                 ctypes.c_float(0.0), fake, 1 << 20, st)
+    assert r == sa.E_INVALID_ARG                  # eps must be positive
+    assert lib.sparkattn_comp_workspace_bytes(ctypes.byref(s128), bad_grid) == 0
+    assert lib.sparkattn_comp_workspace_bytes(ctypes.byref(s128), grid) > 256
 
 
 def test_binding_checks_layout():
