@@ -12,19 +12,19 @@
 //   pool_kernel    one warp per (tensor, batch, head, block); reads Q and K once
 //                  from HBM (the only HBM-heavy step: 2 bytes per element) and
 //                  writes pooled Q [BH][nb][d] and pooled K transposed [BH][d][nbp].
-//   topk_kernel    one CTA per 8 query blocks of one (batch, head): scores against
-//                  all key blocks (pooled K streamed from L2, coalesced along j,
-//                  packed fp32x2 FMAs over row pairs), then one warp per query
-//                  block does an exact radix select of the topk-th largest key
-//                  (keys in registers for nb <= 768) and an ordered ballot compaction.
+//   topk_kernel    one CTA per 16 (8 for very long sequences) query blocks of one
+//                  (batch, head): scores against all key blocks as a 16 x 4 register
+//                  tile per thread (pooled K streamed from L2 in 16-byte loads along j,
+//                  packed fp32x2 FMAs over row pairs), then one warp per query block
+//                  does an exact radix select of the topk-th largest key (keys in
+//                  registers for nb <= 1280) and an ordered ballot compaction.
 #include "common.cuh"
 #include "launch.h"
 
 namespace sparkattn {
 
 constexpr int kPoolThreads = 256;
-constexpr int kTopkThreads = 320;  // 2 x 320 key-block slots per sweep (591 blocks of the 720P shape fit one sweep)
-constexpr int kRowsPerCta = 8;     // query blocks per CTA; warps 0-7 select one row each
+constexpr int kTopkThreads = 160;  // 4 x 160 key-block slots per sweep (591 blocks of the 720P shape fit one sweep)
 
 static inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
@@ -150,152 +150,248 @@ __device__ __forceinline__ void select_row(KeyAt key_at, int nb, int jlo, int jh
   }
 }
 
-constexpr int kKeysInRegs = 24;   // rows with nb <= 32 * 24 keep their keys in registers during the selection
-
-template <int D, bool WINDOW>
-__global__ void __launch_bounds__(kTopkThreads)
-topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
-            int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh, int N, int blk_size,
-            int frame_tokens, int window) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  // pooled Q of the CTA's 8 query blocks, channel-major: s_pq[c][r], so that one 16-byte load
-  // yields four rows of one channel as two packed fp32x2 operands
-  float* s_pq = reinterpret_cast<float*>(smem_raw);                          // [D][kRowsPerCta]
-  uint32_t* s_key = reinterpret_cast<uint32_t*>(s_pq + kRowsPerCta * D);     // [kRowsPerCta][nbp]
-
-  const int64_t bh = blockIdx.x / groups_per_bh;
-  const int i0 = (blockIdx.x % groups_per_bh) * kRowsPerCta;
-  const int nrows = min(kRowsPerCta, nb - i0);
-
-  for (int e = threadIdx.x; e < kRowsPerCta * D; e += kTopkThreads) {
-    const int r = e / D, c = e % D;
-    s_pq[c * kRowsPerCta + r] = (r < nrows) ? pq[(bh * nb + i0 + r) * D + c] : 0.0f;
-  }
-  __syncthreads();
-
-  // scores: a thread owns kJT key blocks (j, j + kTopkThreads) and walks the channels in ascending
-  // order for the CTA's 8 query blocks at once.  fma.rn.f32x2 is a pair of IEEE fmaf, so every
-  // accumulator still sees exactly the chain a = fmaf(pq[i,c], pk[j,c], a), c ascending.
-  const float* kcol = pkT + bh * D * (int64_t)nbp;
-  const ulonglong2* s_pq2 = reinterpret_cast<const ulonglong2*>(s_pq);       // [D][kRowsPerCta / 4]
-  constexpr int kJT = 2;
-  constexpr int kPairs = kRowsPerCta / 2;
-  for (int j0 = threadIdx.x; j0 < nb; j0 += kTopkThreads * kJT) {
-    int jcl[kJT];
-#pragma unroll
-    for (int u = 0; u < kJT; ++u) jcl[u] = min(j0 + u * kTopkThreads, nb - 1);  // clamped: loads stay in range
-    uint64_t acc[kJT][kPairs];
-#pragma unroll
-    for (int u = 0; u < kJT; ++u)
-#pragma unroll
-      for (int r = 0; r < kPairs; ++r) acc[u][r] = pack_f32x2(0.0f, 0.0f);
-    constexpr int kCB = 16;  // channels per batch of loads (2 x 16 loads in flight per thread)
-#pragma unroll 1
-    for (int c0 = 0; c0 < D; c0 += kCB) {
-      float kv[kJT][kCB];
-#pragma unroll
-      for (int u = 0; u < kJT; ++u)
-#pragma unroll
-        for (int cc = 0; cc < kCB; ++cc) kv[u][cc] = __ldg(kcol + (int64_t)(c0 + cc) * nbp + jcl[u]);
-#pragma unroll
-      for (int cc = 0; cc < kCB; ++cc) {
-        const ulonglong2 qa = s_pq2[(c0 + cc) * 2], qb = s_pq2[(c0 + cc) * 2 + 1];   // rows (0,1),(2,3) | (4,5),(6,7)
-#pragma unroll
-        for (int u = 0; u < kJT; ++u) {
-          const uint64_t k2 = pack_f32x2(kv[u][cc], kv[u][cc]);
-          acc[u][0] = ffma2(qa.x, k2, acc[u][0]);
-          acc[u][1] = ffma2(qa.y, k2, acc[u][1]);
-          acc[u][2] = ffma2(qb.x, k2, acc[u][2]);
-          acc[u][3] = ffma2(qb.y, k2, acc[u][3]);
-        }
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kJT; ++u) {
-      const int j = j0 + u * kTopkThreads;
-      if (j < nb) {
-#pragma unroll
-        for (int r = 0; r < kPairs; ++r) {
-          const float2 a = unpack_f32x2(acc[u][r]);
-          s_key[(2 * r) * nbp + j] = score_key(a.x);
-          s_key[(2 * r + 1) * nbp + j] = score_key(a.y);
-        }
-      }
-    }
-  }
-  __syncthreads();
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp >= nrows) return;   // (warps beyond the 8 rows of the CTA have no row)
-  const uint32_t* key = s_key + warp * nbp;
-  int32_t* dst = kept_idx + (bh * nb + i0 + warp) * (int64_t)topk;
-  // Causal frame window (Sec. 1, auto-regressive extension): only the key blocks that hold a key some
-  // row of this query block may attend to are candidates, a contiguous run jlo..jhi.
-  int jlo = 0, jhi = nb - 1;
-  if constexpr (WINDOW) {
-    const int r0 = (i0 + warp) * blk_size, r1 = min((i0 + warp + 1) * blk_size, N) - 1;
-    const int f0 = max(r0 / frame_tokens - window + 1, 0);
-    const int kend = (int)min((long long)(r1 / frame_tokens + 1) * frame_tokens, (long long)N);
-    jlo = (int)((long long)f0 * frame_tokens / blk_size);
-    jhi = (kend - 1) / blk_size;
-  }
-  const int topk_all = topk;
-  topk = min(topk, jhi - jlo + 1);
+// select_row with the row's keys held in KR registers per lane (nb <= 32 * KR): the key loops unroll
+// over registers.  Keys outside the candidate range are held as 0, below every candidate (candidates
+// are >= 1).
+//
+// The threshold (the topk-th largest key) is first sought among the four largest keys of every lane,
+// 128 values: their topk-th largest, T, never exceeds the true threshold, and when no lane holds more
+// than four keys >= T every key >= T is among the 128, so T is the true threshold.  The bitwise search
+// then costs 4 compares per pass instead of KR.  Otherwise (a lane with five such keys, or topk > 128)
+// the search runs over all KR keys.  Either way the threshold is exact; only the cost differs.
+template <int KR, bool WINDOW>
+__device__ __forceinline__ void select_row_regs(const uint32_t* __restrict__ key, int nb, int jlo, int jhi, int topk,
+                                                int lane, int32_t* __restrict__ dst) {
+  constexpr uint32_t kFull = 0xffffffffu;
   auto in_range = [&](int j) { return WINDOW ? (j >= jlo && j <= jhi) : (j < nb); };
-  if (nb <= 32 * kKeysInRegs) {
-    uint32_t kr[kKeysInRegs];
+  uint32_t kr[KR];
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u) {
-      const int j = lane + 32 * u;
-      kr[u] = in_range(j) ? key[j] : 0u;
+  for (int u = 0; u < KR; ++u) {
+    const int j = lane + 32 * u;
+    kr[u] = in_range(j) ? key[j] : 0u;
+  }
+  // sorted four largest keys of the lane
+  uint32_t m1 = 0u, m2 = 0u, m3 = 0u, m4 = 0u;
+#pragma unroll
+  for (int u = 0; u < KR; ++u) {
+    uint32_t x = kr[u], t;
+    t = min(m1, x); m1 = max(m1, x); x = t;
+    t = min(m2, x); m2 = max(m2, x); x = t;
+    t = min(m3, x); m3 = max(m3, x); x = t;
+    m4 = max(m4, x);
+  }
+  const uint32_t kmaxv = __reduce_max_sync(kFull, m1);
+  uint32_t thr = 0u;
+  bool exact = false;
+  int nge = 0;
+  if (topk <= 128) {
+    // T lies between the smallest lane maximum (32 >= topk values are at least that) and the row maximum;
+    // the bits above the highest bit in which the two differ are common to both and need no pass
+    const uint32_t lo = (topk <= 32) ? __reduce_min_sync(kFull, m1) : 0u;
+    const int top_bit = 31 - __clz(lo ^ kmaxv);              // -1 when the two are equal
+    thr = (top_bit >= 31) ? 0u : (kmaxv & ~((2u << max(top_bit, 0)) - 1u));
+    if (top_bit < 0) thr = kmaxv;
+    for (int bit = top_bit; bit >= 0; --bit) {
+      const uint32_t cand = thr | (1u << bit);
+      int cnt = (m1 >= cand) + (m2 >= cand) + (m3 >= cand) + (m4 >= cand);
+      cnt = __reduce_add_sync(kFull, cnt);
+      if (cnt >= topk) thr = cand;
     }
-    // same algorithm as select_row, with the key loops unrolled over registers; a padding key
-    // of 0 is below every candidate (candidates are >= 1) and is excluded by index where needed
-    uint32_t kmin = 0xffffffffu, kmaxv = 0u;
+    int c = 0;
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u)
-      if (in_range(lane + 32 * u)) { kmin = min(kmin, kr[u]); kmaxv = max(kmaxv, kr[u]); }
-    kmin = __reduce_min_sync(0xffffffffu, kmin);
-    kmaxv = __reduce_max_sync(0xffffffffu, kmaxv);
+    for (int u = 0; u < KR; ++u) c += (kr[u] >= thr);
+    exact = thr != 0u && __ballot_sync(kFull, c > 4) == 0u;
+    nge = c;
+  }
+  if (!exact) {
+    // bitwise search over all keys, from the highest bit in which the row's candidates differ
+    uint32_t kmin = 0xffffffffu;
+#pragma unroll
+    for (int u = 0; u < KR; ++u)
+      if (in_range(lane + 32 * u)) kmin = min(kmin, kr[u]);
+    kmin = __reduce_min_sync(kFull, kmin);
     const int top_bit = 31 - __clz(kmin ^ kmaxv);
-    uint32_t thr = (top_bit >= 31) ? 0u : (kmaxv & ~((2u << max(top_bit, 0)) - 1u));
+    thr = (top_bit >= 31) ? 0u : (kmaxv & ~((2u << max(top_bit, 0)) - 1u));
     if (top_bit < 0) thr = kmaxv;
     for (int bit = top_bit; bit >= 0; --bit) {
       const uint32_t cand = thr | (1u << bit);
       int cnt = 0;
 #pragma unroll
-      for (int u = 0; u < kKeysInRegs; ++u) cnt += (kr[u] >= cand);
-      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      for (int u = 0; u < KR; ++u) cnt += (kr[u] >= cand);
+      cnt = __reduce_add_sync(kFull, cnt);
       if (cnt >= topk) thr = cand;
     }
-    int ngreater = 0;
+    nge = 0;
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u) ngreater += in_range(lane + 32 * u) && (kr[u] > thr);
-    ngreater = __reduce_add_sync(0xffffffffu, ngreater);
-    const int ties_allowed = topk - ngreater;
-    int out = 0, ties_seen = 0;
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int u = 0; u < KR; ++u) nge += (kr[u] >= thr);
+  }
+  // ordered compaction: keys above the threshold, then the lowest-indexed keys equal to it.  With thr >= 1
+  // the zero keys that stand for blocks outside the candidate range never pass a comparison (thr = 0 only
+  // when a candidate's own key is 0, the key of one NaN pattern: the general path below handles it).
+  nge = __reduce_add_sync(kFull, nge);
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  int out = 0;
+  if (nge == topk && thr != 0u) {   // no surplus of keys equal to the threshold: keep every key >= thr
 #pragma unroll
-    for (int u = 0; u < kKeysInRegs; ++u) {
-      if (32 * u < nb) {
-        const int j = lane + 32 * u;
-        const bool valid = in_range(j);
-        const bool tie = valid && (kr[u] == thr);
-        const uint32_t tie_ballot = __ballot_sync(0xffffffffu, tie);
-        const int tie_rank = ties_seen + __popc(tie_ballot & lt_mask);
-        const bool keep = valid && ((kr[u] > thr) || (tie && tie_rank < ties_allowed));
-        const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
-        if (keep) dst[out + __popc(keep_ballot & lt_mask)] = j;
+    for (int u = 0; u < KR; ++u) {
+      const uint32_t keep_ballot = __ballot_sync(kFull, kr[u] >= thr);
+      if (keep_ballot != 0u) {
+        if (kr[u] >= thr) dst[out + __popc(keep_ballot & lt_mask)] = lane + 32 * u;
         out += __popc(keep_ballot);
-        ties_seen += __popc(tie_ballot);
       }
     }
-  } else {
-    select_row([&](int j) { return in_range(j) ? key[j] : 0u; }, nb, jlo, jhi, topk, lane, dst);
+    return;
   }
-  if constexpr (WINDOW)
-    for (int t = topk + lane; t < topk_all; t += 32) dst[t] = -1;    // unused tail of a list cut short by the window
-  if (lane == 0 && kept_cnt != nullptr) kept_cnt[bh * nb + i0 + warp] = topk;
+  int ngreater = 0;
+#pragma unroll
+  for (int u = 0; u < KR; ++u) ngreater += (kr[u] > thr);
+  ngreater = __reduce_add_sync(kFull, ngreater);
+  const int ties_allowed = topk - ngreater;  // >= 1: lowest indices among the keys equal to thr
+  int ties_seen = 0;
+#pragma unroll
+  for (int u = 0; u < KR; ++u) {
+    if (32 * u < nb) {
+      const int j = lane + 32 * u;
+      const bool valid = in_range(j);
+      const bool tie = valid && (kr[u] == thr);
+      const uint32_t tie_ballot = __ballot_sync(kFull, tie);
+      const int tie_rank = ties_seen + __popc(tie_ballot & lt_mask);
+      const bool keep = valid && ((kr[u] > thr) || (tie && tie_rank < ties_allowed));
+      const uint32_t keep_ballot = __ballot_sync(kFull, keep);
+      if (keep) dst[out + __popc(keep_ballot & lt_mask)] = j;
+      out += __popc(keep_ballot);
+      ties_seen += __popc(tie_ballot);
+    }
+  }
+}
+
+template <int D, int ROWS, bool WINDOW>
+__global__ void __launch_bounds__(kTopkThreads, ROWS == 16 ? 3 : 4)
+topk_kernel(const float* __restrict__ pq, const float* __restrict__ pkT, int32_t* __restrict__ kept_idx,
+            int32_t* __restrict__ kept_cnt, int nb, int nbp, int topk, int groups_per_bh, int N, int blk_size,
+            int frame_tokens, int window) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  // pooled Q of the CTA's ROWS query blocks, channel-major: s_pq[c][r], so that one 16-byte load
+  // yields four rows of one channel as two packed fp32x2 operands
+  float* s_pq = reinterpret_cast<float*>(smem_raw);                   // [D][ROWS]
+  uint32_t* s_key = reinterpret_cast<uint32_t*>(s_pq + ROWS * D);     // [ROWS][nbp]
+
+  const int64_t bh = blockIdx.x / groups_per_bh;
+  const int i0 = (blockIdx.x % groups_per_bh) * ROWS;
+  const int nrows = min(ROWS, nb - i0);
+
+  for (int e = threadIdx.x; e < ROWS * D; e += kTopkThreads) {
+    const int r = e / D, c = e % D;
+    s_pq[c * ROWS + r] = (r < nrows) ? pq[(bh * nb + i0 + r) * D + c] : 0.0f;
+  }
+  __syncthreads();
+
+  // scores: a thread owns 4 adjacent key blocks (one 16-byte load per channel) and walks the channels
+  // in ascending order for the CTA's ROWS query blocks at once: a ROWS x 4 register tile.
+  // fma.rn.f32x2 is a pair of IEEE fmaf over two rows, so every accumulator still sees exactly the
+  // chain a = fmaf(pq[i,c], pk[j,c], a), c ascending.  Columns nb..nbp-1 of pooled K are padding
+  // whose scores are stored but never read.
+  const float* kcol = pkT + bh * D * (int64_t)nbp;
+  const ulonglong2* s_pq2 = reinterpret_cast<const ulonglong2*>(s_pq);       // [D][ROWS / 4]
+  constexpr int kPairs = ROWS / 2;
+  constexpr int kCB = 4;   // channels per batch of loads; two batches (2 x 4 x 16 bytes) in flight per thread
+  for (int j0 = threadIdx.x * 4; j0 < nb; j0 += kTopkThreads * 4) {
+    uint64_t acc[4][kPairs];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int r = 0; r < kPairs; ++r) acc[u][r] = pack_f32x2(0.0f, 0.0f);
+    const float* kp = kcol + j0;
+    auto load_batch = [&](float4 (&kv)[kCB], int c0) {
+#pragma unroll
+      for (int cc = 0; cc < kCB; ++cc) kv[cc] = __ldg(reinterpret_cast<const float4*>(kp + (int64_t)(c0 + cc) * nbp));
+    };
+    auto fma_batch = [&](const float4 (&kv)[kCB], int c0) {
+#pragma unroll
+      for (int cc = 0; cc < kCB; ++cc) {
+        uint64_t q2[kPairs];
+#pragma unroll
+        for (int g = 0; g < ROWS / 4; ++g) {
+          const ulonglong2 t = s_pq2[(c0 + cc) * (ROWS / 4) + g];   // rows (4g, 4g+1), (4g+2, 4g+3)
+          q2[2 * g] = t.x;
+          q2[2 * g + 1] = t.y;
+        }
+        const uint64_t k2[4] = {pack_f32x2(kv[cc].x, kv[cc].x), pack_f32x2(kv[cc].y, kv[cc].y),
+                                pack_f32x2(kv[cc].z, kv[cc].z), pack_f32x2(kv[cc].w, kv[cc].w)};
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int r = 0; r < kPairs; ++r) acc[u][r] = ffma2(q2[r], k2[u], acc[u][r]);
+      }
+    };
+    float4 kva[kCB], kvb[kCB];
+    load_batch(kva, 0);
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 2 * kCB) {
+      load_batch(kvb, c0 + kCB);
+      fma_batch(kva, c0);
+      if (c0 + 2 * kCB < D) load_batch(kva, c0 + 2 * kCB);
+      fma_batch(kvb, c0 + kCB);
+    }
+#pragma unroll
+    for (int r = 0; r < kPairs; ++r) {
+      uint4 lo, hi;
+      float2 a;
+      a = unpack_f32x2(acc[0][r]); lo.x = score_key(a.x); hi.x = score_key(a.y);
+      a = unpack_f32x2(acc[1][r]); lo.y = score_key(a.x); hi.y = score_key(a.y);
+      a = unpack_f32x2(acc[2][r]); lo.z = score_key(a.x); hi.z = score_key(a.y);
+      a = unpack_f32x2(acc[3][r]); lo.w = score_key(a.x); hi.w = score_key(a.y);
+      *reinterpret_cast<uint4*>(s_key + (2 * r) * nbp + j0) = lo;
+      *reinterpret_cast<uint4*>(s_key + (2 * r + 1) * nbp + j0) = hi;
+    }
+  }
+  __syncthreads();
+
+  // selection: the CTA's warps take the rows round-robin, one warp per row
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int row = warp; row < nrows; row += kTopkThreads / 32) {
+    const uint32_t* key = s_key + row * nbp;
+    int32_t* dst = kept_idx + (bh * nb + i0 + row) * (int64_t)topk;
+    // Causal frame window (Sec. 1, auto-regressive extension): only the key blocks that hold a key some
+    // row of this query block may attend to are candidates, a contiguous run jlo..jhi.
+    int jlo = 0, jhi = nb - 1;
+    if constexpr (WINDOW) {
+      const int r0 = (i0 + row) * blk_size, r1 = min((i0 + row + 1) * blk_size, N) - 1;
+      const int f0 = max(r0 / frame_tokens - window + 1, 0);
+      const int kend = (int)min((long long)(r1 / frame_tokens + 1) * frame_tokens, (long long)N);
+      jlo = (int)((long long)f0 * frame_tokens / blk_size);
+      jhi = (kend - 1) / blk_size;
+    }
+    const int k_row = min(topk, jhi - jlo + 1);
+    if (nb <= 32 * 8) {
+      select_row_regs<8, WINDOW>(key, nb, jlo, jhi, k_row, lane, dst);
+    } else if (nb <= 32 * 20) {
+      select_row_regs<20, WINDOW>(key, nb, jlo, jhi, k_row, lane, dst);
+    } else if (nb <= 32 * 40) {
+      select_row_regs<40, WINDOW>(key, nb, jlo, jhi, k_row, lane, dst);
+    } else {
+      select_row([&](int j) { return (WINDOW ? (j >= jlo && j <= jhi) : (j < nb)) ? key[j] : 0u; }, nb, jlo, jhi, k_row,
+                 lane, dst);
+    }
+    if constexpr (WINDOW)
+      for (int t = k_row + lane; t < topk; t += 32) dst[t] = -1;    // unused tail of a list cut short by the window
+    if (lane == 0 && kept_cnt != nullptr) kept_cnt[bh * nb + i0 + row] = k_row;
+  }
+}
+
+template <int D, int ROWS>
+static int launch_topk(const float* pq, const float* pkT, int32_t* kept_idx, int32_t* kept_cnt, int nb, int nbp, int topk,
+                       int64_t bh, int N, int block, int frame_tokens, int window, cudaStream_t stream) {
+  const int groups = (nb + ROWS - 1) / ROWS;
+  const int64_t ctas = bh * groups;
+  if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  const size_t smem = (size_t)ROWS * D * sizeof(float) + (size_t)ROWS * nbp * sizeof(uint32_t);
+  auto kern = frame_tokens > 0 ? topk_kernel<D, ROWS, true> : topk_kernel<D, ROWS, false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return SPARKATTN_E_CUDA;
+  kern<<<(unsigned)ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, groups, N, block,
+                                                       frame_tokens, window);
+  return SPARKATTN_OK;
 }
 
 int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int frame_tokens, int window,
@@ -311,30 +407,24 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
 
   const int64_t pool_ctas = (2 * n_items + kPoolThreads / 32 - 1) / (kPoolThreads / 32);
-  const int groups = (nb + kRowsPerCta - 1) / kRowsPerCta;
-  const int64_t topk_ctas = bh * groups;
-  if (pool_ctas > 0x7fffffffLL || topk_ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
-  const size_t smem = (size_t)kRowsPerCta * s.d * sizeof(float) + (size_t)kRowsPerCta * nbp * sizeof(uint32_t);
-
+  if (pool_ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  // 16 query blocks per CTA while two CTAs' score rows fit one SM's shared memory, else 8
+  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u;
+  int rc;
   if (s.d == 128) {
     pool_kernel<128><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
-    auto kern = frame_tokens > 0 ? topk_kernel<128, true> : topk_kernel<128, false>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SPARKATTN_E_CUDA;
-    kern<<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, groups, s.N,
-                                                             s.block, frame_tokens, window);
+    rc = rows16 ? launch_topk<128, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
+                : launch_topk<128, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
   } else if (s.d == 64) {
     pool_kernel<64><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
-    auto kern = frame_tokens > 0 ? topk_kernel<64, true> : topk_kernel<64, false>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return SPARKATTN_E_CUDA;
-    kern<<<(unsigned)topk_ctas, kTopkThreads, smem, stream>>>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, groups, s.N,
-                                                             s.block, frame_tokens, window);
+    rc = rows16 ? launch_topk<64, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
+                : launch_topk<64, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
   } else {
     return SPARKATTN_E_UNSUPPORTED_SHAPE;
   }
+  if (rc != SPARKATTN_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
