@@ -408,8 +408,9 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
 
   const int64_t pool_ctas = (2 * n_items + kPoolThreads / 32 - 1) / (kPoolThreads / 32);
   if (pool_ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
-  // 16 query blocks per CTA while two CTAs' score rows fit one SM's shared memory, else 8
-  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u;
+  // 16 query blocks per CTA while two CTAs' score rows fit one SM's shared memory and the grid still
+  // fills the device several times over (small problems are bound by the latency of one CTA), else 8
+  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u && bh * ((nb + 15) / 16) >= 6 * 148;
   int rc;
   if (s.d == 128) {
     pool_kernel<128><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(

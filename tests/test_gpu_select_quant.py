@@ -50,6 +50,54 @@ def test_select_tiny_workload_and_ties():
     assert torch.equal(idx[0].cpu(), ref_idx)
 
 
+def _crafted_qk(nb, block, d, pattern, tail=0):
+    """Q/K whose pooled block scores are known exactly: channel 0 of key block j holds v_j on all its tokens,
+    channel 0 of query block i holds a_i, every other channel is 0, so score(i, j) = a_i * v_j without rounding."""
+    N = nb * block - tail
+    j = torch.arange(nb)
+    if pattern == "one_lane":          # the largest keys all sit in one lane (j % 32 == 5) of the selecting warp
+        v = torch.where(j % 32 == 5, 64.0 + (j // 32).float(), ((j * 37) % 97).float() / 128.0)
+    elif pattern == "ties":            # two values only: most of the kept keys are ties at the threshold
+        v = (j % 3 == 0).float()
+    elif pattern == "few_then_ties":   # three clear winners, then a long run of equal keys
+        v = torch.where(j % 101 == 7, 5.0 + (j // 101).float(), torch.where((j % 4) != 1, 2.0, 0.25))
+    else:
+        raise ValueError(pattern)
+    a = torch.tensor([1.0, -1.0, 0.5, -0.75, 2.0])[torch.arange(nb) % 5]      # sign flips reverse the order
+    q = torch.zeros((1, 2, N, d), dtype=torch.bfloat16)
+    k = torch.zeros((1, 2, N, d), dtype=torch.bfloat16)
+    tok_blk = torch.arange(N) // block
+    q[0, :, :, 0] = a[tok_blk].to(torch.bfloat16)
+    k[0, 0, :, 0] = v[tok_blk].to(torch.bfloat16)
+    k[0, 1, :, 0] = v.flip(0)[tok_blk].to(torch.bfloat16)
+    return q, k
+
+
+@pytest.mark.parametrize("nb,topk", [(100, 7), (300, 8), (300, 40), (1000, 30), (1000, 140), (1400, 12)])
+@pytest.mark.parametrize("pattern", ["one_lane", "ties", "few_then_ties"])
+def test_select_crafted_scores(nb, topk, pattern):
+    """Score layouts aimed at the branches of the selection: many of the largest keys in one lane of the warp
+    (the search over per-lane maxima must give way to the full search), long runs of ties at the threshold,
+    every register-resident key count (nb <= 256, 640, 1280) and the shared-memory path above."""
+    block, d = 64, 128
+    q, k = _crafted_qk(nb, block, d, pattern, tail=13)
+    ref_idx, ref_cnt = oracle.select(q[0], k[0], block, topk)
+    idx, cnt = sa.select(q.to(DEV), k.to(DEV), block, topk)
+    assert torch.equal(idx[0].cpu(), ref_idx)
+    assert torch.equal(cnt[0].cpu(), ref_cnt)
+
+
+@pytest.mark.parametrize("pattern", ["one_lane", "ties"])
+def test_select_crafted_scores_with_window(pattern):
+    nb, block, d, topk = 300, 64, 128, 9
+    q, k = _crafted_qk(nb, block, d, pattern, tail=13)
+    F, window = 1000, 6                       # frames of 1000 tokens straddle the 64-token blocks
+    ref_idx, ref_cnt = oracle.select(q[0], k[0], block, topk, frame_tokens=F, window=window)
+    idx, cnt = sa.select(q.to(DEV), k.to(DEV), block, topk, frame_tokens=F, window=window)
+    assert torch.equal(idx[0].cpu(), ref_idx)
+    assert torch.equal(cnt[0].cpu(), ref_cnt)
+
+
 def test_select_strided_layout_and_batch():
     # [B, N, H, d] storage viewed as [B, H, N, d]; two batches
     w = workloads.small_structured(H=2, d=128, grid=(2, 10, 26), block=128, sparsity=0.75, cfg_id=16)
