@@ -191,6 +191,16 @@ int sparkattn_read_status(void* workspace, void* cuda_stream);
  * pinned) host memory; kept_idx_host may be NULL or int32 [B,H,nb,topk] to
  * receive the selected lists.  arena: device scratch of at least
  * sparkattn_arena_bytes(shape, dtype, topk) bytes, 256-byte aligned.
+ * The heads are independent, so the call runs as a pipeline over groups of
+ * heads (about eight groups, at most 16): while one group is selected and
+ * attended on `cuda_stream`, the next is copied in and the previous one's
+ * output copied out on two copy streams that the library creates once per
+ * device and keeps; both are ordered after work already queued on
+ * `cuda_stream`, and `cuda_stream` ends after the last copy.  With pageable
+ * host memory the copies are staged by the driver and the overlap is lost;
+ * the result is the same.  Returns the first non-zero device status of any
+ * group (SPARKATTN_E_BAD_INDEX, SPARKATTN_E_DEVICE_TIMEOUT), an argument or
+ * CUDA error, or SPARKATTN_OK; on an error the output is undefined.
  */
 size_t sparkattn_arena_bytes(const sparkattn_shape_t* shape, int32_t dtype, int32_t topk);
 int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, const void* q_host,

@@ -4,6 +4,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "launch.h"
 
@@ -226,11 +228,11 @@ int sparkattn_read_status(void* workspace, void* cuda_stream) {
 }
 
 // Arena layout of the host-buffer path (every region 256-byte aligned):
-//   q, k, v, out (bf16) | kept_idx | kept_cnt | select workspace | fwd workspace |
+//   q, k, v, out (bf16) | kept_idx | kept_cnt | select workspace | fwd workspace | status words |
 //   FP8 only: q/k/v codes, q/k/v scales
 namespace {
 struct Arena {
-  size_t q, k, v, out, idx, cnt, ws_sel, ws_fwd, cq, ck, cv, sq, sk, sv, total;
+  size_t q, k, v, out, idx, cnt, ws_sel, ws_fwd, status, cq, ck, cv, sq, sk, sv, total;
 };
 Arena plan_arena(const sparkattn_shape_t& s, int dtype, int topk) {
   Arena a;
@@ -245,6 +247,7 @@ Arena plan_arena(const sparkattn_shape_t& s, int dtype, int topk) {
   c.stride_n = s.d; c.stride_h = (int64_t)s.N * s.d; c.stride_b = (int64_t)s.H * s.N * s.d;
   a.ws_sel = take(select_workspace_bytes(c));
   a.ws_fwd = take(fwd_workspace_bytes(c, topk));
+  a.status = take(256);
   a.cq = a.ck = a.cv = a.sq = a.sk = a.sv = 0;
   if (dtype == SPARKATTN_FP8_E4M3) {
     a.cq = take(elems); a.ck = take(elems); a.cv = take(elems);
@@ -260,6 +263,29 @@ size_t sparkattn_arena_bytes(const sparkattn_shape_t* shape, int32_t dtype, int3
   return plan_arena(*shape, dtype, topk).total;
 }
 
+namespace {
+// Copy streams of the host-buffer path, one pair per device, created on first use and kept.
+struct HostPathStreams {
+  cudaStream_t in = nullptr, out = nullptr;
+};
+HostPathStreams* host_path_streams() {
+  static HostPathStreams per_device[64];
+  static std::mutex lock;
+  std::lock_guard<std::mutex> guard(lock);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPathStreams& hs = per_device[dev];
+  if (hs.in == nullptr && cudaStreamCreateWithFlags(&hs.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  if (hs.out == nullptr && cudaStreamCreateWithFlags(&hs.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  return &hs;
+}
+constexpr int kHostPathMaxChunks = 16;   // two status words per chunk fit the arena's 256-byte status region
+}  // namespace
+
+// The heads are independent problems, so the host path runs them as a pipeline of head groups:
+// group c+1 is copied in (copy stream) while group c is selected and attended (the caller's stream)
+// and the output of group c-1 is copied out (second copy stream); host->device and device->host
+// copies use different copy engines.  Each group's two status words are kept in the arena.
 int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, const void* q_host,
                              const void* k_host, const void* v_host, int32_t topk, void* out_host,
                              int32_t* kept_idx_host, void* arena, size_t arena_bytes, void* cuda_stream) {
@@ -275,46 +301,115 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
   const Arena a = plan_arena(s, dtype, topk);
   if (arena_bytes < a.total) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  HostPathStreams* hs = host_path_streams();
+  if (hs == nullptr) return SPARKATTN_E_CUDA;
   char* base = static_cast<char*>(arena);
-  const size_t bytes = (size_t)s.B * s.H * s.N * s.d * 2;
-  if (cudaMemcpyAsync(base + a.q, q_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(base + a.k, k_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(base + a.v, v_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-    return SPARKATTN_E_CUDA;
-  int32_t* idx = reinterpret_cast<int32_t*>(base + a.idx);
-  int32_t* cnt = reinterpret_cast<int32_t*>(base + a.cnt);
-  rc = sparkattn_select(&s, base + a.q, base + a.k, topk, idx, cnt, base + a.ws_sel, select_workspace_bytes(s),
-                        cuda_stream);
-  if (rc != SPARKATTN_OK) return rc;
-  const void *fq = base + a.q, *fk = base + a.k, *fv = base + a.v;
-  const float *sq = nullptr, *sk = nullptr, *sv = nullptr;
-  if (dtype == SPARKATTN_FP8_E4M3) {
-    const size_t tensor_off[3] = {a.q, a.k, a.v}, code_off[3] = {a.cq, a.ck, a.cv}, scale_off[3] = {a.sq, a.sk, a.sv};
-    for (int i = 0; i < 3; ++i) {
-      rc = sparkattn_quant_fp8(&s, base + tensor_off[i], reinterpret_cast<uint8_t*>(base + code_off[i]),
-                               reinterpret_cast<float*>(base + scale_off[i]), 0, cuda_stream);
-      if (rc != SPARKATTN_OK) return rc;
+
+  // head groups: about 8 per call, never across a batch boundary
+  const int total_heads = s.B * s.H;
+  int heads_per_chunk = (s.H + 7) / 8;
+  while ((int64_t)s.B * ((s.H + heads_per_chunk - 1) / heads_per_chunk) > kHostPathMaxChunks) ++heads_per_chunk;
+  struct Chunk { int b, h0, hc; };
+  Chunk chunks[kHostPathMaxChunks];
+  int n_chunks = 0;
+  for (int b = 0; b < s.B; ++b)
+    for (int h0 = 0; h0 < s.H; h0 += heads_per_chunk) chunks[n_chunks++] = Chunk{b, h0, min(heads_per_chunk, s.H - h0)};
+  (void)total_heads;
+
+  cudaEvent_t ev_start = nullptr, ev_in[kHostPathMaxChunks] = {}, ev_done[kHostPathMaxChunks] = {}, ev_out = nullptr;
+  auto destroy_events = [&]() {
+    if (ev_start) cudaEventDestroy(ev_start);
+    if (ev_out) cudaEventDestroy(ev_out);
+    for (int c = 0; c < n_chunks; ++c) {
+      if (ev_in[c]) cudaEventDestroy(ev_in[c]);
+      if (ev_done[c]) cudaEventDestroy(ev_done[c]);
     }
-    fq = base + a.cq; fk = base + a.ck; fv = base + a.cv;
-    sq = reinterpret_cast<const float*>(base + a.sq);
-    sk = reinterpret_cast<const float*>(base + a.sk);
-    sv = reinterpret_cast<const float*>(base + a.sv);
+  };
+  // after an enqueue error: let what is already in flight finish before the events go
+  auto fail = [&](int code) {
+    cudaStreamSynchronize(hs->in); cudaStreamSynchronize(stream); cudaStreamSynchronize(hs->out);
+    destroy_events();
+    return code;
+  };
+  bool ev_ok = cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming) == cudaSuccess &&
+               cudaEventCreateWithFlags(&ev_out, cudaEventDisableTiming) == cudaSuccess;
+  for (int c = 0; ev_ok && c < n_chunks; ++c)
+    ev_ok = cudaEventCreateWithFlags(&ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&ev_done[c], cudaEventDisableTiming) == cudaSuccess;
+  if (!ev_ok) { destroy_events(); return SPARKATTN_E_CUDA; }
+
+  // the copy streams start after whatever the caller already queued on its stream
+  if (cudaEventRecord(ev_start, stream) != cudaSuccess || cudaStreamWaitEvent(hs->in, ev_start, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(hs->out, ev_start, 0) != cudaSuccess)
+    return fail(SPARKATTN_E_CUDA);
+  if (cudaMemsetAsync(base + a.status, 0, 256, stream) != cudaSuccess) return fail(SPARKATTN_E_CUDA);
+
+  int32_t* idx_all = reinterpret_cast<int32_t*>(base + a.idx);
+  int32_t* cnt_all = reinterpret_cast<int32_t*>(base + a.cnt);
+  int32_t* status_dev = reinterpret_cast<int32_t*>(base + a.status);
+  for (int c = 0; c < n_chunks; ++c) {
+    const Chunk& ch = chunks[c];
+    const size_t elem_off = ((size_t)ch.b * s.H + ch.h0) * (size_t)s.N * s.d;   // elements before the group
+    const size_t bytes = (size_t)ch.hc * s.N * s.d * 2;
+    const size_t row_off = ((size_t)ch.b * s.H + ch.h0) * nb;                   // (head, block) rows before it
+    if (cudaMemcpyAsync(base + a.q + elem_off * 2, static_cast<const char*>(q_host) + elem_off * 2, bytes,
+                        cudaMemcpyHostToDevice, hs->in) != cudaSuccess ||
+        cudaMemcpyAsync(base + a.k + elem_off * 2, static_cast<const char*>(k_host) + elem_off * 2, bytes,
+                        cudaMemcpyHostToDevice, hs->in) != cudaSuccess ||
+        cudaMemcpyAsync(base + a.v + elem_off * 2, static_cast<const char*>(v_host) + elem_off * 2, bytes,
+                        cudaMemcpyHostToDevice, hs->in) != cudaSuccess ||
+        cudaEventRecord(ev_in[c], hs->in) != cudaSuccess || cudaStreamWaitEvent(stream, ev_in[c], 0) != cudaSuccess)
+      return fail(SPARKATTN_E_CUDA);
+
+    sparkattn_shape_t cs = s;      // one batch entry, the group's heads, strides of the full tensors
+    cs.B = 1; cs.H = ch.hc;
+    int32_t* idx = idx_all + row_off * topk;
+    int32_t* cnt = cnt_all + row_off;
+    rc = sparkattn_select(&cs, base + a.q + elem_off * 2, base + a.k + elem_off * 2, topk, idx, cnt, base + a.ws_sel,
+                          select_workspace_bytes(cs), cuda_stream);
+    if (rc != SPARKATTN_OK) return fail(rc);
+    const void *fq = base + a.q + elem_off * 2, *fk = base + a.k + elem_off * 2, *fv = base + a.v + elem_off * 2;
+    const float *sq = nullptr, *sk = nullptr, *sv = nullptr;
+    if (dtype == SPARKATTN_FP8_E4M3) {
+      const size_t tensor_off[3] = {a.q, a.k, a.v}, code_off[3] = {a.cq, a.ck, a.cv}, scale_off[3] = {a.sq, a.sk, a.sv};
+      for (int i = 0; i < 3; ++i) {
+        rc = sparkattn_quant_fp8(&cs, base + tensor_off[i] + elem_off * 2,
+                                 reinterpret_cast<uint8_t*>(base + code_off[i] + elem_off),
+                                 reinterpret_cast<float*>(base + scale_off[i]) + row_off, 0, cuda_stream);
+        if (rc != SPARKATTN_OK) return fail(rc);
+      }
+      fq = base + a.cq + elem_off; fk = base + a.ck + elem_off; fv = base + a.cv + elem_off;
+      sq = reinterpret_cast<const float*>(base + a.sq) + row_off;
+      sk = reinterpret_cast<const float*>(base + a.sk) + row_off;
+      sv = reinterpret_cast<const float*>(base + a.sv) + row_off;
+    }
+    rc = sparkattn_fwd(&cs, dtype, fq, fk, fv, sq, sk, sv, idx, cnt, topk, base + a.out + elem_off * 2, nullptr,
+                       base + a.ws_fwd, fwd_workspace_bytes(cs, topk), cuda_stream);
+    if (rc != SPARKATTN_OK) return fail(rc);
+    // the next group reuses both workspaces: keep this group's status words
+    if (cudaMemcpyAsync(status_dev + 2 * c, base + a.ws_sel, 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(status_dev + 2 * c + 1, base + a.ws_fwd, 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+        cudaEventRecord(ev_done[c], stream) != cudaSuccess || cudaStreamWaitEvent(hs->out, ev_done[c], 0) != cudaSuccess)
+      return fail(SPARKATTN_E_CUDA);
+    if (cudaMemcpyAsync(static_cast<char*>(out_host) + elem_off * 2, base + a.out + elem_off * 2, bytes,
+                        cudaMemcpyDeviceToHost, hs->out) != cudaSuccess)
+      return fail(SPARKATTN_E_CUDA);
+    if (kept_idx_host != nullptr &&
+        cudaMemcpyAsync(kept_idx_host + row_off * topk, idx, (size_t)ch.hc * nb * topk * 4, cudaMemcpyDeviceToHost,
+                        hs->out) != cudaSuccess)
+      return fail(SPARKATTN_E_CUDA);
   }
-  rc = sparkattn_fwd(&s, dtype, fq, fk, fv, sq, sk, sv, idx, cnt, topk, base + a.out, nullptr, base + a.ws_fwd,
-                     fwd_workspace_bytes(s, topk), cuda_stream);
-  if (rc != SPARKATTN_OK) return rc;
-  if (cudaMemcpyAsync(out_host, base + a.out, bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-    return SPARKATTN_E_CUDA;
-  if (kept_idx_host != nullptr &&
-      cudaMemcpyAsync(kept_idx_host, idx, (size_t)s.B * s.H * nb * topk * 4, cudaMemcpyDeviceToHost, stream) !=
-          cudaSuccess)
-    return SPARKATTN_E_CUDA;
-  int32_t st[2] = {0, 0};
-  if (cudaMemcpyAsync(&st[0], base + a.ws_sel, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-      cudaMemcpyAsync(&st[1], base + a.ws_fwd, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-    return SPARKATTN_E_CUDA;
-  if (cudaStreamSynchronize(stream) != cudaSuccess) return SPARKATTN_E_CUDA;
-  return st[0] != 0 ? st[0] : st[1];
+  // the caller's stream ends after the last copy out
+  if (cudaEventRecord(ev_out, hs->out) != cudaSuccess || cudaStreamWaitEvent(stream, ev_out, 0) != cudaSuccess)
+    return fail(SPARKATTN_E_CUDA);
+  int32_t st[2 * kHostPathMaxChunks] = {};
+  if (cudaMemcpyAsync(st, status_dev, sizeof(int32_t) * 2 * n_chunks, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return fail(SPARKATTN_E_CUDA);
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(SPARKATTN_E_CUDA);
+  destroy_events();
+  for (int i = 0; i < 2 * n_chunks; ++i)
+    if (st[i] != 0) return st[i];
+  return SPARKATTN_OK;
 }
 
 }  // extern "C"

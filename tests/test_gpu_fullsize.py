@@ -107,6 +107,24 @@ def test_host_buffer_call_matches_device_call():
         assert torch.equal(hidx, idx.cpu())
 
 
+@pytest.mark.parametrize("B,H,block", [(2, 5, 128), (1, 20, 64), (3, 7, 128)])
+def test_host_buffer_call_head_groups(B, H, block):
+    """The host path runs groups of heads as a pipeline; groups never straddle a batch entry, the last group of a
+    batch entry may be short, and with B*H > 16 groups the groups grow.  Result identical to the device calls."""
+    g = torch.Generator().manual_seed(100 * B + H)
+    N, d, topk = 700, 128, 3
+    q, k, v = (torch.randn((B, H, N, d), generator=g).to(torch.bfloat16) for _ in range(3))
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    idx, cnt = sa.select(qd, kd, block, topk)
+    ref = sa.fwd(qd, kd, vd, idx, cnt, block, check_status=True)
+    hidx = torch.empty(idx.shape, dtype=torch.int32).pin_memory()
+    out = sa.attention_host(q.pin_memory(), k.pin_memory(), v.pin_memory(), block, topk, kept_idx=hidx)
+    assert torch.equal(hidx, idx.cpu())
+    assert torch.equal(out, ref.cpu())
+    out2 = sa.attention_host(q, k, v, block, topk)          # pageable host memory: same result
+    assert torch.equal(out2, ref.cpu())
+
+
 def test_fullsize_paper_block_size_64_bf16_and_fp8():
     """Wan2.1-14B-720P shape with the paper's trained 64x64 blocks (nb = 1182, 35 kept at 97 %)."""
     w64 = workloads.Workload("wan14b_b64", 3, 1, 40, 128, (21, 45, 80), 64, 0.97)
