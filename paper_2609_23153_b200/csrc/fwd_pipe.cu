@@ -486,32 +486,63 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         q_sc = PAIR ? __ldg(p.q_scale + (int64_t)bh * p.nb + min(2 * qb + (row >> 6), p.nb - 1)) : __ldg(p.q_scale + item);
         v_max = __ldg(p.v_max + bh);
       }
-      for (int n = 0; ok && n < cnt; ++n) {
+      // This warpgroup's tiles are n0, n0 + 2, ...  List entries are fetched two of its tiles ahead and the FP8
+      // scales of a tile one tile ahead, so that neither load (nor the two in a row, entry then scale) is waited
+      // for inside the tile loop.
+      const int n0 = (g ^ t) & 1;
+      const int32_t* lst = p.clean_list + (int64_t)item * p.lstride;
+      const float* ksc = FP8 ? p.k_scale + (int64_t)bh * p.nb : nullptr;
+      const float* vsc = FP8 ? p.v_scale + (int64_t)bh * p.nb : nullptr;
+      auto ld_ent = [&](int n, int e) { return n < cnt ? __ldg(lst + n * kEnt + e) : 0; };
+      int e_cur0 = ld_ent(n0, 0), e_cur1 = PAIR ? ld_ent(n0, 1) : 0;
+      int e_nx0 = ld_ent(n0 + 2, 0), e_nx1 = PAIR ? ld_ent(n0 + 2, 1) : 0;
+      float ks_cur0 = 1.0f, vs_cur0 = 1.0f, ks_cur1 = 1.0f, vs_cur1 = 1.0f;
+      if constexpr (FP8) {
+        ks_cur0 = __ldg(ksc + (e_cur0 & 0x3fffffff));
+        vs_cur0 = __ldg(vsc + (e_cur0 & 0x3fffffff));
+        if constexpr (PAIR) {
+          ks_cur1 = __ldg(ksc + (e_cur1 & 0x3fffffff));
+          vs_cur1 = __ldg(vsc + (e_cur1 & 0x3fffffff));
+        }
+      }
+      const float inv_vmax = 1.0f / v_max;
+      for (int n = n0; ok && n < cnt; n += 2) {
         const int tt = t + n;
-        if ((tt & 1) != g) continue;
         const int buf = g;                          // (tt & 1) == g: this warpgroup's S and P buffers
         // the tile's key block(s); PAIR: two 64-token blocks, each with a flag per query block of the pair
+        const int e0 = e_cur0, e1 = e_cur1;
+        const float ks0 = ks_cur0, vs0 = vs_cur0, ks1 = ks_cur1, vs1 = vs_cur1;
+        // next tile of this warpgroup: its scales (its entries arrived a tile ago), and the entries of the one after
+        if constexpr (FP8) {
+          ks_cur0 = __ldg(ksc + (e_nx0 & 0x3fffffff));
+          vs_cur0 = __ldg(vsc + (e_nx0 & 0x3fffffff));
+          if constexpr (PAIR) {
+            ks_cur1 = __ldg(ksc + (e_nx1 & 0x3fffffff));
+            vs_cur1 = __ldg(vsc + (e_nx1 & 0x3fffffff));
+          }
+        }
+        e_cur0 = e_nx0; e_cur1 = e_nx1;
+        e_nx0 = ld_ent(n + 4, 0);
+        if constexpr (PAIR) e_nx1 = ld_ent(n + 4, 1);
         int kb, kb1 = 0;
         bool mem0 = true, mem1 = true;
         if constexpr (PAIR) {
-          const int e0 = __ldg(p.clean_list + (int64_t)item * p.lstride + 2 * n);
-          const int e1 = __ldg(p.clean_list + (int64_t)item * p.lstride + 2 * n + 1);
           kb = e0 & 0x3fffffff;
           kb1 = e1 & 0x3fffffff;
           mem0 = (((uint32_t)e0 >> (30 + (row >> 6))) & 1u) != 0u;
           mem1 = (((uint32_t)e1 >> (30 + (row >> 6))) & 1u) != 0u;
         } else {
-          kb = __ldg(p.clean_list + (int64_t)item * p.lstride + n);
+          kb = e0;
         }
         float c = p.scale_log2;                      // logit -> log2 units
         float p_off = 0.0f;                          // log2 of the factor folded into P
         float c1 = c, p_off1 = 0.0f;                 // PAIR + FP8: the second key block of the tile has its own scales
         if constexpr (FP8) {
-          c *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb);
-          p_off = kPipeFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb) / v_max);
+          c *= q_sc * ks0;
+          p_off = kPipeFp8PScaleLog2 + log2f(vs0 * inv_vmax);
           if constexpr (PAIR) {
-            c1 *= q_sc * __ldg(p.k_scale + (int64_t)bh * p.nb + kb1);
-            p_off1 = kPipeFp8PScaleLog2 + log2f(__ldg(p.v_scale + (int64_t)bh * p.nb + kb1) / v_max);
+            c1 *= q_sc * ks1;
+            p_off1 = kPipeFp8PScaleLog2 + log2f(vs1 * inv_vmax);
           }
         }
         // this row's valid columns: [c_lo, c_hi) of the tile, or (PAIR) [c_lo, c_hi) of its first 64 and
