@@ -343,7 +343,24 @@ def run_ours(args, w):
                "fwd_frac_of_nominal_fp8_peak_4500": flops / (ms_f8 * 1e-3) / 1e12 / 4500.0,
                "fwd_frac_of_2x_measured_bf16_peak": flops / (ms_f8 * 1e-3) / 1e12 / (2 * peaks["bf16"]),
                "note": "FP8 peak = measured bf16 peak x 2 (nominal ratio); torch._scaled_mm 8192^3 measured 3122 TFLOP/s on this pool"}
-        del codes
+        # per-token activation quantisation (the paper's fused scale-and-cast kernel), one tensor, outside the step
+        tok_scales = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+        evt = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+
+        def step_tok(i):
+            if i >= 0:
+                evt[i][0].record(stream)
+            sa.quant_fp8_per_token(v if i % 2 else k, codes=codes[0], scales=tok_scales)
+            if i >= 0:
+                evt[i][1].record(stream)
+
+        time_region(step_tok, K, args.warmup, stream, dist_on)
+        ms_tok = statistics.mean(a.elapsed_time(b) for a, b in evt)
+        tbytes = elems * 3 + tok_scales.numel() * 4
+        fp8["quant_per_token_ms"] = ms_tok
+        fp8["quant_per_token_GBps"] = tbytes / (ms_tok * 1e-3) / 1e9
+        fp8["quant_per_token_frac_of_hbm_peak"] = tbytes / (ms_tok * 1e-3) / 1e9 / peaks["hbm"]
+        del codes, tok_scales
 
     # ---- compensation branch + gate fusion (d = 128 only): state pass over K, V, then the fused apply pass
     comp = None

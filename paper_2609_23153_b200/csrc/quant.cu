@@ -86,23 +86,26 @@ quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ code
   }
 }
 
-// Per-token variant: a token row (d channels) is spread over d/8 lanes, 16 bytes per lane, so a
-// warp covers 32/(d/8) rows per step; it walks kTokenSteps steps with all loads issued first
-// (128 bytes in flight per thread).  absmax by shuffles inside the lane group, then scale,
-// encode and store from the same registers: one HBM read, one write.
-constexpr int kTokenSteps = 8;
+// Per-token variant: a token row (d channels) is spread over 4 lanes; lane c of the group takes the
+// 16-byte chunks c, c + 4, ... of the row, so that one load instruction of the warp covers 64
+// contiguous bytes of each of 8 rows.  A warp walks kTokenSteps steps of 8 rows with all loads issued
+// first (128 bytes in flight per thread).  absmax over the lane's chunks, two shuffles inside the lane
+// group, then the two IEEE divisions once per row (they are a third of the instructions when a lane
+// holds a single chunk), encode and store from the same registers: one HBM read, one write.
+constexpr int kTokenSteps = 2;
+constexpr int kTokenLanes = 4;                   // lanes per row
+constexpr int kTokenRows = 32 / kTokenLanes;     // rows per warp step
 
 template <int D>
 __global__ void __launch_bounds__(kQuantThreads)
 quant_fp8_token_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ scales,
                        int H, int N, int64_t stride_b, int64_t stride_h, int64_t stride_n, int64_t n_rows) {
-  constexpr int LPR = D / 8;                     // lanes per row: 16 (d=128) or 8 (d=64)
-  constexpr int RPS = 32 / LPR;                  // rows per warp step
+  constexpr int CPL = D / 8 / kTokenLanes;       // chunks per lane: 4 (d=128) or 2 (d=64)
   const int lane = threadIdx.x & 31;
-  const int sub = lane / LPR, chunk = lane % LPR;
+  const int sub = lane / kTokenLanes, chunk = lane % kTokenLanes;
   const int64_t warp_id = (int64_t)blockIdx.x * (kQuantThreads / 32) + (threadIdx.x >> 5);
-  const int64_t row0 = warp_id * (kTokenSteps * RPS);
-  uint4 v[kTokenSteps];
+  const int64_t row0 = warp_id * (kTokenSteps * kTokenRows);
+  uint4 v[kTokenSteps][CPL];
   int64_t off[kTokenSteps];
   // (batch, head, token) of this lane's first row: divisions once, then the rows just count up
   const uint32_t first = (uint32_t)(row0 + sub);            // n_rows < 2^31 (checked by the launcher)
@@ -111,45 +114,53 @@ quant_fp8_token_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict_
   int b = (int)(bh0 / (uint32_t)H), h = (int)(bh0 - (uint32_t)b * (uint32_t)H);
 #pragma unroll
   for (int u = 0; u < kTokenSteps; ++u) {
-    const int64_t r = row0 + u * RPS + sub;
+    const int64_t r = row0 + u * kTokenRows + sub;
     off[u] = b * stride_b + h * stride_h + (int64_t)n * stride_n + chunk * 8;
-    n += RPS;
+    n += kTokenRows;
     while (n >= N) {
       n -= N;
       if (++h == H) { h = 0; ++b; }
     }
-    v[u] = (r < n_rows) ? __ldg(reinterpret_cast<const uint4*>(x + off[u])) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int c = 0; c < CPL; ++c)
+      v[u][c] = (r < n_rows) ? __ldg(reinterpret_cast<const uint4*>(x + off[u] + c * (kTokenLanes * 8)))
+                             : make_uint4(0u, 0u, 0u, 0u);
   }
 #pragma unroll
   for (int u = 0; u < kTokenSteps; ++u) {
-    const int64_t r = row0 + u * RPS + sub;
-    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v[u]);
-    float f[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float2 t = __bfloat1622float2(p2[j]);
-      f[2 * j] = t.x;
-      f[2 * j + 1] = t.y;
-    }
+    const int64_t r = row0 + u * kTokenRows + sub;
+    float f[CPL][8];
     float amax = 0.0f;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(f[j]));
+    for (int c = 0; c < CPL; ++c) {
+      const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&v[u][c]);
 #pragma unroll
-    for (int o = LPR / 2; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      for (int j = 0; j < 4; ++j) {
+        const float2 t = __bfloat1622float2(p2[j]);
+        f[c][2 * j] = t.x;
+        f[c][2 * j + 1] = t.y;
+        amax = fmaxf(amax, fmaxf(fabsf(t.x), fabsf(t.y)));
+      }
+    }
+#pragma unroll
+    for (int o = kTokenLanes / 2; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
     amax = fmaxf(amax, 1e-12f);
     const float inv = __fdiv_rn(448.0f, amax);
     if (r >= n_rows) continue;
     if (chunk == 0) scales[r] = __fdiv_rn(amax, 448.0f);
-    uint32_t w[2];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f[4 * j], inv), __fmul_rn(f[4 * j + 1], inv)),
-                                                    __NV_SATFINITE, __NV_E4M3);
-      const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f[4 * j + 2], inv), __fmul_rn(f[4 * j + 3], inv)),
-                                                    __NV_SATFINITE, __NV_E4M3);
-      w[j] = lo | (hi << 16);
+    for (int c = 0; c < CPL; ++c) {
+      uint32_t w[2];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f[c][4 * j], inv), __fmul_rn(f[c][4 * j + 1], inv)),
+                                                      __NV_SATFINITE, __NV_E4M3);
+        const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(__fmul_rn(f[c][4 * j + 2], inv), __fmul_rn(f[c][4 * j + 3], inv)),
+                                                      __NV_SATFINITE, __NV_E4M3);
+        w[j] = lo | (hi << 16);
+      }
+      *reinterpret_cast<uint2*>(codes + off[u] + c * (kTokenLanes * 8)) = make_uint2(w[0], w[1]);
     }
-    *reinterpret_cast<uint2*>(codes + off[u]) = make_uint2(w[0], w[1]);
   }
 }
 
@@ -157,7 +168,7 @@ int launch_quant_fp8_per_token(const sparkattn_shape_t& s, const void* x, uint8_
                                cudaStream_t stream) {
   const int64_t n_rows = (int64_t)s.B * s.H * s.N;
   if (n_rows >= (1LL << 31) - 4096) return SPARKATTN_E_UNSUPPORTED_SHAPE;
-  const int64_t rows_per_cta = (kQuantThreads / 32) * kTokenSteps * (32 / (s.d / 8));
+  const int64_t rows_per_cta = (kQuantThreads / 32) * kTokenSteps * kTokenRows;
   const int64_t ctas = (n_rows + rows_per_cta - 1) / rows_per_cta;
   if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
