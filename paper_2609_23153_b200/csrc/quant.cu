@@ -17,7 +17,7 @@ namespace sparkattn {
 constexpr int kQuantThreads = 256;
 
 template <int D, int BLK>
-__global__ void __launch_bounds__(kQuantThreads)
+__global__ void __launch_bounds__(kQuantThreads, 3)
 quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ scales,
                  int H, int N, int nb, int64_t stride_b, int64_t stride_h, int64_t stride_n) {
   constexpr int kChunksPerRow = D / 8;                      // 16-byte chunks per token row
@@ -97,7 +97,7 @@ constexpr int kTokenLanes = 4;                   // lanes per row
 constexpr int kTokenRows = 32 / kTokenLanes;     // rows per warp step
 
 template <int D>
-__global__ void __launch_bounds__(kQuantThreads)
+__global__ void __launch_bounds__(kQuantThreads, 3)
 quant_fp8_token_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ scales,
                        int H, int N, int64_t stride_b, int64_t stride_h, int64_t stride_n, int64_t n_rows) {
   constexpr int CPL = D / 8 / kTokenLanes;       // chunks per lane: 4 (d=128) or 2 (d=64)
