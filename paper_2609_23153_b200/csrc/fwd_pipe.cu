@@ -66,7 +66,7 @@ struct PipeParams {
   float scale_log2;
 };
 
-// one warp per item: drop (and report) kept indices outside [0, nb), clamp the count
+// one warp per item: drop (and report) kept indices outside [0, nb), clamp the count, own block first
 __global__ void compact_lists_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restrict__ kept_cnt,
                                      int32_t* __restrict__ clean_cnt, int32_t* __restrict__ clean_list, int items,
                                      int nb, int kmax, int32_t* status) {
@@ -87,6 +87,29 @@ __global__ void compact_lists_kernel(const int32_t* __restrict__ kept_idx, const
     out += __popc(ballot);
   }
   if (lane == 0) clean_cnt[item] = out;
+  // The query block's own key block goes first.  The result does not depend on the order of the tiles, the
+  // work does: a row's running maximum is usually set by its own block, and when that block comes late (it is
+  // the last entry of an ascending list under a causal window) nearly every row's maximum jumps past the lazy
+  // threshold there and the whole O tile is rescaled; with it first the later tiles stay below the reference.
+  __syncwarp();
+  const int qb = item % nb;
+  int p = -1;
+  for (int base = 0; base < out && p < 0; base += 32) {
+    const int t = base + lane;
+    const uint32_t hit = __ballot_sync(0xffffffffu, t < out && dst[t] == qb);
+    if (hit) p = base + __ffs(hit) - 1;
+  }
+  if (p > 0) {
+    for (int base = (p / 32) * 32; base >= 0; base -= 32) {      // shift entries 0..p-1 up by one, highest chunk first
+      const int t = base + lane;
+      const bool mine = t <= p;
+      int val = 0;
+      if (mine) val = (t == 0) ? qb : dst[t - 1];
+      __syncwarp();
+      if (mine) dst[t] = val;
+      __syncwarp();
+    }
+  }
 }
 
 // 64-token blocks: the kernel works on pairs of adjacent query blocks (128 query rows, the MMA's M) and on
