@@ -146,12 +146,23 @@ pair_lists_kernel(const int32_t* __restrict__ kept_idx, const int32_t* __restric
   __syncwarp();
   int32_t* dst = clean_list + (int64_t)pair * (2 * kmax);
   int out = 0;
+  // the pair's own two key blocks first (see compact_lists_kernel), then the rest in ascending order
+  const int own0 = 2 * qp;
+  for (int kb = own0; kb <= own0 + 1 && kb < nb; ++kb) {
+    const bool ina = (bits[kb >> 5] >> (kb & 31)) & 1u, inb = (bits[words + (kb >> 5)] >> (kb & 31)) & 1u;
+    if (ina || inb) {
+      if (lane == 0) dst[out] = kb | (ina ? (1 << 30) : 0) | (inb ? (int)(1u << 31) : 0);
+      ++out;
+    }
+  }
   for (int base = 0; base < nb; base += 32) {
     const int kb = base + lane;
     const uint32_t a = bits[base >> 5], bmask = bits[words + (base >> 5)];
     const bool ina = (a >> lane) & 1u, inb = (bmask >> lane) & 1u;
-    const uint32_t u = a | bmask;
-    if (ina || inb) dst[out + __popc(u & ((1u << lane) - 1u))] = kb | (ina ? (1 << 30) : 0) | (inb ? (int)(1u << 31) : 0);
+    uint32_t u = a | bmask;
+    if (base == (own0 & ~31)) u &= ~(3u << (own0 & 31));        // own0 is even: both own blocks lie in one word
+    const bool sel = (u >> lane) & 1u;
+    if (sel) dst[out + __popc(u & ((1u << lane) - 1u))] = kb | (ina ? (1 << 30) : 0) | (inb ? (int)(1u << 31) : 0);
     out += __popc(u);
   }
   __syncwarp();
