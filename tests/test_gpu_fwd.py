@@ -195,3 +195,46 @@ def test_persistent_path_short_and_empty_lists(seed, kmax, block):
             if cnt[h, i] == 0:
                 rows = slice(i * w.block, min(w.N, (i + 1) * w.block))
                 assert torch.all(out[0, h, rows] == 0) and torch.all(torch.isneginf(lse[0, h, rows]))
+
+
+@pytest.mark.parametrize("block,fp8", [(128, False), (128, True), (64, False)])
+def test_long_permuted_lists_own_block_anywhere(block, fp8):
+    """Kept lists of 70-100 entries in random order: the forward's list pre-pass moves the query block's own
+    key block to the front, wherever it stands (first, inside the first 32 entries, beyond them, at a
+    multiple of 32, last, absent), and must keep every other entry exactly once.  Compared with the oracle,
+    which walks the lists as given."""
+    nbk = 100
+    N = nbk * block - 17
+    g = torch.Generator().manual_seed(7 + block + int(fp8))
+    H, d, kmax = 2, 128, 100
+    q, k, v = (torch.randn((1, H, N, d), generator=g).to(torch.bfloat16) for _ in range(3))
+    idx = torch.stack([torch.stack([torch.randperm(nbk, generator=g) for _ in range(nbk)]) for _ in range(H)]).to(torch.int32)
+    cnt = torch.randint(70, kmax + 1, (H, nbk), generator=g, dtype=torch.int32)
+    for h in range(H):                      # the own block at chosen places of some lists
+        for qb, pos in [(0, 0), (1, 5), (2, 31), (3, 32), (4, 33), (5, 64), (6, 69), (7, 96)]:
+            row = idx[h, qb].tolist()
+            row.remove(qb)
+            row.insert(pos, qb)
+            idx[h, qb] = torch.tensor(row, dtype=torch.int32)
+        cnt[h, 7] = 97                      # own block last
+        cnt[h, 8] = 70
+        row = [j for j in idx[h, 8].tolist() if j != 8] + [8]
+        idx[h, 8] = torch.tensor(row, dtype=torch.int32)    # own block beyond the count: absent
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    items = [(h, qb) for h in range(H) for qb in (0, 1, 2, 3, 4, 5, 6, 7, 8, 50, nbk - 1)]
+    if fp8:
+        cs = [sa.quant_fp8(t, block) for t in (qd, kd, vd)]
+        out = sa.fwd(cs[0][0], cs[1][0], cs[2][0], idx[None].to(DEV), cnt[None].to(DEV), block,
+                     scales=tuple(s for _, s in cs), check_status=True)
+        ref, _ = oracle.attention(cs[0][0][0].cpu(), cs[1][0][0].cpu(), cs[2][0][0].cpu(), idx, cnt, block,
+                                  scales=tuple(s[0].cpu() for _, s in cs), items=items)
+    else:
+        out = sa.fwd(qd, kd, vd, idx[None].to(DEV), cnt[None].to(DEV), block, check_status=True)
+        ref, _ = oracle.attention(q[0], k[0], v[0], idx, cnt, block, items=items)
+    num = den = 0.0
+    for n, (h, qb) in enumerate(items):
+        rows = slice(qb * block, min(N, (qb + 1) * block))
+        got = out[0, h, rows].cpu().double()
+        want = ref[n, : got.shape[0]]
+        num += float(((got - want) ** 2).sum()); den += float((want ** 2).sum())
+    assert (num / den) ** 0.5 <= (5e-2 if fp8 else 1e-2)
