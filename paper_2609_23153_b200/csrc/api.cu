@@ -306,7 +306,6 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
   char* base = static_cast<char*>(arena);
 
   // head groups: about 8 per call, never across a batch boundary
-  const int total_heads = s.B * s.H;
   int heads_per_chunk = (s.H + 7) / 8;
   while ((int64_t)s.B * ((s.H + heads_per_chunk - 1) / heads_per_chunk) > kHostPathMaxChunks) ++heads_per_chunk;
   struct Chunk { int b, h0, hc; };
@@ -314,7 +313,6 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
   int n_chunks = 0;
   for (int b = 0; b < s.B; ++b)
     for (int h0 = 0; h0 < s.H; h0 += heads_per_chunk) chunks[n_chunks++] = Chunk{b, h0, min(heads_per_chunk, s.H - h0)};
-  (void)total_heads;
 
   cudaEvent_t ev_start = nullptr, ev_in[kHostPathMaxChunks] = {}, ev_done[kHostPathMaxChunks] = {}, ev_out = nullptr;
   auto destroy_events = [&]() {
