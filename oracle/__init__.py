@@ -100,6 +100,7 @@ def attention(
     softmax_scale: float = 0.0,
     frame_tokens: int = 0,
     window: int = 0,
+    block_valid: Optional[torch.Tensor] = None,
 ):
     """ATT-0.  q, k, v: [H, N, d] bf16, or uint8 E4M3 codes with
     ``scales = (q_scale, k_scale, v_scale)`` each fp32 [H, nb].
@@ -107,7 +108,9 @@ def attention(
     Returns (out fp64 [n_items, block, d], lse fp64 [n_items, block]) for the
     (head, query-block) pairs in ``items`` (default: all, head-major).
     WIN-0: with ``frame_tokens`` = F > 0, key j counts for query i only if its frame j // F lies in
-    (i // F - window, i // F]; a row with no such kept key gives out = 0, lse = -inf."""
+    (i // F - window, i // F]; a row with no such kept key gives out = 0, lse = -inf.
+    ORD-0: with ``block_valid`` (int32 [nb]) block b holds block_valid[b] tokens followed by padding rows,
+    which are neither keys nor evaluated as queries (their output rows stay 0)."""
     L = _load()
     H, N, d = q.shape
     nb = (N + block - 1) // block
@@ -134,25 +137,28 @@ def attention(
         ctypes.c_int(dtype), _ptr(qq), _ptr(kk), _ptr(vv), _ptr(sq), _ptr(sk), _ptr(sv),
         ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d), ctypes.c_int(block),
         _ptr(ki), _ptr(kc), ctypes.c_int(kmax), ctypes.c_double(softmax_scale),
-        _ptr(it), ctypes.c_int(n_items), ctypes.c_int(frame_tokens), ctypes.c_int(window), _ptr(out), _ptr(lse))
+        _ptr(it), ctypes.c_int(n_items), ctypes.c_int(frame_tokens), ctypes.c_int(window),
+        _ptr(None if block_valid is None else block_valid.contiguous().to(torch.int32)), _ptr(out), _ptr(lse))
     if rc != 0:
         raise ValueError("kept_idx holds a block index outside [0, nb)")
     return out, lse
 
 
-def pool(x: torch.Tensor, block: int) -> torch.Tensor:
-    """SEL-1 steps 1-2: pooled fp32 block means [H, nb, d] of a bf16 [H, N, d] tensor."""
+def pool(x: torch.Tensor, block: int, block_valid: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """SEL-1 steps 1-2: pooled fp32 block means [H, nb, d] of a bf16 [H, N, d] tensor (ORD-0: over the first
+    block_valid[b] tokens of block b)."""
     L = _load()
     H, N, d = x.shape
     nb = (N + block - 1) // block
     out = torch.empty((H, nb, d), dtype=torch.float32)
     L.oracle_pool(_ptr(_raw16(x)), ctypes.c_int(H), ctypes.c_int(N), ctypes.c_int(d),
-                  ctypes.c_int(block), _ptr(out))
+                  ctypes.c_int(block), _ptr(None if block_valid is None else block_valid.contiguous().to(torch.int32)),
+                  _ptr(out))
     return out
 
 
 def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, return_scores: bool = False,
-           frame_tokens: int = 0, window: int = 0):
+           frame_tokens: int = 0, window: int = 0, block_valid: Optional[torch.Tensor] = None):
     """SEL-1.  q, k: [H, N, d] bf16.  Returns kept_idx int32 [H, nb, topk]
     (ascending), kept_cnt int32 [H, nb] (and the fp32 scores [H, nb, nb]).
     WIN-0: with ``frame_tokens`` > 0 only key blocks inside the causal frame window of the query
@@ -165,7 +171,9 @@ def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, return_score
     scores = torch.empty((H, nb, nb), dtype=torch.float32) if return_scores else None
     rc = L.oracle_select(_ptr(_raw16(q)), _ptr(_raw16(k)), ctypes.c_int(H), ctypes.c_int(N),
                          ctypes.c_int(d), ctypes.c_int(block), ctypes.c_int(topk),
-                         ctypes.c_int(frame_tokens), ctypes.c_int(window), _ptr(idx), _ptr(cnt), _ptr(scores))
+                         ctypes.c_int(frame_tokens), ctypes.c_int(window),
+                         _ptr(None if block_valid is None else block_valid.contiguous().to(torch.int32)),
+                         _ptr(idx), _ptr(cnt), _ptr(scores))
     if rc != 0:
         raise ValueError("topk must be in [1, nb]")
     return (idx, cnt, scores) if return_scores else (idx, cnt)
@@ -237,3 +245,29 @@ def comp_apply(q: torch.Tensor, pq: torch.Tensor, state: torch.Tensor, gate: tor
                         _ptr(freq.contiguous().float()), ctypes.c_double(eps), _ptr(rr), ctypes.c_int(rr.shape[0]),
                         _ptr(out))
     return out
+
+
+def brick_layout(grid, brick, block: int):
+    """ORD-0, token order of 3-D bricks padded to whole blocks (the paper fixes contiguous blocks, Sec. 2, not
+    the order of the tokens): the (T, Hg, Wg) grid is cut into bricks of (bt, bh, bw) cells with
+    bt * bh * bw <= block, cut short at the far faces; bricks are visited in raster order of the brick grid,
+    the cells of a brick in raster order inside it; every brick takes one block, its cells first, padding
+    after them.  Written as that enumeration.  Returns (gather int32 [nbricks * block]: the raster index
+    n = (t * Hg + y) * Wg + x of the token at each padded position, -1 for padding; block_valid int32
+    [nbricks]; scatter int32 [N]: the padded position of raster token n)."""
+    T, Hg, Wg = (int(v) for v in grid)
+    bt, bh, bw = (int(v) for v in brick)
+    assert bt * bh * bw <= block
+    gather, valid = [], []
+    for t0 in range(0, T, bt):
+        for y0 in range(0, Hg, bh):
+            for x0 in range(0, Wg, bw):
+                cells = [(t * Hg + y) * Wg + x for t in range(t0, min(T, t0 + bt)) for y in range(y0, min(Hg, y0 + bh))
+                         for x in range(x0, min(Wg, x0 + bw))]
+                valid.append(len(cells))
+                gather.extend(cells + [-1] * (block - len(cells)))
+    gather = torch.tensor(gather, dtype=torch.int32)
+    scatter = torch.empty(T * Hg * Wg, dtype=torch.int32)
+    pos = torch.nonzero(gather >= 0).flatten()
+    scatter[gather[pos].long()] = pos.to(torch.int32)
+    return gather, torch.tensor(valid, dtype=torch.int32), scatter

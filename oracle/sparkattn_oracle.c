@@ -34,6 +34,14 @@
  *                             j / F lies in (i / F - window, i / F].  Selection only
  *                             ranks the key blocks that hold such a key for some row
  *                             of the query block.
+ *   ORD-0  block_valid argument of oracle_attention, oracle_pool and oracle_select: tokens
+ *                             stored in bricks padded to whole blocks (block b holds
+ *                             block_valid[b] tokens followed by padding rows).  The paper
+ *                             only says that blocks are contiguous (Sec. 2) and fixes no
+ *                             token order; reading: padding rows are not keys, do not
+ *                             enter the pooled means, and their query rows are not
+ *                             evaluated.  The brick order itself is index arithmetic in
+ *                             the Python front-end.
  *
  * OpenMP only distributes independent work items (one (head, query block) or
  * one (head, block) each); inside an item everything is a scalar loop in the
@@ -119,7 +127,8 @@ static inline double load_elem(const void* x, const float* scale, int dtype, int
 int oracle_attention(int dtype, const void* q, const void* k, const void* v, const float* q_scale,
                      const float* k_scale, const float* v_scale, int H, int N, int d, int blk,
                      const int32_t* kept_idx, const int32_t* kept_cnt, int kmax, double scale,
-                     const int32_t* items, int n_items, int frame_tokens, int window, double* out, double* lse) {
+                     const int32_t* items, int n_items, int frame_tokens, int window,
+                     const int32_t* block_valid /* [nb] or NULL */, double* out, double* lse) {
   const int64_t nb = ((int64_t)N + blk - 1) / blk;
   if (scale == 0.0) scale = 1.0 / sqrt((double)d);
   int bad = 0;
@@ -137,13 +146,15 @@ int oracle_attention(int dtype, const void* q, const void* k, const void* v, con
       for (int c = 0; c < d; ++c) o[c] = 0.0;
       lse[(int64_t)it * blk + r] = 0.0;
       if (i >= N) continue;
+      if (block_valid && r >= block_valid[qb]) continue;       /* ORD-0: a padding row */
       for (int c = 0; c < d; ++c) qrow[c] = load_elem(q, q_scale, dtype, N, d, blk, nb, h, i, c);
       int64_t nk = 0;
       double m = -INFINITY;
       for (int t = 0; t < cnt; ++t) {
         const int64_t kb = list[t];
         if (kb < 0 || kb >= nb) { bad = 1; continue; }
-        for (int64_t j = kb * blk; j < (kb + 1) * blk && j < N; ++j) {
+        const int64_t jend = kb * blk + (block_valid ? block_valid[kb] : blk);    /* ORD-0: padding rows are not keys */
+        for (int64_t j = kb * blk; j < jend && j < N; ++j) {
           /* causal window over frames (WIN-0): key frame in (query frame - window, query frame] */
           if (frame_tokens > 0) {
             const int64_t fi = i / frame_tokens, fj = j / frame_tokens;
@@ -183,12 +194,14 @@ int oracle_attention(int dtype, const void* q, const void* k, const void* v, con
  * Step 5  write the kept indices in ascending index order.
  * The 1/sqrt(d) factor is omitted: it does not change the ranking.
  */
-void oracle_pool(const uint16_t* x, int H, int N, int d, int blk, float* pooled /* [H][nb][d] */) {
+void oracle_pool(const uint16_t* x, int H, int N, int d, int blk, const int32_t* block_valid /* [nb] or NULL */,
+                 float* pooled /* [H][nb][d] */) {
   const int64_t nb = ((int64_t)N + blk - 1) / blk;
 #pragma omp parallel for schedule(static)
   for (int64_t hb = 0; hb < (int64_t)H * nb; ++hb) {
     const int64_t h = hb / nb, b = hb % nb;
-    const int64_t t0 = b * blk, t1 = (t0 + blk < N) ? t0 + blk : N;
+    int64_t t0 = b * blk, t1 = (t0 + blk < N) ? t0 + blk : N;
+    if (block_valid && t0 + block_valid[b] < t1) t1 = t0 + block_valid[b];      /* ORD-0: valid tokens only */
     for (int c = 0; c < d; ++c) {
       float sum = 0.0f;
       for (int64_t t = t0; t < t1; ++t) sum = sum + bf16_to_f32(x[(h * N + t) * d + c]);
@@ -215,15 +228,15 @@ static int int_cmp(const void* a, const void* b) {
 
 /* scores_out (optional, may be NULL): [H][nb][nb] fp32 scores, for inspection in tests. */
 int oracle_select(const uint16_t* q, const uint16_t* k, int H, int N, int d, int blk, int topk,
-                  int frame_tokens, int window,
+                  int frame_tokens, int window, const int32_t* block_valid /* [nb] or NULL */,
                   int32_t* kept_idx /* [H][nb][topk] */, int32_t* kept_cnt /* [H][nb] or NULL */,
                   float* scores_out) {
   const int64_t nb = ((int64_t)N + blk - 1) / blk;
   if (topk < 1 || topk > nb) return -1;
   float* pq = (float*)malloc(sizeof(float) * (size_t)H * nb * d);
   float* pk = (float*)malloc(sizeof(float) * (size_t)H * nb * d);
-  oracle_pool(q, H, N, d, blk, pq);
-  oracle_pool(k, H, N, d, blk, pk);
+  oracle_pool(q, H, N, d, blk, block_valid, pq);
+  oracle_pool(k, H, N, d, blk, block_valid, pk);
 #pragma omp parallel for schedule(static)
   for (int64_t hi = 0; hi < (int64_t)H * nb; ++hi) {
     const int64_t h = hi / nb;
