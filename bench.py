@@ -24,6 +24,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -42,6 +43,8 @@ METRIC = "block-sparse attn effective TFLOP/s (kept FLOPs), select+fwd, 97% spar
 UNIT = "TFLOP/s"
 # DRAM bytes (read + write) of one bf16 forward launch on the default workload (wan14b, 97 %),
 # from the one-pass ncu capture summarised in profiles/launch_list_wan14b_s97.md.
+# bricks (frames x rows x columns of the token grid) that tile the grid of each workload; one 128-token block each
+BRICKS = {"wan14b": (3, 5, 8), "wan1p3b": (3, 5, 4)}
 FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2580123136 + 761104384}   # ncu one-pass capture of the full-size fwd_pipe_kernel launch
 
 
@@ -397,6 +400,66 @@ def run_ours(args, w):
                 "launches_per_step": 3}
         del fused, state, ws_c, pq, pk, gate
 
+    # ---- brick token order (d = 128, 128-token blocks): gather into bricks padded to whole blocks, selection and
+    # forward with per-block token counts, and how much of the attention mass the kept blocks hold in either order
+    bricks = None
+    if not args.no_bricks and w.d == 128 and w.block == 128 and not args.block:
+        brick = BRICKS.get(w.name)
+        gather, valid, scatter = sa.brick_layout(w.grid, brick, w.block, device=dev)
+        nbr = valid.numel()
+        topk_b = max(1, int((1.0 - w.sparsity) * nbr + 0.5))
+        qb_ = sa.gather_tokens(q, gather); kb_ = sa.gather_tokens(k, gather); vb_ = sa.gather_tokens(v, gather)
+        shape_b = sa.make_shape(qb_, w.block)
+        ws_sb = sa.alloc_workspace(shape_b, 0, topk_b, dev); ws_fb = sa.alloc_workspace(shape_b, 1, topk_b, dev)
+        idx_b, cnt_b = sa.select(qb_, kb_, w.block, topk_b, block_valid=valid, workspace=ws_sb)
+        out_b = torch.empty_like(qb_)
+        evg = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        evs_b = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        evf_b = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+
+        def step_b(i):
+            if i >= 0:
+                evg[i][0].record(stream)
+            sa.gather_tokens(q, gather, out=qb_)
+            if i >= 0:
+                evg[i][1].record(stream); evs_b[i][0].record(stream)
+            sa.select(qb_, kb_, w.block, topk_b, block_valid=valid, kept_idx=idx_b, kept_cnt=cnt_b, workspace=ws_sb)
+            if i >= 0:
+                evs_b[i][1].record(stream); evf_b[i][0].record(stream)
+            sa.fwd(qb_, kb_, vb_, idx_b, cnt_b, w.block, out=out_b, workspace=ws_fb, block_valid=valid)
+            if i >= 0:
+                evf_b[i][1].record(stream)
+
+        time_region(step_b, K, args.warmup, stream, dist_on)
+        if sa.read_status(ws_fb) != sa.OK:
+            raise RuntimeError("device status after the brick-order forward")
+        ms_g = statistics.mean(a.elapsed_time(b) for a, b in evg)
+        gbytes = elems * 2 + qb_.numel() * 2
+        # attention mass held by the kept blocks, raster order against brick order, on sampled query rows
+        gen = torch.Generator().manual_seed(11)
+        heads = list(range(min(w.H, 4)))
+        rows = torch.randint(0, w.N, (64,), generator=gen).to(dev)
+        mass_r = mass_b = 0.0
+        for hh in heads:
+            logits = (q[0, hh, rows].float() @ k[0, hh].float().T) / math.sqrt(w.d)
+            pr = torch.softmax(logits, dim=-1)                                         # [rows, N]
+            blk_of_key = torch.arange(w.N, device=dev) // w.block
+            keep_r = torch.zeros((rows.numel(), nb), dtype=torch.bool, device=dev)
+            keep_r.scatter_(1, kept_idx[0, hh, rows // w.block].long(), True)
+            mass_r += float((pr * keep_r[:, blk_of_key]).sum()) / rows.numel()
+            pos = scatter[rows].long()                                                 # the rows' positions in brick order
+            keep_b = torch.zeros((rows.numel(), nbr), dtype=torch.bool, device=dev)
+            keep_b.scatter_(1, idx_b[0, hh, pos // w.block].long(), True)
+            mass_b += float((pr * keep_b[:, scatter.long() // w.block]).sum()) / rows.numel()
+        bricks = {"brick": list(brick), "blocks": nbr, "real_rows_per_block": [int(valid.min()), int(valid.max())], "topk": topk_b,
+                  "gather_ms_per_tensor": ms_g, "gather_GBps": gbytes / (ms_g * 1e-3) / 1e9,
+                  "gather_frac_of_hbm_peak": gbytes / (ms_g * 1e-3) / 1e9 / peaks["hbm"],
+                  "select_ms": statistics.mean(a.elapsed_time(b) for a, b in evs_b),
+                  "fwd_ms": statistics.mean(a.elapsed_time(b) for a, b in evf_b),
+                  "attention_mass_in_kept_blocks": {"raster": mass_r / len(heads), "bricks": mass_b / len(heads),
+                                                    "sample": f"{rows.numel()} query rows of heads {heads[0]}-{heads[-1]}, equal budget ({w.topk} of {nb} / {topk_b} of {nbr} blocks)"}}
+        del qb_, kb_, vb_, out_b, ws_sb, ws_fb
+
     # ---- sparsity sweep (optional): fwd only, lists from sparkattn_select
     sweep = None
     if args.sweep:
@@ -447,7 +510,8 @@ def run_ours(args, w):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": config_dict(w, "bf16"),
             "kept_flops_per_step_per_gpu": flops, "clocks": clocks, "gpu_launches": (4 if pipelined else 3) * K,
-            "kernels": kernels, "roofline": roofline, "fp8": fp8, "compensation": comp, "e2e": e2e, "cpu_baseline": cpu,
+            "kernels": kernels, "roofline": roofline, "fp8": fp8, "compensation": comp, "bricks": bricks, "e2e": e2e,
+            "cpu_baseline": cpu,
         }
         if sweep is not None:
             line["sweep"] = sweep
@@ -469,6 +533,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fp8", action="store_true")
     ap.add_argument("--no-comp", action="store_true", help="skip the compensation-branch leg")
+    ap.add_argument("--no-bricks", action="store_true", help="skip the brick-token-order leg")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

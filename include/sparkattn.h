@@ -81,7 +81,8 @@ const char* sparkattn_status_string(int status);
  * topk), 1 = sparkattn_fwd (pass kmax: for d = 128 with 128-token blocks the
  * forward keeps a range-checked copy of the kept lists and one scale per head
  * behind the status words, about 4 * B * H * nb * (kmax + 1) bytes; 256 bytes
- * otherwise).  Returns 0 for an invalid shape or a non-positive topk / kmax. */
+ * otherwise), 2 = sparkattn_gather_tokens (256).  Returns 0 for an invalid shape or, for 0 and 1, a
+ * non-positive topk / kmax. */
 size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t topk_or_kmax);
 
 /*
@@ -179,6 +180,58 @@ int sparkattn_fwd_window(const sparkattn_shape_t* shape, int32_t dtype, const vo
                          const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                          const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window_frames,
                          void* out_bf16, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Tokens stored brick by brick.  The paper partitions the sequence into
+ * contiguous blocks (Sec. 2) and does not fix the order of the tokens; with
+ * the raster order n = (t*Hg + y)*Wg + x a block is a strip of grid rows.
+ * Here the (T, Hg, Wg) grid is cut into bricks of bt x bh x bw cells with
+ * bt*bh*bw <= block (bricks at the far faces are cut to what the grid holds),
+ * the bricks follow one another in raster order of the brick grid, the cells
+ * of a brick in raster order inside it, and every brick takes one whole block
+ * of the reordered tensors: its cells first, zero padding rows after them.
+ * A block is then a compact box of the video; the reordered tensors have
+ * N' = bricks * block tokens, and block_valid[b] says how many rows of block
+ * b are real.  Padding rows are not keys, do not enter the pooled means of
+ * the selection, and their output rows are to be ignored.
+ *
+ * sparkattn_brick_count : bricks of the layout (host arithmetic; 0 for invalid
+ *                         arguments): the nb of the reordered tensors
+ * sparkattn_brick_layout: grid_host, brick_host HOST int32[3]; block 64 or 128.
+ *     gather_index  out, device int32 [bricks*block]: raster index of the token
+ *                   at each padded position, -1 for padding (gather raster ->
+ *                   bricks); may be NULL
+ *     block_valid   out, device int32 [bricks]; may be NULL
+ *     scatter_index out, device int32 [N]: padded position of raster token n
+ *                   (gather bricks -> raster); may be NULL (not all three)
+ * sparkattn_gather_tokens: out[b,h,i,:] = x[b,h,index[i],:] for i < N of
+ *     dst_shape, one pass over memory; x bf16 with src_shape, out bf16 with
+ *     dst_shape (same B, H, d; the two must not overlap); index device int32
+ *     [dst N]: -1 leaves a zero row, any other value outside [0, src N) leaves
+ *     a zero row and sets SPARKATTN_E_BAD_INDEX in the status word of
+ *     `workspace` (>= sparkattn_workspace_bytes(shape, 2, 0) = 256 bytes,
+ *     256-byte aligned; only the status header is used).
+ * sparkattn_select_padded / sparkattn_fwd_padded: sparkattn_select /
+ *     sparkattn_fwd on reordered tensors (N a multiple of the block size;
+ *     d = 128 with 128-token blocks, else SPARKATTN_E_UNSUPPORTED_SHAPE) with
+ *     block_valid device int32 [nb], every entry in [1, block]: pooled means
+ *     over the real rows of a block, keys beyond block_valid[kb] of a kept
+ *     block get weight 0.  Output rows of padding queries hold finite values
+ *     without meaning.  All other arguments as in the plain calls.
+ */
+int64_t sparkattn_brick_count(const int32_t* grid_host, const int32_t* brick_host);
+int sparkattn_brick_layout(const int32_t* grid_host, const int32_t* brick_host, int32_t block, int32_t* gather_index,
+                           int32_t* block_valid, int32_t* scatter_index, void* cuda_stream);
+int sparkattn_gather_tokens(const sparkattn_shape_t* src_shape, const void* x_bf16, const sparkattn_shape_t* dst_shape,
+                            const int32_t* index, void* out_bf16, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream);
+int sparkattn_select_padded(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                            const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream);
+int sparkattn_fwd_padded(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+                         const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                         const int32_t* kept_cnt, int32_t kmax, const int32_t* block_valid, void* out_bf16, float* lse,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Synchronises the stream and returns the device status word of a workspace
  * (SPARKATTN_OK, SPARKATTN_E_BAD_INDEX or SPARKATTN_E_DEVICE_TIMEOUT). */

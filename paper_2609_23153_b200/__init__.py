@@ -36,7 +36,8 @@ EXPORTS = (
     "sparkattn_quant_fp8", "sparkattn_quant_fp8_per_token", "sparkattn_fwd", "sparkattn_read_status", "sparkattn_arena_bytes",
     "sparkattn_attention_host", "sparkattn_select_noalloc", "sparkattn_select_noalloc_max_bytes",
     "sparkattn_select_noalloc_status", "sparkattn_comp_workspace_bytes", "sparkattn_comp_state",
-    "sparkattn_comp_apply", "sparkattn_select_window", "sparkattn_fwd_window",
+    "sparkattn_comp_apply", "sparkattn_select_window", "sparkattn_fwd_window", "sparkattn_brick_count",
+    "sparkattn_brick_layout", "sparkattn_gather_tokens", "sparkattn_select_padded", "sparkattn_fwd_padded",
 )
 
 
@@ -86,6 +87,16 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_fwd.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.sparkattn_read_status.restype = ctypes.c_int
         L.sparkattn_read_status.argtypes = [vp, vp]
+        L.sparkattn_brick_count.restype = ctypes.c_int64
+        L.sparkattn_brick_count.argtypes = [vp, vp]
+        L.sparkattn_brick_layout.restype = ctypes.c_int
+        L.sparkattn_brick_layout.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.sparkattn_gather_tokens.restype = ctypes.c_int
+        L.sparkattn_gather_tokens.argtypes = [sp, vp, sp, vp, vp, vp, sz, vp]
+        L.sparkattn_select_padded.restype = ctypes.c_int
+        L.sparkattn_select_padded.argtypes = [sp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+        L.sparkattn_fwd_padded.restype = ctypes.c_int
+        L.sparkattn_fwd_padded.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
         L.sparkattn_arena_bytes.restype = sz
         L.sparkattn_arena_bytes.argtypes = [sp, i32, i32]
         L.sparkattn_attention_host.restype = ctypes.c_int
@@ -160,9 +171,11 @@ def read_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = N
 def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, *,
            kept_idx: Optional[torch.Tensor] = None, kept_cnt: Optional[torch.Tensor] = None,
            workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-           frame_tokens: int = 0, window: int = 0) -> Tuple[torch.Tensor, torch.Tensor]:
-    """``sparkattn_select`` (``sparkattn_select_window`` when ``frame_tokens`` > 0): q, k bf16
-    [B,H,N,d] on the device -> (kept_idx int32 [B,H,nb,topk] ascending, kept_cnt int32 [B,H,nb])."""
+           frame_tokens: int = 0, window: int = 0, block_valid: Optional[torch.Tensor] = None,
+           ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_select`` (``sparkattn_select_window`` when ``frame_tokens`` > 0, ``sparkattn_select_padded``
+    with ``block_valid``, device int32 [nb]): q, k bf16 [B,H,N,d] on the device -> (kept_idx int32
+    [B,H,nb,topk] ascending, kept_cnt int32 [B,H,nb])."""
     _same_layout(q, k)
     shape = make_shape(q, block)
     B, H, N, _ = q.shape
@@ -173,6 +186,13 @@ def select(q: torch.Tensor, k: torch.Tensor, block: int, topk: int, *,
         kept_cnt = torch.empty((B, H, nb), dtype=torch.int32, device=q.device)
     if workspace is None:
         workspace = alloc_workspace(shape, 0, topk, q.device)
+    if block_valid is not None:
+        if frame_tokens > 0:
+            raise ValueError("block_valid and a causal window cannot be combined")
+        rc = lib().sparkattn_select_padded(ctypes.byref(shape), _ptr(q), _ptr(k), topk, _ptr(block_valid), _ptr(kept_idx),
+                                           _ptr(kept_cnt), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+        _check(rc, "sparkattn_select_padded")
+        return kept_idx, kept_cnt
     if frame_tokens > 0:
         rc = lib().sparkattn_select_window(ctypes.byref(shape), _ptr(q), _ptr(k), topk, frame_tokens, window,
                                            _ptr(kept_idx), _ptr(kept_cnt), _ptr(workspace), workspace.numel(),
@@ -235,8 +255,10 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tenso
         scales: Optional[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = None,
         softmax_scale: float = 0.0, out: Optional[torch.Tensor] = None, return_lse: bool = False,
         workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
-        check_status: bool = False, frame_tokens: int = 0, window: int = 0):
-    """``sparkattn_fwd`` (``sparkattn_fwd_window`` when ``frame_tokens`` > 0).  bf16 q,k,v, or uint8
+        check_status: bool = False, frame_tokens: int = 0, window: int = 0,
+        block_valid: Optional[torch.Tensor] = None):
+    """``sparkattn_fwd`` (``sparkattn_fwd_window`` when ``frame_tokens`` > 0, ``sparkattn_fwd_padded`` with
+    ``block_valid``, device int32 [nb]).  bf16 q,k,v, or uint8
     E4M3 codes with ``scales=(q_scale, k_scale, v_scale)``.  Returns out bf16 [B,H,N,d] (and lse
     fp32 [B,H,N])."""
     _same_layout(q, k, v)
@@ -250,7 +272,13 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tenso
     if workspace is None:
         workspace = alloc_workspace(shape, 1, kmax, q.device)
     sq, sk, sv = scales if scales is not None else (None, None, None)
-    if frame_tokens > 0:
+    if block_valid is not None:
+        if frame_tokens > 0:
+            raise ValueError("block_valid and a causal window cannot be combined")
+        rc = lib().sparkattn_fwd_padded(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(sq), _ptr(sk), _ptr(sv),
+                                        _ptr(kept_idx), _ptr(kept_cnt), kmax, _ptr(block_valid), _ptr(out), _ptr(lse),
+                                        _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    elif frame_tokens > 0:
         rc = lib().sparkattn_fwd_window(ctypes.byref(shape), dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(sq), _ptr(sk),
                                         _ptr(sv), _ptr(kept_idx), _ptr(kept_cnt), kmax, frame_tokens, window,
                                         _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
@@ -262,6 +290,46 @@ def fwd(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tenso
     if check_status:
         _check(read_status(workspace, stream), "sparkattn_fwd (device status)")
     return (out, lse) if return_lse else out
+
+
+def brick_layout(grid, brick, block: int, device="cuda:0", stream: Optional[torch.cuda.Stream] = None):
+    """``sparkattn_brick_layout``: (gather int32 [bricks * block] with -1 for padding, block_valid int32 [bricks],
+    scatter int32 [N]) for a (T, Hg, Wg) grid cut into (bt, bh, bw) bricks, one block per brick."""
+    g = (ctypes.c_int32 * 3)(*[int(v) for v in grid])
+    b = (ctypes.c_int32 * 3)(*[int(v) for v in brick])
+    bricks = int(lib().sparkattn_brick_count(ctypes.cast(g, ctypes.c_void_p), ctypes.cast(b, ctypes.c_void_p)))
+    if bricks == 0:
+        raise SparkAttnError(E_INVALID_ARG, "sparkattn_brick_count")
+    n = int(grid[0]) * int(grid[1]) * int(grid[2])
+    gather = torch.empty(bricks * block, dtype=torch.int32, device=device)
+    valid = torch.empty(bricks, dtype=torch.int32, device=device)
+    scatter = torch.empty(n, dtype=torch.int32, device=device)
+    rc = lib().sparkattn_brick_layout(ctypes.cast(g, ctypes.c_void_p), ctypes.cast(b, ctypes.c_void_p), block, _ptr(gather),
+                                      _ptr(valid), _ptr(scatter), _stream_ptr(stream))
+    _check(rc, "sparkattn_brick_layout")
+    return gather, valid, scatter
+
+
+def gather_tokens(x: torch.Tensor, index: torch.Tensor, *, out: Optional[torch.Tensor] = None,
+                  workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+                  check_status: bool = False) -> torch.Tensor:
+    """``sparkattn_gather_tokens``: out[b,h,i,:] = x[b,h,index[i],:] (zero row for index -1); x bf16 [B,H,N,d],
+    index int32 [N_out] on the device, out bf16 [B,H,N_out,d]."""
+    blk = 64 if x.shape[-1] == 64 else 128
+    B, H, _, d = x.shape
+    if index.dtype != torch.int32 or index.dim() != 1 or not index.is_contiguous():
+        raise ValueError("index must be a contiguous 1-D int32 tensor")
+    if out is None:
+        out = torch.empty((B, H, index.numel(), d), dtype=x.dtype, device=x.device)
+    src, dst = make_shape(x, blk), make_shape(out, blk)
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=x.device)
+    rc = lib().sparkattn_gather_tokens(ctypes.byref(src), _ptr(x), ctypes.byref(dst), _ptr(index), _ptr(out), _ptr(workspace),
+                                       workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_gather_tokens")
+    if check_status:
+        _check(read_status(workspace, stream), "sparkattn_gather_tokens (device status)")
+    return out
 
 
 def arena_bytes(shape: Shape, dtype: int, topk: int) -> int:

@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparkattn.so")
-SOURCES = ["api.cu", "select.cu", "quant.cu", "fwd.cu", "noalloc.cu", "comp.cu", "fwd_pipe.cu"]
+SOURCES = ["api.cu", "select.cu", "quant.cu", "fwd.cu", "noalloc.cu", "comp.cu", "fwd_pipe.cu", "reorder.cu"]
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",

@@ -58,33 +58,35 @@ size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, 
   if (check_shape(shape) != SPARKATTN_OK) return 0;
   if (which == 0) return select_workspace_bytes(*shape);
   if (which == 1) return topk_or_kmax >= 1 ? fwd_workspace_bytes(*shape, topk_or_kmax) : 0;
+  if (which == 2) return kWorkspaceHeaderBytes;   // sparkattn_gather_tokens: the status header only
   return 0;
 }
 
 namespace {
 int select_impl(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
-                int32_t frame_tokens, int32_t window, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
-                size_t workspace_bytes, void* cuda_stream);
+                int32_t frame_tokens, int32_t window, const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt,
+                void* workspace, size_t workspace_bytes, void* cuda_stream);
 }  // namespace
 
 int sparkattn_select(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
                      int32_t* kept_idx, int32_t* kept_cnt, void* workspace, size_t workspace_bytes,
                      void* cuda_stream) {
-  return select_impl(shape, q_bf16, k_bf16, topk, 0, 0, kept_idx, kept_cnt, workspace, workspace_bytes, cuda_stream);
+  return select_impl(shape, q_bf16, k_bf16, topk, 0, 0, nullptr, kept_idx, kept_cnt, workspace, workspace_bytes,
+                     cuda_stream);
 }
 
 int sparkattn_select_window(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
                             int32_t frame_tokens, int32_t window_frames, int32_t* kept_idx, int32_t* kept_cnt,
                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (frame_tokens < 1 || window_frames < 1 || kept_cnt == nullptr) return SPARKATTN_E_INVALID_ARG;
-  return select_impl(shape, q_bf16, k_bf16, topk, frame_tokens, window_frames, kept_idx, kept_cnt, workspace,
+  return select_impl(shape, q_bf16, k_bf16, topk, frame_tokens, window_frames, nullptr, kept_idx, kept_cnt, workspace,
                      workspace_bytes, cuda_stream);
 }
 
 namespace {
 int select_impl(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
-                int32_t frame_tokens, int32_t window, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
-                size_t workspace_bytes, void* cuda_stream) {
+                int32_t frame_tokens, int32_t window, const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt,
+                void* workspace, size_t workspace_bytes, void* cuda_stream) {
   int rc = check_shape(shape);
   if (rc != SPARKATTN_OK) return rc;
   if (!q_bf16 || !k_bf16 || !kept_idx || !workspace) return SPARKATTN_E_INVALID_ARG;
@@ -95,7 +97,8 @@ int select_impl(const sparkattn_shape_t* shape, const void* q_bf16, const void* 
   if (workspace_bytes < select_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
-  return launch_select(*shape, q_bf16, k_bf16, topk, frame_tokens, window, kept_idx, kept_cnt, workspace, stream);
+  return launch_select(*shape, q_bf16, k_bf16, topk, frame_tokens, window, block_valid, kept_idx, kept_cnt, workspace,
+                       stream);
 }
 }  // namespace
 
@@ -120,15 +123,15 @@ int sparkattn_quant_fp8_per_token(const sparkattn_shape_t* shape, const void* x_
 namespace {
 int fwd_impl(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
              const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
-             const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window, void* out_bf16, float* lse,
-             void* workspace, size_t workspace_bytes, void* cuda_stream);
+             const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window, const int32_t* block_valid,
+             void* out_bf16, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);
 }  // namespace
 
 int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
                   const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                   const int32_t* kept_cnt, int32_t kmax, void* out_bf16, float* lse, void* workspace,
                   size_t workspace_bytes, void* cuda_stream) {
-  return fwd_impl(shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, 0, 0, out_bf16, lse,
+  return fwd_impl(shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, 0, 0, nullptr, out_bf16, lse,
                   workspace, workspace_bytes, cuda_stream);
 }
 
@@ -138,14 +141,14 @@ int sparkattn_fwd_window(const sparkattn_shape_t* shape, int32_t dtype, const vo
                          void* out_bf16, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   if (frame_tokens < 1 || window_frames < 1) return SPARKATTN_E_INVALID_ARG;
   return fwd_impl(shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens,
-                  window_frames, out_bf16, lse, workspace, workspace_bytes, cuda_stream);
+                  window_frames, nullptr, out_bf16, lse, workspace, workspace_bytes, cuda_stream);
 }
 
 namespace {
 int fwd_impl(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
              const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
-             const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window, void* out_bf16, float* lse,
-             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+             const int32_t* kept_cnt, int32_t kmax, int32_t frame_tokens, int32_t window, const int32_t* block_valid,
+             void* out_bf16, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   int rc = check_shape(shape);
   if (rc != SPARKATTN_OK) return rc;
   if (dtype != SPARKATTN_BF16 && dtype != SPARKATTN_FP8_E4M3) return SPARKATTN_E_INVALID_ARG;
@@ -160,7 +163,7 @@ int fwd_impl(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const
     return SPARKATTN_E_MISALIGNED;
   if (workspace_bytes < fwd_workspace_bytes(*shape, kmax)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   return launch_fwd(*shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
-                    out_bf16, lse, workspace, static_cast<cudaStream_t>(cuda_stream));
+                    block_valid, out_bf16, lse, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 }  // namespace
 
@@ -215,6 +218,75 @@ int sparkattn_comp_apply(const sparkattn_shape_t* shape, const void* q_bf16, con
   if (workspace_bytes < comp_workspace_bytes(*shape, grid_host, false)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
   return launch_comp_apply(*shape, q_bf16, pq_bf16, grid_host, rope_axis_host, rope_freq_host, state, gate,
                            o_sparse_bf16, out_bf16, eps, workspace, static_cast<cudaStream_t>(cuda_stream));
+}
+
+namespace {
+// bricks padded to whole blocks: every block is whole, so N is a multiple of the block size
+int check_padded(const sparkattn_shape_t* shape, const int32_t* block_valid) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (block_valid == nullptr) return SPARKATTN_E_INVALID_ARG;
+  if (shape->N % shape->block != 0) return SPARKATTN_E_INVALID_ARG;
+  if (shape->d != 128 || shape->block != 128) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  return SPARKATTN_OK;
+}
+}  // namespace
+
+int64_t sparkattn_brick_count(const int32_t* grid_host, const int32_t* brick_host) {
+  if (!grid_host || !brick_host) return 0;
+  int64_t n = 1;
+  for (int a = 0; a < 3; ++a) {
+    if (grid_host[a] < 1 || brick_host[a] < 1) return 0;
+    n *= (grid_host[a] + brick_host[a] - 1) / brick_host[a];
+  }
+  return n;
+}
+
+int sparkattn_brick_layout(const int32_t* grid_host, const int32_t* brick_host, int32_t block, int32_t* gather_index,
+                           int32_t* block_valid, int32_t* scatter_index, void* cuda_stream) {
+  const int64_t bricks = sparkattn_brick_count(grid_host, brick_host);
+  if (bricks == 0 || (block != 64 && block != 128) || (!gather_index && !block_valid && !scatter_index))
+    return SPARKATTN_E_INVALID_ARG;
+  if ((int64_t)brick_host[0] * brick_host[1] * brick_host[2] > block) return SPARKATTN_E_INVALID_ARG;
+  const int64_t n = (int64_t)grid_host[0] * grid_host[1] * grid_host[2];
+  if (n > 0x7fffffffLL || bricks * block > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  return launch_brick_layout(grid_host, brick_host, block, gather_index, block_valid, scatter_index,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sparkattn_gather_tokens(const sparkattn_shape_t* src_shape, const void* x_bf16, const sparkattn_shape_t* dst_shape,
+                            const int32_t* index, void* out_bf16, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream) {
+  int rc = check_shape(src_shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if ((rc = check_shape(dst_shape)) != SPARKATTN_OK) return rc;
+  if (src_shape->B != dst_shape->B || src_shape->H != dst_shape->H || src_shape->d != dst_shape->d)
+    return SPARKATTN_E_INVALID_ARG;
+  if (!x_bf16 || !index || !out_bf16 || !workspace || x_bf16 == out_bf16) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned16(x_bf16) || !aligned16(out_bf16) || !aligned256(workspace)) return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < (size_t)kWorkspaceHeaderBytes) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  return launch_gather_tokens(*src_shape, x_bf16, *dst_shape, index, out_bf16, workspace, stream);
+}
+
+int sparkattn_select_padded(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, int32_t topk,
+                            const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+  const int rc = check_padded(shape, block_valid);
+  if (rc != SPARKATTN_OK) return rc;
+  return select_impl(shape, q_bf16, k_bf16, topk, 0, 0, block_valid, kept_idx, kept_cnt, workspace, workspace_bytes,
+                     cuda_stream);
+}
+
+int sparkattn_fwd_padded(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
+                         const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                         const int32_t* kept_cnt, int32_t kmax, const int32_t* block_valid, void* out_bf16, float* lse,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  const int rc = check_padded(shape, block_valid);
+  if (rc != SPARKATTN_OK) return rc;
+  return fwd_impl(shape, dtype, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, 0, 0, block_valid, out_bf16,
+                  lse, workspace, workspace_bytes, cuda_stream);
 }
 
 int sparkattn_read_status(void* workspace, void* cuda_stream) {

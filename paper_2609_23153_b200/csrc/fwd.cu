@@ -522,14 +522,15 @@ static int launch_fwd_t(const sparkattn_shape_t& s, const CUtensorMap& mq, const
 
 int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void* k, const void* v,
                const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
-               const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse, void* workspace,
-               cudaStream_t stream) {
+               const int32_t* kept_cnt, int kmax, int frame_tokens, int window, const int32_t* block_valid, void* out,
+               float* lse, void* workspace, cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
 #ifndef SPARKATTN_FWD_NO_PIPE
-  if (fwd_pipe_supported(s))
-    return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window, out,
-                           lse, workspace, stream);
+  if (fwd_pipe_supported(s) && (block_valid == nullptr || s.block == 128))
+    return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
+                           block_valid, out, lse, workspace, stream);
 #endif
+  if (block_valid != nullptr) return SPARKATTN_E_UNSUPPORTED_SHAPE;   // padded bricks: d = 128 with 128-token blocks only
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;
   int rc;

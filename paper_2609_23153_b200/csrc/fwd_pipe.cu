@@ -62,6 +62,7 @@ struct PipeParams {
   int nbq;                     // work items per (batch, head): query blocks, or pairs of 64-token query blocks
   int lstride;                 // list entries per item in clean_list
   int frame_tokens, window;    // causal frame window (0 = none): key frame in (query frame - window, query frame]
+  const int32_t* blk_valid;    // [nb] real tokens per block (bricks padded to whole blocks), or NULL; not with PAIR
   int64_t stride_b, stride_h, stride_n;
   float scale_log2;
 };
@@ -531,6 +532,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       int e_cur0 = ld_ent(n0, 0), e_cur1 = PAIR ? ld_ent(n0, 1) : 0;
       int e_nx0 = ld_ent(n0 + 2, 0), e_nx1 = PAIR ? ld_ent(n0 + 2, 1) : 0;
       float ks_cur0 = 1.0f, vs_cur0 = 1.0f, ks_cur1 = 1.0f, vs_cur1 = 1.0f;
+      int bv_cur = kPBLK;                          // real tokens of the tile's key block (bricks padded to whole blocks)
+      if constexpr (!PAIR) {
+        if (p.blk_valid != nullptr) bv_cur = __ldg(p.blk_valid + e_cur0);
+      }
       if constexpr (FP8) {
         ks_cur0 = __ldg(ksc + (e_cur0 & 0x3fffffff));
         vs_cur0 = __ldg(vsc + (e_cur0 & 0x3fffffff));
@@ -546,6 +551,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // the tile's key block(s); PAIR: two 64-token blocks, each with a flag per query block of the pair
         const int e0 = e_cur0, e1 = e_cur1;
         const float ks0 = ks_cur0, vs0 = vs_cur0, ks1 = ks_cur1, vs1 = vs_cur1;
+        const int bv0 = bv_cur;
+        if constexpr (!PAIR) {
+          if (p.blk_valid != nullptr) bv_cur = __ldg(p.blk_valid + e_nx0);
+        }
         // next tile of this warpgroup: its scales (its entries arrived a tile ago), and the entries of the one after
         if constexpr (FP8) {
           ks_cur0 = __ldg(ksc + (e_nx0 & 0x3fffffff));
@@ -581,7 +590,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
         // this row's valid columns: [c_lo, c_hi) of the tile, or (PAIR) [c_lo, c_hi) of its first 64 and
         // [c_lo1, c_hi1) of its second 64 columns (empty when the block is not in this query block's list)
-        const int c_lo = klo - kb * kKeyBlk, c_hi = PAIR ? (mem0 ? min(khi - kb * 64, 64) : 0) : khi - kb * kPBLK;
+        const int c_lo = klo - kb * kKeyBlk, c_hi = PAIR ? (mem0 ? min(khi - kb * 64, 64) : 0) : min(khi - kb * kPBLK, bv0);
         const int c_lo1 = klo - kb1 * 64, c_hi1 = mem1 ? min(khi - kb1 * 64, 64) : 0;
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt >> 1) & 1, s_abort, p.status, 4));
         if (!ok) break;
@@ -601,10 +610,16 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
               if ((WINDOW && i < c_lo1) || i >= c_hi1) sr[64 + i] = 0xff800000u;
             }
           }
-        } else if ((WINDOW && c_lo > 0) || c_hi < kPBLK) {   // ragged last key block / keys outside the causal window get weight 0
+        } else if ((WINDOW && c_lo > 0) || c_hi < kPBLK) {   // ragged last key block / padding rows of a brick / keys outside the causal window get weight 0
+          if (!WINDOW && c_hi >= kPBLK - 32) {                // a short tail (every tile of a padded brick layout): 32 tests, not 128
 #pragma unroll
-          for (int i = 0; i < kPBLK; ++i)
-            if ((WINDOW && i < c_lo) || i >= c_hi) sr[i] = 0xff800000u;
+            for (int i = kPBLK - 32; i < kPBLK; ++i)
+              if (i >= c_hi) sr[i] = 0xff800000u;
+          } else {
+#pragma unroll
+            for (int i = 0; i < kPBLK; ++i)
+              if ((WINDOW && i < c_lo) || i >= c_hi) sr[i] = 0xff800000u;
+          }
         }
         float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
         float mx2 = __uint_as_float(sr[2]), mx3 = __uint_as_float(sr[3]);
@@ -875,8 +890,8 @@ size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
 
 int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
                     const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
-                    const int32_t* kept_cnt, int kmax, int frame_tokens, int window, void* out, float* lse,
-                    void* workspace, cudaStream_t stream) {
+                    const int32_t* kept_cnt, int kmax, int frame_tokens, int window, const int32_t* block_valid,
+                    void* out, float* lse, void* workspace, cudaStream_t stream) {
   CUtensorMap mq, mk, mv, mo;
   int rc;
   const int elt = fp8 ? 1 : 2;
@@ -904,6 +919,7 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   prm.status = static_cast<int32_t*>(workspace);
   prm.H = s.H; prm.N = s.N; prm.nb = nb; prm.items = (int)items; prm.nbq = nbq; prm.lstride = lstride;
   prm.frame_tokens = frame_tokens; prm.window = window;
+  prm.blk_valid = block_valid;
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
   const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
   prm.scale_log2 = sc * 1.4426950408889634f;

@@ -39,7 +39,8 @@ template <int D>
 __global__ void __launch_bounds__(kPoolThreads)
 pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k, float* __restrict__ pq,
             float* __restrict__ pkT, int H, int N, int blk_size, int nb, int nbp, int64_t stride_b,
-            int64_t stride_h, int64_t stride_n, int64_t n_items /* B*H*nb */) {
+            int64_t stride_h, int64_t stride_n, int64_t n_items /* B*H*nb */,
+            const int32_t* __restrict__ block_valid /* [nb] real tokens per block, or NULL */) {
   constexpr int VEC = D / 32;  // channels per lane: 4 (8-byte loads) or 2 (4-byte loads)
   const int lane = threadIdx.x & 31;
   const int64_t gw = (int64_t)blockIdx.x * (kPoolThreads / 32) + (threadIdx.x >> 5);
@@ -50,7 +51,8 @@ pool_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict
   const int64_t bh = item / nb;
   const int h = (int)(bh % H), b = (int)(bh / H);
   const int row0 = blk * blk_size;
-  const int nvalid = min(blk_size, N - row0);
+  int nvalid = min(blk_size, N - row0);
+  if (block_valid != nullptr) nvalid = max(1, min(nvalid, __ldg(block_valid + blk)));   // bricks padded to whole blocks
   const __nv_bfloat16* src = (is_k ? k : q) + b * stride_b + h * stride_h + (int64_t)row0 * stride_n + lane * VEC;
 
   float sum[VEC];
@@ -395,7 +397,7 @@ static int launch_topk(const float* pq, const float* pkT, int32_t* kept_idx, int
 }
 
 int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int frame_tokens, int window,
-                  int32_t* kept_idx, int32_t* kept_cnt, void* workspace, cudaStream_t stream) {
+                  const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt, void* workspace, cudaStream_t stream) {
   const int nb = (s.N + s.block - 1) / s.block;
   const int nbp = round_up(nb, 32);
   if (nb > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
@@ -414,12 +416,12 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
   int rc;
   if (s.d == 128) {
     pool_kernel<128><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
-        qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
+        qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items, block_valid);
     rc = rows16 ? launch_topk<128, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
                 : launch_topk<128, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
   } else if (s.d == 64) {
     pool_kernel<64><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
-        qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items);
+        qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items, block_valid);
     rc = rows16 ? launch_topk<64, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
                 : launch_topk<64, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
   } else {

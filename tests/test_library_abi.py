@@ -57,7 +57,8 @@ def test_workspace_sizes(lib):
     nb = 32
     assert sa.workspace_bytes(s, 1, 16) == 256
     assert sa.workspace_bytes(s, 0, 16) == 256 + 2 * nb * 64 * 4 + 2 * 64 * 32 * 4
-    assert sa.workspace_bytes(s, 2, 16) == 0
+    assert sa.workspace_bytes(s, 2, 0) == 256          # the gather call: status header only
+    assert sa.workspace_bytes(s, 3, 16) == 0
     bad = _shape(d=96)
     assert sa.workspace_bytes(bad, 0, 16) == 0
     assert sa.arena_bytes(s, sa.BF16, 16) > 4 * 2 * 2048 * 64 * 2
@@ -164,3 +165,43 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(sa, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         sa.lib()
+
+
+def test_padded_brick_entry_points_validate_on_the_host(lib):
+    s128 = _shape(d=128, block=128, N=4096)
+    s64 = _shape()
+    fake = ctypes.c_void_p(0x1000)
+    null = ctypes.c_void_p(0)
+    st = ctypes.c_void_p(0)
+    grid = (ctypes.c_int32 * 3)(21, 45, 80)
+    brick = (ctypes.c_int32 * 3)(3, 5, 8)
+    gp, bp = ctypes.cast(grid, ctypes.c_void_p), ctypes.cast(brick, ctypes.c_void_p)
+    lib.sparkattn_brick_count.restype = ctypes.c_int64
+    assert lib.sparkattn_brick_count(gp, bp) == 7 * 9 * 10
+    assert lib.sparkattn_brick_count(null, bp) == 0
+    zero = (ctypes.c_int32 * 3)(3, 0, 8)
+    assert lib.sparkattn_brick_count(gp, ctypes.cast(zero, ctypes.c_void_p)) == 0
+    big = (ctypes.c_int32 * 3)(3, 9, 8)                                   # 216 cells > 128
+    assert lib.sparkattn_brick_layout(gp, ctypes.cast(big, ctypes.c_void_p), 128, fake, fake, fake, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_brick_layout(gp, bp, 100, fake, fake, fake, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_brick_layout(gp, bp, 128, null, null, null, st) == sa.E_INVALID_ARG
+    # select / fwd on padded bricks: block_valid required, N a multiple of the block, d = 128 with 128-token blocks
+    r = lib.sparkattn_select_padded(ctypes.byref(s128), fake, fake, 4, null, fake, null, fake, 1 << 24, st)
+    assert r == sa.E_INVALID_ARG
+    ragged = _shape(d=128, block=128, N=4000)
+    r = lib.sparkattn_select_padded(ctypes.byref(ragged), fake, fake, 4, fake, fake, null, fake, 1 << 24, st)
+    assert r == sa.E_INVALID_ARG
+    r = lib.sparkattn_select_padded(ctypes.byref(s64), fake, fake, 4, fake, fake, null, fake, 1 << 24, st)
+    assert r == sa.E_UNSUPPORTED_SHAPE
+    r = lib.sparkattn_fwd_padded(ctypes.byref(s64), sa.BF16, fake, fake, fake, null, null, null, fake, fake, 4, fake, fake,
+                                 null, fake, 1 << 24, st)
+    assert r == sa.E_UNSUPPORTED_SHAPE
+    r = lib.sparkattn_fwd_padded(ctypes.byref(s128), sa.BF16, fake, fake, fake, null, null, null, fake, fake, 4, null, fake,
+                                 null, fake, 1 << 24, st)
+    assert r == sa.E_INVALID_ARG
+    # gather: shapes must agree in B, H, d; buffers must differ; workspace holds the status header
+    other = _shape(d=128, block=128, N=4096)
+    other.H = s128.H + 1
+    assert lib.sparkattn_gather_tokens(ctypes.byref(s128), fake, ctypes.byref(other), fake, ctypes.c_void_p(0x2000), fake, 256, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_gather_tokens(ctypes.byref(s128), fake, ctypes.byref(s128), fake, fake, fake, 256, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_gather_tokens(ctypes.byref(s128), fake, ctypes.byref(s128), fake, ctypes.c_void_p(0x2000), fake, 16, st) == sa.E_WORKSPACE_TOO_SMALL
