@@ -13,9 +13,10 @@
 //                        it are counted by brick index, so no prefix sums are needed); writes the
 //                        gather index (raster token at each padded position; padding keeps the -1 a
 //                        memset put there), the scatter index and the per-brick token count.
-//   gather_tokens_kernel out[b,h,i,:] = x[b,h,index[i],:] (zero row for index -1); rows move as
-//                        16-byte pieces, 8 in flight per thread; bound by HBM (2 bytes read + 2
-//                        written per element).
+//   gather_tokens_kernel out[b,h,i,:] = x[b,h,index[i],:] (zero row for index -1); a CTA moves 128
+//                        (d = 128) or 256 (d = 64) consecutive rows of one (batch, head) as 16-byte
+//                        pieces, 8 in flight per thread; bound by HBM (2 bytes read + 2 written per
+//                        element).
 #include "common.cuh"
 #include "launch.h"
 
@@ -41,36 +42,36 @@ brick_layout_kernel(int T, int Hg, int Wg, int bt, int bh, int bw, int block, in
 
 constexpr int kGatherThreads = 256, kGatherUnroll = 8;
 
-template <int PIECES>   // 16-byte pieces per token row
+// One CTA moves kGatherUnroll * 256 / PIECES consecutive token rows of one (batch, head): a thread keeps its
+// 16-byte column of the row and steps over the rows, all loads issued before the first store.
+template <int PIECES>   // 16-byte pieces per token row: 16 (d = 128) or 8 (d = 64)
 __global__ void __launch_bounds__(kGatherThreads)
 gather_tokens_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ index, uint4* __restrict__ out, int H,
                      int n_src, int n_dst, int64_t src_b, int64_t src_h, int64_t src_n, int64_t dst_b, int64_t dst_h,
-                     int64_t dst_n /* strides in 16-byte pieces */, int64_t total, int32_t* __restrict__ status) {
-  const int64_t step = (int64_t)gridDim.x * kGatherThreads;
-  int64_t id = (int64_t)blockIdx.x * kGatherThreads + threadIdx.x;
-  for (; id < total; id += step * kGatherUnroll) {
-    uint4 v[kGatherUnroll];
-    int64_t dst[kGatherUnroll];
+                     int64_t dst_n /* strides in 16-byte pieces */, int chunks_per_bh, int32_t* __restrict__ status) {
+  constexpr int kRowsPerPass = kGatherThreads / PIECES;
+  constexpr int kRowsPerCta = kRowsPerPass * kGatherUnroll;
+  const int bh = blockIdx.x / chunks_per_bh;
+  const int row0 = (blockIdx.x - bh * chunks_per_bh) * kRowsPerCta + threadIdx.x / PIECES;
+  const int piece = threadIdx.x % PIECES;
+  const int b = bh / H, h = bh - b * H;
+  const uint4* xs = x + b * src_b + h * src_h + piece;
+  uint4* os = out + b * dst_b + h * dst_h + piece;
+  uint4 v[kGatherUnroll];
 #pragma unroll
-    for (int u = 0; u < kGatherUnroll; ++u) {
-      const int64_t e = id + u * step;
-      dst[u] = -1;
-      v[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (e < total) {
-        const int piece = (int)(e % PIECES);
-        const int64_t row = e / PIECES;
-        const int i = (int)(row % n_dst);
-        const int64_t bh = row / n_dst;
-        const int64_t b = bh / H, h = bh % H;
-        const int src = __ldg(index + i);
-        dst[u] = b * dst_b + h * dst_h + (int64_t)i * dst_n + piece;
-        if ((unsigned)src < (unsigned)n_src) v[u] = __ldg(x + b * src_b + h * src_h + (int64_t)src * src_n + piece);
-        else if (src != -1) report_status(status, SPARKATTN_E_BAD_INDEX, src);     // the row is written as zeros
-      }
+  for (int u = 0; u < kGatherUnroll; ++u) {
+    const int i = row0 + u * kRowsPerPass;
+    v[u] = make_uint4(0u, 0u, 0u, 0u);
+    if (i < n_dst) {
+      const int src = __ldg(index + i);
+      if ((unsigned)src < (unsigned)n_src) v[u] = __ldg(xs + (int64_t)src * src_n);
+      else if (src != -1) report_status(status, SPARKATTN_E_BAD_INDEX, src);     // the row is written as zeros
     }
+  }
 #pragma unroll
-    for (int u = 0; u < kGatherUnroll; ++u)
-      if (dst[u] >= 0) out[dst[u]] = v[u];
+  for (int u = 0; u < kGatherUnroll; ++u) {
+    const int i = row0 + u * kRowsPerPass;
+    if (i < n_dst) os[(int64_t)i * dst_n] = v[u];
   }
 }
 
@@ -90,21 +91,21 @@ int launch_brick_layout(const int32_t* grid, const int32_t* brick, int block, in
 int launch_gather_tokens(const sparkattn_shape_t& src, const void* x, const sparkattn_shape_t& dst, const int32_t* index,
                          void* out, void* workspace, cudaStream_t stream) {
   const int pieces = dst.d * 2 / 16;
-  const int64_t total = (int64_t)dst.B * dst.H * dst.N * pieces;
-  // a few waves of CTAs, each thread with kGatherUnroll pieces in flight per trip
-  const int64_t want = (total + (int64_t)kGatherThreads * kGatherUnroll - 1) / ((int64_t)kGatherThreads * kGatherUnroll);
-  const unsigned ctas = (unsigned)max((int64_t)1, min(want, (int64_t)148 * 32));
+  const int rows_per_cta = kGatherThreads / pieces * kGatherUnroll;
+  const int chunks = (dst.N + rows_per_cta - 1) / rows_per_cta;
+  const int64_t ctas = (int64_t)dst.B * dst.H * chunks;
+  if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   int32_t* status = static_cast<int32_t*>(workspace);
   const uint4* xs = static_cast<const uint4*>(x);
   uint4* os = static_cast<uint4*>(out);
   if (dst.d == 128)
-    gather_tokens_kernel<16><<<ctas, kGatherThreads, 0, stream>>>(xs, index, os, dst.H, src.N, dst.N, src.stride_b / 8,
-                                                                src.stride_h / 8, src.stride_n / 8, dst.stride_b / 8,
-                                                                dst.stride_h / 8, dst.stride_n / 8, total, status);
+    gather_tokens_kernel<16><<<(unsigned)ctas, kGatherThreads, 0, stream>>>(
+        xs, index, os, dst.H, src.N, dst.N, src.stride_b / 8, src.stride_h / 8, src.stride_n / 8, dst.stride_b / 8,
+        dst.stride_h / 8, dst.stride_n / 8, chunks, status);
   else
-    gather_tokens_kernel<8><<<ctas, kGatherThreads, 0, stream>>>(xs, index, os, dst.H, src.N, dst.N, src.stride_b / 8,
-                                                               src.stride_h / 8, src.stride_n / 8, dst.stride_b / 8,
-                                                               dst.stride_h / 8, dst.stride_n / 8, total, status);
+    gather_tokens_kernel<8><<<(unsigned)ctas, kGatherThreads, 0, stream>>>(
+        xs, index, os, dst.H, src.N, dst.N, src.stride_b / 8, src.stride_h / 8, src.stride_n / 8, dst.stride_b / 8,
+        dst.stride_h / 8, dst.stride_n / 8, chunks, status);
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
