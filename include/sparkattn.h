@@ -213,7 +213,7 @@ int sparkattn_fwd_window(const sparkattn_shape_t* shape, int32_t dtype, const vo
  *     256-byte aligned; only the status header is used).
  * sparkattn_select_padded / sparkattn_fwd_padded: sparkattn_select /
  *     sparkattn_fwd on reordered tensors (N a multiple of the block size;
- *     d = 128 with 128-token blocks, else SPARKATTN_E_UNSUPPORTED_SHAPE) with
+ *     d = 128 with 128- or 64-token blocks, else SPARKATTN_E_UNSUPPORTED_SHAPE) with
  *     block_valid device int32 [nb], every entry in [1, block]: pooled means
  *     over the real rows of a block, keys beyond block_valid[kb] of a kept
  *     block get weight 0.  Output rows of padding queries hold finite values

@@ -227,7 +227,7 @@ int check_padded(const sparkattn_shape_t* shape, const int32_t* block_valid) {
   if (rc != SPARKATTN_OK) return rc;
   if (block_valid == nullptr) return SPARKATTN_E_INVALID_ARG;
   if (shape->N % shape->block != 0) return SPARKATTN_E_INVALID_ARG;
-  if (shape->d != 128 || shape->block != 128) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (shape->d != 128) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   return SPARKATTN_OK;
 }
 }  // namespace

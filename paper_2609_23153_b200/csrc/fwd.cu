@@ -526,11 +526,11 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                float* lse, void* workspace, cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
 #ifndef SPARKATTN_FWD_NO_PIPE
-  if (fwd_pipe_supported(s) && (block_valid == nullptr || s.block == 128))
+  if (fwd_pipe_supported(s))
     return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
                            block_valid, out, lse, workspace, stream);
 #endif
-  if (block_valid != nullptr) return SPARKATTN_E_UNSUPPORTED_SHAPE;   // padded bricks: d = 128 with 128-token blocks only
+  if (block_valid != nullptr) return SPARKATTN_E_UNSUPPORTED_SHAPE;   // padded bricks: d = 128 (the pipelined kernel) only
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;
   int rc;

@@ -62,7 +62,7 @@ struct PipeParams {
   int nbq;                     // work items per (batch, head): query blocks, or pairs of 64-token query blocks
   int lstride;                 // list entries per item in clean_list
   int frame_tokens, window;    // causal frame window (0 = none): key frame in (query frame - window, query frame]
-  const int32_t* blk_valid;    // [nb] real tokens per block (bricks padded to whole blocks), or NULL; not with PAIR
+  const int32_t* blk_valid;    // [nb] real tokens per block (bricks padded to whole blocks), or NULL
   int64_t stride_b, stride_h, stride_n;
   float scale_log2;
 };
@@ -532,9 +532,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       int e_cur0 = ld_ent(n0, 0), e_cur1 = PAIR ? ld_ent(n0, 1) : 0;
       int e_nx0 = ld_ent(n0 + 2, 0), e_nx1 = PAIR ? ld_ent(n0 + 2, 1) : 0;
       float ks_cur0 = 1.0f, vs_cur0 = 1.0f, ks_cur1 = 1.0f, vs_cur1 = 1.0f;
-      int bv_cur = kPBLK;                          // real tokens of the tile's key block (bricks padded to whole blocks)
-      if constexpr (!PAIR) {
-        if (p.blk_valid != nullptr) bv_cur = __ldg(p.blk_valid + e_cur0);
+      int bv_cur = kKeyBlk, bv_cur1 = kKeyBlk;     // real tokens of the tile's key block(s) (bricks padded to whole blocks)
+      if (p.blk_valid != nullptr) {
+        bv_cur = __ldg(p.blk_valid + (e_cur0 & 0x3fffffff));
+        if constexpr (PAIR) bv_cur1 = __ldg(p.blk_valid + (e_cur1 & 0x3fffffff));
       }
       if constexpr (FP8) {
         ks_cur0 = __ldg(ksc + (e_cur0 & 0x3fffffff));
@@ -551,9 +552,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // the tile's key block(s); PAIR: two 64-token blocks, each with a flag per query block of the pair
         const int e0 = e_cur0, e1 = e_cur1;
         const float ks0 = ks_cur0, vs0 = vs_cur0, ks1 = ks_cur1, vs1 = vs_cur1;
-        const int bv0 = bv_cur;
-        if constexpr (!PAIR) {
-          if (p.blk_valid != nullptr) bv_cur = __ldg(p.blk_valid + e_nx0);
+        const int bv0 = bv_cur, bv1 = bv_cur1;
+        if (p.blk_valid != nullptr) {
+          bv_cur = __ldg(p.blk_valid + (e_nx0 & 0x3fffffff));
+          if constexpr (PAIR) bv_cur1 = __ldg(p.blk_valid + (e_nx1 & 0x3fffffff));
         }
         // next tile of this warpgroup: its scales (its entries arrived a tile ago), and the entries of the one after
         if constexpr (FP8) {
@@ -590,8 +592,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
         // this row's valid columns: [c_lo, c_hi) of the tile, or (PAIR) [c_lo, c_hi) of its first 64 and
         // [c_lo1, c_hi1) of its second 64 columns (empty when the block is not in this query block's list)
-        const int c_lo = klo - kb * kKeyBlk, c_hi = PAIR ? (mem0 ? min(khi - kb * 64, 64) : 0) : min(khi - kb * kPBLK, bv0);
-        const int c_lo1 = klo - kb1 * 64, c_hi1 = mem1 ? min(khi - kb1 * 64, 64) : 0;
+        const int c_lo = klo - kb * kKeyBlk, c_hi = PAIR ? (mem0 ? min(khi - kb * 64, bv0) : 0) : min(khi - kb * kPBLK, bv0);
+        const int c_lo1 = klo - kb1 * 64, c_hi1 = mem1 ? min(khi - kb1 * 64, bv1) : 0;
         ok = __all_sync(0xffffffffu, mbar_wait(bar_s_full + buf, (tt >> 1) & 1, s_abort, p.status, 4));
         if (!ok) break;
         tc_fence_after();

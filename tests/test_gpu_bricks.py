@@ -55,13 +55,15 @@ def _to_bricks(x, gather):
     return sa.gather_tokens(x, gather)
 
 
-def test_select_and_fwd_with_block_valid_match_oracle():
-    grid, brick, block = (6, 10, 23), (2, 4, 16), 128           # bricks of 128, 92 (x tail), 64 (y tail) ... cells
+@pytest.mark.parametrize("grid,brick,block", [((6, 10, 23), (2, 4, 16), 128),     # bricks of 128, 92 (x tail), 64 (y tail) ... cells
+                                              ((6, 10, 23), (2, 4, 8), 64),        # 64-token blocks: pairs of query blocks over merged lists
+                                              ((5, 9, 21), (1, 3, 20), 64)])       # an odd number of bricks, 60 or 3 real rows
+def test_select_and_fwd_with_block_valid_match_oracle(grid, brick, block):
     H, d, topk = 3, 128, 5
     w = workloads.small_structured(H, d, grid, block, 0.0, cfg_id=71)
     q, k, v = (t.to(DEV) for t in workloads.structured_qkv(w))
     gather, valid, scatter = sa.brick_layout(grid, brick, block)
-    assert int(valid.min()) < block and int(valid.max()) == block
+    assert int(valid.min()) < block
     qb, kb, vb = (_to_bricks(t, gather) for t in (q, k, v))
     nbr = valid.numel()
     idx, cnt = sa.select(qb, kb, block, topk, block_valid=valid)

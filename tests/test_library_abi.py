@@ -185,7 +185,7 @@ def test_padded_brick_entry_points_validate_on_the_host(lib):
     assert lib.sparkattn_brick_layout(gp, ctypes.cast(big, ctypes.c_void_p), 128, fake, fake, fake, st) == sa.E_INVALID_ARG
     assert lib.sparkattn_brick_layout(gp, bp, 100, fake, fake, fake, st) == sa.E_INVALID_ARG
     assert lib.sparkattn_brick_layout(gp, bp, 128, null, null, null, st) == sa.E_INVALID_ARG
-    # select / fwd on padded bricks: block_valid required, N a multiple of the block, d = 128 with 128-token blocks
+    # select / fwd on padded bricks: block_valid required, N a multiple of the block, d = 128
     r = lib.sparkattn_select_padded(ctypes.byref(s128), fake, fake, 4, null, fake, null, fake, 1 << 24, st)
     assert r == sa.E_INVALID_ARG
     ragged = _shape(d=128, block=128, N=4000)
