@@ -412,7 +412,8 @@ int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int 
   if (pool_ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   // 16 query blocks per CTA while two CTAs' score rows fit one SM's shared memory and the grid still
   // fills the device several times over (small problems are bound by the latency of one CTA), else 8
-  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u && bh * ((nb + 15) / 16) >= 6 * 148;
+  constexpr int kNumSMs = 148;   // B200; another count only moves the point where the CTAs get smaller
+  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u && bh * ((nb + 15) / 16) >= 6 * kNumSMs;
   int rc;
   if (s.d == 128) {
     pool_kernel<128><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
