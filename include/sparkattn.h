@@ -151,7 +151,11 @@ int sparkattn_quant_fp8_per_token(const sparkattn_shape_t* shape, const void* x_
  * lse        : out, fp32 [B,H,N] contiguous (natural log); may be NULL
  * workspace  : >= sparkattn_workspace_bytes(shape, 1, kmax) bytes, 256-byte aligned
  * Accumulation, row maximum and row sum are fp32; P is rounded to the input
- * dtype for the second product.
+ * dtype for the second product.  The kept blocks of a list may come in any
+ * order and are processed in an order of the library's choosing (the query
+ * block's own key block first); the same inputs always give the same bits.
+ * Out-of-range entries of a list are skipped and reported through the status
+ * word of the workspace (SPARKATTN_E_BAD_INDEX).
  */
 int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, const void* k, const void* v,
                   const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
