@@ -2,7 +2,8 @@
 """Benchmark of the block-sparse attention path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload wan14b|wan1p3b] [--no-e2e] [--no-cpu] [--sweep]
+                    [--workload wan14b|wan1p3b] [--shard batch|heads] [--no-e2e] [--no-cpu]
+                    [--no-sweep] [--no-sustained] [--no-second-workload]
 
 One "step" is one pass of the whole path over one batch of synthetic input
 resident in HBM: block selection (pool + top-k kernels) followed by the
@@ -17,6 +18,15 @@ the CPU oracle timed on a bounded sample.
 With N > 1 (torchrun, one rank per GPU) every rank runs the same-shaped
 problem on its own seeded batch: batches are independent, so there is no
 data-path collective; the value is the aggregate over ranks ("weak" scaling).
+``--shard heads`` instead splits the heads of ONE problem over the ranks
+(40 heads -> 5 per GPU on 8): total work is fixed ("strong" scaling), still
+without any exchange, and the value is the total kept FLOPs over the slowest
+rank's time.
+
+The line also carries the sparsity sweep (0 / 50 / 75 / 90 / 97 %, bf16 and
+FP8), the second workload (Wan2.1-1.3B-480P at 90 %), a sustained leg (two
+seconds of back-to-back forward launches against the sustained GEMM peak) and
+GEMM / copy peaks measured in the same run.
 
 ``--impl reference`` times the CPU oracle as it stands on the host cores.
 """
@@ -41,11 +51,11 @@ import workloads  # noqa: E402
 
 METRIC = "block-sparse attn effective TFLOP/s (kept FLOPs), select+fwd, 97% sparse"
 UNIT = "TFLOP/s"
-# DRAM bytes (read + write) of one bf16 forward launch on the default workload (wan14b, 97 %),
-# from the one-pass ncu capture summarised in profiles/launch_list_wan14b_s97.md.
 # bricks (frames x rows x columns of the token grid) that tile the grid of each workload; one 128-token block each
 BRICKS = {"wan14b": (3, 5, 8), "wan1p3b": (3, 5, 4)}
-FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2580123136 + 761104384}   # ncu one-pass capture of the full-size fwd_pipe_kernel launch
+# DRAM bytes (read + write) of one bf16 forward launch on the default workload (wan14b, 97 %): the dram__bytes_read.sum +
+# dram__bytes_write.sum of a one-pass ncu capture of that launch (a profiler figure: it cannot be taken inside a timed run)
+FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2580123136 + 761104384}
 
 
 def load_peaks():
@@ -235,12 +245,14 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def config_dict(w, dtype):
+def config_dict(w, dtype, shard_heads=False, world=1):
+    par = (f"one problem, its {w.H} heads split over {world} GPUs, no collective" if shard_heads
+           else "independent batch per GPU, no collective")
     return {"workload": f"{w.name}: B={w.B} H={w.H} N={w.N} d={w.d} grid={'x'.join(map(str, w.grid))} "
                         f"block={w.block} sparsity={w.sparsity} (kept {w.topk} of {w.nb} key blocks per query block)",
             "dtype_inputs": dtype, "selection": "pooled-score top-k (sparkattn_select)",
             "l2": "inputs (3 x 774 MB) exceed the 126 MB L2; no explicit flush",
-            "parallelism": "independent batch per GPU, no collective"}
+            "parallelism": par}
 
 
 # --------------------------------------------------------------------------- GPU leg
@@ -252,6 +264,58 @@ def max_over_ranks(value: float, device) -> float:
     t = torch.tensor([value], device=device, dtype=torch.float64)
     torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
     return float(t.item())
+
+
+def sum_over_ranks(value: float, device) -> float:
+    """Sum of a value over all ranks of the default process group (identity without one)."""
+    if not (torch.distributed.is_available() and torch.distributed.is_initialized()):
+        return value
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.SUM)
+    return float(t.item())
+
+
+def sharded_throughput(flops_this_rank: float, ms: float, device) -> float:
+    """Whole-job TFLOP/s of ONE problem whose heads are split over the ranks: the ranks' kept FLOPs added up,
+    over `ms` (the max over ranks)."""
+    return sum_over_ranks(flops_this_rank, device) / (ms * 1e-3) / 1e12
+
+
+def peaks_in_run(dev):
+    """GEMM and copy rates measured in this run with library routines, outside every timed region: the
+    denominators' method (8192^3 bf16 matmul, 1 Gi-element bf16 copy, best of a few) plus an FP8 GEMM."""
+    out = {}
+
+    def best(fn, reps=5):
+        fn(); torch.cuda.synchronize()
+        t = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize()
+            t.append(a.elapsed_time(b))
+        return min(t)
+
+    n = 8192
+    x = torch.randn((n, n), device=dev, dtype=torch.bfloat16)
+    y = torch.randn((n, n), device=dev, dtype=torch.bfloat16)
+    out["bf16_gemm_tflops"] = 2 * n ** 3 / (best(lambda: torch.matmul(x, y)) * 1e-3) / 1e12
+    try:
+        xa = x.to(torch.float8_e4m3fn)
+        yb = y.to(torch.float8_e4m3fn).t().contiguous().t()          # column-major second operand
+        one = torch.ones((), device=dev, dtype=torch.float32)
+        out["fp8_gemm_tflops"] = 2 * n ** 3 / (best(lambda: torch._scaled_mm(xa, yb, one, one, out_dtype=torch.bfloat16)) * 1e-3) / 1e12
+        del xa, yb
+    except Exception as exc:  # the routine's signature differs between library versions
+        out["fp8_gemm_tflops"] = None
+        out["fp8_gemm_error"] = str(exc)[:120]
+    del x, y
+    src = torch.empty(1 << 30, device=dev, dtype=torch.bfloat16)
+    dst = torch.empty_like(src)
+    out["copy_GBps"] = 2 * src.numel() * 2 / (best(lambda: dst.copy_(src)) * 1e-3) / 1e9
+    del src, dst
+    torch.cuda.empty_cache()
+    out["how"] = "torch.matmul bf16 8192^3, torch._scaled_mm e4m3 8192^3, copy_ of 1 Gi bf16 elements; best of 5 each"
+    return out
 
 
 def aggregate_throughput(flops_per_rank: float, ms: float, world: int) -> float:
@@ -297,16 +361,26 @@ def run_ours(args, w):
     sa.lib()
     peaks = load_peaks()
     stream = torch.cuda.current_stream()
+    run_peaks = peaks_in_run(dev) if not args.no_run_peaks else None
 
-    # every rank owns an independent batch of the same shape (different seed)
-    wr = workloads.Workload(w.name, w.cfg_id + 1000 * rank, w.B, w.H, w.d, w.grid, w.block, w.sparsity)
-    q, k, v = workloads.structured_qkv(wr, device=dev)
+    shard_heads = args.shard == "heads" and world > 1
+    if shard_heads:
+        # ONE problem, its heads split over the ranks (fixed total work): no exchange, heads are independent
+        mine = list(workloads.shard_heads(w.H, world, rank))
+        wr = w
+        q, k, v = workloads.structured_qkv(w, heads=mine, device=dev)
+    else:
+        # every rank owns an independent batch of the same shape (different seed)
+        mine = list(range(w.H))
+        wr = workloads.Workload(w.name, w.cfg_id + 1000 * rank, w.B, w.H, w.d, w.grid, w.block, w.sparsity)
+        q, k, v = workloads.structured_qkv(wr, device=dev)
+    Hl = len(mine)
     topk, nb = w.topk, w.nb
     shape = sa.make_shape(q, w.block)
     ws_sel = sa.alloc_workspace(shape, 0, topk, dev)
-    ws_fwd = sa.alloc_workspace(shape, 1, nb if args.sweep else topk, dev)
-    kept_idx = torch.empty((w.B, w.H, nb, topk), dtype=torch.int32, device=dev)
-    kept_cnt = torch.empty((w.B, w.H, nb), dtype=torch.int32, device=dev)
+    ws_fwd = sa.alloc_workspace(shape, 1, topk if args.no_sweep else nb, dev)
+    kept_idx = torch.empty((w.B, Hl, nb, topk), dtype=torch.int32, device=dev)
+    kept_cnt = torch.empty((w.B, Hl, nb), dtype=torch.int32, device=dev)
     out = torch.empty_like(q)
 
     K = args.steps
@@ -335,9 +409,9 @@ def run_ours(args, w):
     ms_fwd = statistics.mean(a.elapsed_time(b) for a, b in ev["fwd"])
     idx_cpu, cnt_cpu = kept_idx.cpu(), kept_cnt.cpu()
     flops = kept_flops(w, idx_cpu, cnt_cpu)
-    value = aggregate_throughput(flops, ms_step, world)
+    value = sharded_throughput(flops, ms_step, dev) if shard_heads else aggregate_throughput(flops, ms_step, world)
     fwd_tflops = flops / (ms_fwd * 1e-3) / 1e12
-    elems = w.B * w.H * w.N * w.d
+    elems = q.numel()
     sel_bytes = 2 * elems * 2 + kept_idx.numel() * 4 + kept_cnt.numel() * 4
     kernels = {
         "select": {"ms": ms_sel, "launches_per_step": 2, "algorithmic_bytes": sel_bytes,
@@ -352,9 +426,10 @@ def run_ours(args, w):
 
     # ---- FP8 leg: 3 quantise launches + FP8 forward (selection reuses the bf16 lists)
     fp8 = None
+    codes = scales = None
     if not args.no_fp8:
         codes = [torch.empty(q.shape, dtype=torch.uint8, device=dev) for _ in range(3)]
-        scales = [torch.empty((w.B, w.H, nb), dtype=torch.float32, device=dev) for _ in range(3)]
+        scales = [torch.empty((w.B, Hl, nb), dtype=torch.float32, device=dev) for _ in range(3)]
         evq = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         evf = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
 
@@ -381,9 +456,11 @@ def run_ours(args, w):
                "fwd_ms": ms_f8, "fwd_TFLOPs": flops / (ms_f8 * 1e-3) / 1e12,
                "fwd_frac_of_nominal_fp8_peak_4500": flops / (ms_f8 * 1e-3) / 1e12 / 4500.0,
                "fwd_frac_of_2x_measured_bf16_peak": flops / (ms_f8 * 1e-3) / 1e12 / (2 * peaks["bf16"]),
-               "note": "FP8 peak = measured bf16 peak x 2 (nominal ratio); torch._scaled_mm 8192^3 measured 3122 TFLOP/s on this pool"}
+               "fwd_frac_of_fp8_gemm_measured_in_run": (flops / (ms_f8 * 1e-3) / 1e12 / run_peaks["fp8_gemm_tflops"]
+                                                        if run_peaks and run_peaks.get("fp8_gemm_tflops") else None),
+               "note": "FP8 peak = measured bf16 peak x 2 (nominal ratio); the FP8 GEMM rate measured in this run is in peaks_in_run"}
         # per-token activation quantisation (the paper's fused scale-and-cast kernel), one tensor, outside the step
-        tok_scales = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=dev)
+        tok_scales = torch.empty((w.B, Hl, w.N), dtype=torch.float32, device=dev)
         evt = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
 
         def step_tok(i):
@@ -399,15 +476,15 @@ def run_ours(args, w):
         fp8["quant_per_token_ms"] = ms_tok
         fp8["quant_per_token_GBps"] = tbytes / (ms_tok * 1e-3) / 1e9
         fp8["quant_per_token_frac_of_hbm_peak"] = tbytes / (ms_tok * 1e-3) / 1e9 / peaks["hbm"]
-        del codes, tok_scales
+        del tok_scales
 
     # ---- compensation branch + gate fusion (d = 128 only): state pass over K, V, then the fused apply pass
     comp = None
     if not args.no_comp and w.d == 128:
-        pq, pk, gate = workloads.compensation_params(wr, 64, device=dev)
+        pq, pk, gate = workloads.compensation_params(wr, 64, heads=mine, device=dev)
         axis, freq = workloads.rope_schedule(w.d, 64)
         ws_c = torch.empty(sa.comp_workspace_bytes(shape, w.grid), dtype=torch.uint8, device=dev)
-        state = torch.empty((w.B, w.H, 64, w.d), dtype=torch.float32, device=dev)
+        state = torch.empty((w.B, Hl, 64, w.d), dtype=torch.float32, device=dev)
         fused = torch.empty_like(q)
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         eva = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
@@ -471,51 +548,99 @@ def run_ours(args, w):
             raise RuntimeError("device status after the brick-order forward")
         ms_g = statistics.mean(a.elapsed_time(b) for a, b in evg)
         gbytes = elems * 2 + qb_.numel() * 2
-        # attention mass held by the kept blocks, raster order against brick order, on sampled query rows
-        gen = torch.Generator().manual_seed(11)
-        heads = list(range(min(w.H, 4)))
-        rows = torch.randint(0, w.N, (64,), generator=gen).to(dev)
-        mass_r = mass_b = 0.0
-        for hh in heads:
-            logits = (q[0, hh, rows].float() @ k[0, hh].float().T) / math.sqrt(w.d)
-            pr = torch.softmax(logits, dim=-1)                                         # [rows, N]
-            blk_of_key = torch.arange(w.N, device=dev) // w.block
-            keep_r = torch.zeros((rows.numel(), nb), dtype=torch.bool, device=dev)
-            keep_r.scatter_(1, kept_idx[0, hh, rows // w.block].long(), True)
-            mass_r += float((pr * keep_r[:, blk_of_key]).sum()) / rows.numel()
-            pos = scatter[rows].long()                                                 # the rows' positions in brick order
-            keep_b = torch.zeros((rows.numel(), nbr), dtype=torch.bool, device=dev)
-            keep_b.scatter_(1, idx_b[0, hh, pos // w.block].long(), True)
-            mass_b += float((pr * keep_b[:, scatter.long() // w.block]).sum()) / rows.numel()
         bricks = {"brick": list(brick), "blocks": nbr, "real_rows_per_block": [int(valid.min()), int(valid.max())], "topk": topk_b,
                   "gather_ms_per_tensor": ms_g, "gather_GBps": gbytes / (ms_g * 1e-3) / 1e9,
                   "gather_frac_of_hbm_peak": gbytes / (ms_g * 1e-3) / 1e9 / peaks["hbm"],
                   "select_ms": statistics.mean(a.elapsed_time(b) for a, b in evs_b),
-                  "fwd_ms": statistics.mean(a.elapsed_time(b) for a, b in evf_b),
-                  "attention_mass_in_kept_blocks": {"raster": mass_r / len(heads), "bricks": mass_b / len(heads),
-                                                    "sample": f"{rows.numel()} query rows of heads {heads[0]}-{heads[-1]}, equal budget ({w.topk} of {nb} / {topk_b} of {nbr} blocks)"}}
+                  "fwd_ms": statistics.mean(a.elapsed_time(b) for a, b in evf_b)}
         del qb_, kb_, vb_, out_b, ws_sb, ws_fb
 
-    # ---- sparsity sweep (optional): fwd only, lists from sparkattn_select
+    def timed_launches(fn, reps, warm=1):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream); torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    # ---- sustained leg: about two seconds of back-to-back forward launches per dtype (a DiT runs this kernel for
+    # seconds, under the power cap), against the sustained GEMM peak; SM clock sampled during the region
+    sustained = None
+    if not args.no_sustained:
+        sustained = {}
+        legs = [("bf16", lambda: sa.fwd(q, k, v, kept_idx, kept_cnt, w.block, out=out, workspace=ws_fwd), ms_fwd)]
+        if codes is not None:
+            legs.append(("fp8", lambda: sa.fwd(codes[0], codes[1], codes[2], kept_idx, kept_cnt, w.block, scales=tuple(scales),
+                                               out=out, workspace=ws_fwd), fp8["fwd_ms"]))
+        for name, fn, ms_burst in legs:
+            reps = max(20, int(args.sustained_seconds * 1e3 / ms_burst))
+            with ClockSampler(local) as c2:
+                ms = max_over_ranks(timed_launches(fn, reps, warm=3), dev)
+            tf = flops / (ms * 1e-3) / 1e12
+            ck = c2.summary()
+            denom = peaks["bf16_sustained"] * (2.0 if name == "fp8" else 1.0)
+            sustained[name] = {"ms": ms, "launches": reps, "TFLOPs": tf, "peak_sustained": denom,
+                               "frac_sustained": tf / denom, "clocks": ck,
+                               "ms_x_sm_mhz": ms * ck["sm_mhz"] if ck.get("sm_mhz") else None}
+        if sa.read_status(ws_fwd) != sa.OK:
+            raise RuntimeError("device status after the sustained leg")
+        roofline["frac_sustained"] = sustained["bf16"]["frac_sustained"]
+        roofline["sustained"] = {"ms_per_launch": sustained["bf16"]["ms"], "achieved": sustained["bf16"]["TFLOPs"],
+                                 "peak": peaks["bf16_sustained"], "clocks": sustained["bf16"]["clocks"]}
+
+    # ---- sparsity sweep: forward only (lists from sparkattn_select at every level), bf16 and FP8
     sweep = None
-    if args.sweep:
+    if not args.no_sweep:
         sweep = []
         for s in (0.0, 0.5, 0.75, 0.9, 0.97):
             ws_ = w.with_sparsity(s)
             ki, kc = sa.select(q, k, w.block, ws_.topk, workspace=ws_sel)
-            reps = 2 if s < 0.6 else 5
-            sa.fwd(q, k, v, ki, kc, w.block, out=out, workspace=ws_fwd)
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for _ in range(reps):
-                sa.fwd(q, k, v, ki, kc, w.block, out=out, workspace=ws_fwd)
-            b.record(stream); torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / reps
             fl = kept_flops(w, ki.cpu(), kc.cpu())
-            sweep.append({"sparsity": s, "kept": ws_.topk, "dtype": "bf16", "ms": ms, "TFLOPs": fl / ms / 1e9,
-                          "frac_of_bf16_peak": fl / ms / 1e9 / peaks["bf16"]})
+            reps = 2 if s < 0.6 else 5
+            runs = [("bf16", lambda: sa.fwd(q, k, v, ki, kc, w.block, out=out, workspace=ws_fwd), peaks["bf16"])]
+            if codes is not None:
+                runs.append(("fp8", lambda: sa.fwd(codes[0], codes[1], codes[2], ki, kc, w.block, scales=tuple(scales), out=out,
+                                                   workspace=ws_fwd), 2 * peaks["bf16"]))
+            for name, fn, pk in runs:
+                ms = max_over_ranks(timed_launches(fn, reps), dev)
+                sweep.append({"sparsity": s, "kept": ws_.topk, "dtype": name, "ms": ms, "TFLOPs": fl / ms / 1e9,
+                              "frac_of_peak": fl / ms / 1e9 / pk})
+            if sa.read_status(ws_fwd) != sa.OK:
+                raise RuntimeError(f"device status in the sweep at sparsity {s}")
             del ki, kc
+    del codes, scales
+
+    # ---- second workload (the 480P shape at 90 %): select + forward, bf16 and FP8, same calls
+    second = None
+    if not args.no_second_workload and w.name == "wan14b" and not args.block:
+        w2 = workloads.WAN_1P3B_480P
+        heads2 = list(workloads.shard_heads(w2.H, world, rank)) if shard_heads else list(range(w2.H))
+        if heads2:
+            w2r = w2 if shard_heads else workloads.Workload(w2.name, w2.cfg_id + 1000 * rank, w2.B, w2.H, w2.d, w2.grid, w2.block, w2.sparsity)
+            q2, k2, v2 = workloads.structured_qkv(w2r, heads=heads2, device=dev)
+            shape2 = sa.make_shape(q2, w2.block)
+            ws_s2 = sa.alloc_workspace(shape2, 0, w2.topk, dev); ws_f2 = sa.alloc_workspace(shape2, 1, w2.topk, dev)
+            ki2, kc2 = sa.select(q2, k2, w2.block, w2.topk, workspace=ws_s2)
+            out2 = torch.empty_like(q2)
+            cs2 = [sa.quant_fp8(t, w2.block) for t in (q2, k2, v2)]
+            fl2 = kept_flops(w2, ki2.cpu(), kc2.cpu())
+            ms_s2 = timed_launches(lambda: sa.select(q2, k2, w2.block, w2.topk, kept_idx=ki2, kept_cnt=kc2, workspace=ws_s2), K, warm=3)
+            ms_f2 = timed_launches(lambda: sa.fwd(q2, k2, v2, ki2, kc2, w2.block, out=out2, workspace=ws_f2), K, warm=3)
+            ms_q2 = timed_launches(lambda: [sa.quant_fp8(t, w2.block, codes=c, scales=sc) for t, (c, sc) in zip((q2, k2, v2), cs2)], K, warm=3)
+            ms_f82 = timed_launches(lambda: sa.fwd(cs2[0][0], cs2[1][0], cs2[2][0], ki2, kc2, w2.block,
+                                                   scales=tuple(sc for _, sc in cs2), out=out2, workspace=ws_f2), K, warm=3)
+            if sa.read_status(ws_f2) != sa.OK or sa.read_status(ws_s2) != sa.OK:
+                raise RuntimeError("device status on the second workload")
+            second = {"config": config_dict(w2, "bf16")["workload"], "kept_flops": fl2, "select_ms": ms_s2,
+                      "fwd_bf16_ms": ms_f2, "fwd_bf16_TFLOPs": fl2 / ms_f2 / 1e9, "fwd_bf16_frac_of_peak": fl2 / ms_f2 / 1e9 / peaks["bf16"],
+                      "quant_ms_3_tensors": ms_q2, "fwd_fp8_ms": ms_f82, "fwd_fp8_TFLOPs": fl2 / ms_f82 / 1e9,
+                      "fwd_fp8_frac_of_2x_bf16_peak": fl2 / ms_f82 / 1e9 / (2 * peaks["bf16"]),
+                      "step_ms_select_plus_fwd_bf16": ms_s2 + ms_f2, "launches_timed_each": K,
+                      "l2": "Q, K, V of this shape (3 x 101 MB) exceed the 126 MB L2 together; no explicit flush"}
+            del q2, k2, v2, out2, cs2, ws_s2, ws_f2, ki2, kc2
 
     # ---- end to end through the host-buffer C-ABI call (H2D of Q,K,V and D2H of O inside the timed region)
     e2e = None
@@ -531,7 +656,7 @@ def run_ours(args, w):
             sa.attention_host(hq, hk, hv, w.block, topk, out=ho, arena=arena)
 
         ms_e = time_region(step_e2e, ke, 1, stream, dist_on) / ke
-        e2e = {"value": world * flops / (ms_e * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms_e, "steps": ke,
+        e2e = {"value": (sharded_throughput(flops, ms_e, dev) if shard_heads else world * flops / (ms_e * 1e-3) / 1e12), "unit": UNIT, "ms_per_step": ms_e, "steps": ke,
                "h2d_bytes_per_step": 3 * hq.numel() * 2, "d2h_bytes_per_step": ho.numel() * 2 + 8,
                "call": "sparkattn_attention_host (pinned host Q,K,V -> select -> fwd -> host O)"}
         del arena, hq, hk, hv, ho
@@ -543,14 +668,12 @@ def run_ours(args, w):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": config_dict(w, "bf16"),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong" if shard_heads else "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config_dict(w, "bf16", shard_heads, world),
             "kept_flops_per_step_per_gpu": flops, "clocks": clocks, "gpu_launches": (4 if pipelined else 3) * K,
-            "kernels": kernels, "roofline": roofline, "fp8": fp8, "compensation": comp, "bricks": bricks, "e2e": e2e,
-            "cpu_baseline": cpu,
+            "kernels": kernels, "roofline": roofline, "fp8": fp8, "sweep": sweep, "second_workload": second,
+            "compensation": comp, "bricks": bricks, "e2e": e2e, "cpu_baseline": cpu, "peaks_in_run": run_peaks,
         }
-        if sweep is not None:
-            line["sweep"] = sweep
         print(json.dumps(line), flush=True)
     if dist_on:
         torch.distributed.destroy_process_group()
@@ -570,7 +693,13 @@ def main():
     ap.add_argument("--no-fp8", action="store_true")
     ap.add_argument("--no-comp", action="store_true", help="skip the compensation-branch leg")
     ap.add_argument("--no-bricks", action="store_true", help="skip the brick-token-order leg")
-    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sparsity sweep (0/50/75/90/97 %, bf16 and FP8)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the two-second back-to-back forward leg")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0)
+    ap.add_argument("--no-second-workload", action="store_true", help="skip the Wan2.1-1.3B-480P sub-record")
+    ap.add_argument("--no-run-peaks", action="store_true", help="skip the GEMM / copy peaks measured in this run")
+    ap.add_argument("--shard", choices=["batch", "heads"], default="batch",
+                    help="N > 1: batch = an independent problem per GPU (weak scaling); heads = one problem, heads split (strong)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     args = ap.parse_args()

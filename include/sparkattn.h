@@ -19,8 +19,11 @@
  *
  * Conventions shared by all calls
  *   - Every data pointer is DEVICE memory owned by the caller unless a
- *     parameter name ends in `_host`.  The library allocates nothing, keeps
- *     no pointer after the call returns and keeps no per-call global state.
+ *     parameter name ends in `_host`.  The library allocates no device
+ *     memory and keeps no pointer after the call returns.  What it does keep
+ *     between calls, per device: two copy streams that
+ *     sparkattn_attention_host creates on first use, the fixed scratch array
+ *     of sparkattn_select_noalloc with its cached address, and the SM count.
  *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*;
  *     NULL = the legacy default stream) and return without synchronising,
  *     except sparkattn_read_status and sparkattn_attention_host.
@@ -78,16 +81,18 @@ int sparkattn_version(void);
 const char* sparkattn_status_string(int status);
 
 /* Bytes of device workspace a call needs.  which: 0 = sparkattn_select (pass
- * topk), 1 = sparkattn_fwd (pass kmax: for d = 128 with 128-token blocks the
- * forward keeps a range-checked copy of the kept lists and one scale per head
- * behind the status words, about 4 * B * H * nb * (kmax + 1) bytes; 256 bytes
- * otherwise), 2 = sparkattn_gather_tokens (256).  Returns 0 for an invalid shape or, for 0 and 1, a
- * non-positive topk / kmax. */
+ * topk), 1 = sparkattn_fwd (pass kmax: for d = 128 the forward keeps
+ * range-checked, merged copies of the kept lists of every pair of adjacent
+ * query blocks and one scale per head behind the status words, about
+ * 4 * B * H * nb * (kmax + 2) bytes for 128- and for 64-token blocks; 256 bytes
+ * for d = 64), 2 = sparkattn_gather_tokens (256).  Returns 0 for an invalid
+ * shape or, for 0 and 1, a non-positive topk / kmax. */
 size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t topk_or_kmax);
 
 /*
- * Block selection (the selector M_phi of Sec. 2 / Sec. 4.1; the paper names
- * "top-k selection, blockwise scores" without fixing a rule, so the rule is:)
+ * Block selection (the selector M_phi of Sec. 2 / Sec. 4.1; the paper lists
+ * kinds of selectors, top-k over per-block scores among them, without fixing
+ * a rule, so the rule is:)
  *   1. pooled sum over the valid tokens of a block, fp32, ascending token order
  *   2. pooled mean = sum / n_valid (IEEE fp32 divide)
  *   3. score(i, j) = fmaf chain over channels c ascending of pq[i,c] * pk[j,c]
@@ -120,9 +125,9 @@ int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint
                         uint32_t flags, void* cuda_stream);
 
 /*
- * Per-token FP8 quantisation: the activation-quantisation kernel as the paper
- * states it (Sec. 4.3: activations "scaled dynamically per token", scale and
- * cast in one pass).  Same arithmetic as sparkattn_quant_fp8 with the token
+ * Per-token FP8 quantisation: the activation-quantisation kernel at the
+ * paper's own granularity (Sec. 4.3: one dynamic scale per token row, scale
+ * and cast in one pass).  Same arithmetic as sparkattn_quant_fp8 with the token
  * block replaced by one token row: amax over the row's d channels, clamped at
  * 1e-12; scale = amax / 448; code = e4m3_rne_satfinite(x * (448 / amax)).
  * Not consumed by sparkattn_fwd (which takes per-block scales); provided for
@@ -163,9 +168,9 @@ int sparkattn_fwd(const sparkattn_shape_t* shape, int32_t dtype, const void* q, 
                   size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Causal frame window (Sec. 1, "Extension to auto-regressive video diffusion":
- * the compensated sparse attention "can be restricted to a causal window"; the
- * paper gives no formula, so the reading is:)  tokens come in frames of
+ * Causal frame window (Sec. 1, the auto-regressive extension: the paper says
+ * the attention may be limited to a causal window and gives no formula, so
+ * the reading is:)  tokens come in frames of
  * `frame_tokens` consecutive tokens; key token j counts for query token i iff
  *     i / frame_tokens - window_frames  <  j / frame_tokens  <=  i / frame_tokens.
  * sparkattn_select_window ranks only the key blocks that hold such a key for
@@ -249,7 +254,8 @@ int sparkattn_read_status(void* workspace, void* cuda_stream);
  * receive the selected lists.  arena: device scratch of at least
  * sparkattn_arena_bytes(shape, dtype, topk) bytes, 256-byte aligned.
  * The heads are independent, so the call runs as a pipeline over groups of
- * heads (about eight groups, at most 16): while one group is selected and
+ * heads (about eight groups, at most 16; a group never spans two batch
+ * entries, so B > 16 returns SPARKATTN_E_UNSUPPORTED_SHAPE): while one group is selected and
  * attended on `cuda_stream`, the next is copied in and the previous one's
  * output copied out on two copy streams that the library creates once per
  * device and keeps; both are ordered after work already queued on

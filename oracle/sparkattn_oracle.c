@@ -15,9 +15,9 @@
  *                             (paper Sec. 2 "Block sparsity" + the dense
  *                             attention formula there; Sec. 4.1, sparse branch
  *                             O_s = A_M(Q,K,V)).
- *   SEL-1  oracle_select      pooled-block scores + top-k (Sec. 2 names
- *                             "top-k selection, blockwise scores" as the
- *                             selector family but fixes no rule; the rule used
+ *   SEL-1  oracle_select      pooled-block scores + top-k (Sec. 2 lists kinds of
+ *                             selectors, top-k over per-block scores among
+ *                             them, but fixes no rule; the rule used
  *                             here is spelled out step by step below).
  *   QNT-1  oracle_quant_fp8   per-(head, token-block) absmax scale + E4M3
  *                             round-to-nearest-even encode (Sec. 4.3 names FP8
@@ -27,8 +27,8 @@
  *                             token-wise gate fusion (Sec. 4.1), fp64.
  *   WIN-0  frame_tokens / window arguments of oracle_attention and oracle_select:
  *                             the causal window of the auto-regressive extension
- *                             (Sec. 1, "Extension to auto-regressive video diffusion":
- *                             the attention "can be restricted to a causal window";
+ *                             (Sec. 1, the auto-regressive extension: the attention
+ *                             may be limited to a causal window;
  *                             no formula is given).  Reading: tokens come in frames of
  *                             F = frame_tokens; key j counts for query i iff
  *                             j / F lies in (i / F - window, i / F].  Selection only

@@ -368,6 +368,8 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
   const int nb = num_blocks(shape);
   if (topk < 1 || topk > nb) return SPARKATTN_E_INVALID_ARG;
   if (!aligned256(arena)) return SPARKATTN_E_MISALIGNED;
+  // a head group never spans two batch entries, so the batch count bounds the number of groups from below
+  if (shape->B > kHostPathMaxChunks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   sparkattn_shape_t s = *shape;  // host tensors are contiguous
   s.stride_n = s.d; s.stride_h = (int64_t)s.N * s.d; s.stride_b = (int64_t)s.H * s.N * s.d;
   const Arena a = plan_arena(s, dtype, topk);
@@ -379,7 +381,8 @@ int sparkattn_attention_host(const sparkattn_shape_t* shape, int32_t dtype, cons
 
   // head groups: about 8 per call, never across a batch boundary
   int heads_per_chunk = (s.H + 7) / 8;
-  while ((int64_t)s.B * ((s.H + heads_per_chunk - 1) / heads_per_chunk) > kHostPathMaxChunks) ++heads_per_chunk;
+  while (heads_per_chunk < s.H && (int64_t)s.B * ((s.H + heads_per_chunk - 1) / heads_per_chunk) > kHostPathMaxChunks)
+    ++heads_per_chunk;
   struct Chunk { int b, h0, hc; };
   Chunk chunks[kHostPathMaxChunks];
   int n_chunks = 0;

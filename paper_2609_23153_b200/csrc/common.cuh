@@ -64,9 +64,10 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 }
 
 // Bounded wait: polls the barrier until it flips, another thread of the CTA
-// raises `abort_flag`, or kWaitLimitNs of wall time have passed (checked every
-// 64 polls).  On expiry it raises the flag, records a timeout in the status
-// word and returns false; callers then leave their role loop.
+// raises `abort_flag`, or `limit_ns` (kWaitLimitNs unless the caller says
+// otherwise) of wall time have passed (checked every 64 polls).  On expiry it
+// raises the flag, records a timeout and `wait_id` in the status words and
+// returns false; callers then leave their role loop.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
@@ -74,14 +75,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status, int wait_id) {
+                                          int32_t* status, int wait_id, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) break;
+      if (global_timer_ns() - t0 > limit_ns) break;
     }
   }
   *abort_flag = 1;

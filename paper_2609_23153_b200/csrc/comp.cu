@@ -23,6 +23,7 @@
 
 #include "common.cuh"
 #include "launch.h"
+#include "tmap.h"
 
 namespace sparkattn {
 
@@ -615,34 +616,11 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 }
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn comp_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn) return fn;
-  void* ptr = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess)
-    return nullptr;
-  fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  return fn;
-}
-
 static int comp_map(CUtensorMap* map, const void* base, cuuint64_t d0, cuuint64_t d1, cuuint64_t d2, cuuint64_t d3,
                     cuuint64_t s1, cuuint64_t s2, cuuint64_t s3, cuuint32_t box_rows) {
-  EncodeTiledFn enc = comp_encode_fn();
-  if (!enc) return SPARKATTN_E_NO_DEVICE;
-  const cuuint64_t dims[4] = {d0, d1, d2, d3};
-  const cuuint64_t strides[3] = {s1 * 2, s2 * 2, s3 * 2};
-  const cuuint32_t box[4] = {64u, box_rows, 1u, 1u};
-  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+  const uint64_t dims[4] = {d0, d1, d2, d3};
+  const uint64_t strides[3] = {s1, s2, s3};
+  return make_slab_map(map, base, 2, dims, strides, box_rows);
 }
 
 // Chunks of token tiles per (batch, head): CTAs = B*H*chunks should fill whole waves of one CTA per

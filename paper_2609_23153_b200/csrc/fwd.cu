@@ -29,6 +29,7 @@
 
 #include "common.cuh"
 #include "launch.h"
+#include "tmap.h"
 
 namespace sparkattn {
 
@@ -466,39 +467,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ C
 
 // ------------------------------------------------------------------ host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (fn) return fn;
-  void* ptr = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess)
-    return nullptr;
-  fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  return fn;
-}
-
-// [B,H,N,d] tensor, box = one 128-byte-wide slab of `box_rows` token rows, 128-byte swizzle.
-static int make_tile_map(CUtensorMap* map, const void* base, int elt_bytes, const sparkattn_shape_t& s,
-                         int box_rows) {
-  EncodeTiledFn enc = get_encode_fn();
-  if (!enc) return SPARKATTN_E_NO_DEVICE;
-  const cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.H, (cuuint64_t)s.B};
-  const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * elt_bytes, (cuuint64_t)s.stride_h * elt_bytes,
-                                 (cuuint64_t)s.stride_b * elt_bytes};
-  const cuuint32_t box[4] = {(cuuint32_t)(128 / elt_bytes), (cuuint32_t)box_rows, 1u, 1u};
-  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  const CUresult r = enc(map, elt_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
-                         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
-}
-
 size_t fwd_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
   // the pipelined kernel keeps range-checked, compacted copies of the kept lists behind the header
   if (fwd_pipe_supported(s)) return fwd_pipe_workspace_bytes(s, kmax);
@@ -525,18 +493,17 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
                const int32_t* kept_cnt, int kmax, int frame_tokens, int window, const int32_t* block_valid, void* out,
                float* lse, void* workspace, cudaStream_t stream) {
   const bool fp8 = dtype == SPARKATTN_FP8_E4M3;
-#ifndef SPARKATTN_FWD_NO_PIPE
   if (fwd_pipe_supported(s))
     return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
                            block_valid, out, lse, workspace, stream);
-#endif
-  if (block_valid != nullptr) return SPARKATTN_E_UNSUPPORTED_SHAPE;   // padded bricks: d = 128 (the pipelined kernel) only
+  // d = 128 always runs the persistent kernels; a sequence too long for their list pre-pass is not served
+  if (s.d != 64 || s.block != 64 || fp8 || block_valid != nullptr) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;
   int rc;
-  if ((rc = make_tile_map(&mq, q, elt, s, s.block)) != SPARKATTN_OK) return rc;
-  if ((rc = make_tile_map(&mk, k, elt, s, s.block)) != SPARKATTN_OK) return rc;
-  if ((rc = make_tile_map(&mv, v, elt, s, s.block)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mq, q, elt, s, s.block)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mk, k, elt, s, s.block)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mv, v, elt, s, s.block)) != SPARKATTN_OK) return rc;
   FwdParams prm;
   prm.kept_idx = kept_idx;
   prm.kept_cnt = kept_cnt;
@@ -558,16 +525,7 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
   const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
   prm.scale_log2 = sc * 1.4426950408889634f;
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
-  if (s.d == 128 && s.block == 128) {
-    return fp8 ? launch_fwd_t<128, 128, true>(s, mq, mk, mv, prm, stream)
-               : launch_fwd_t<128, 128, false>(s, mq, mk, mv, prm, stream);
-  }
-  if (s.d == 128 && s.block == 64) {
-    return fp8 ? launch_fwd_t<128, 64, true>(s, mq, mk, mv, prm, stream)
-               : launch_fwd_t<128, 64, false>(s, mq, mk, mv, prm, stream);
-  }
-  if (s.d == 64 && s.block == 64 && !fp8) return launch_fwd_t<64, 64, false>(s, mq, mk, mv, prm, stream);
-  return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  return launch_fwd_t<64, 64, false>(s, mq, mk, mv, prm, stream);
 }
 
 }  // namespace sparkattn

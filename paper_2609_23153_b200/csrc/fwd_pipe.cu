@@ -34,6 +34,7 @@
 
 #include "common.cuh"
 #include "launch.h"
+#include "tmap.h"
 
 namespace sparkattn {
 
@@ -837,36 +838,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 }
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*PipeEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static PipeEncodeFn pipe_encode_fn() {
-  static PipeEncodeFn fn = nullptr;
-  if (fn) return fn;
-  void* ptr = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-      qres != cudaDriverEntryPointSuccess)
-    return nullptr;
-  fn = reinterpret_cast<PipeEncodeFn>(ptr);
-  return fn;
-}
-
-// [B,H,N,d] tensor of 2-byte (bf16) or 1-byte (E4M3) elements; box = `rows` rows of one 128-byte slab
-static int pipe_map(CUtensorMap* map, const void* base, const sparkattn_shape_t& s, int elt = 2, int rows = kPBLK) {
-  PipeEncodeFn enc = pipe_encode_fn();
-  if (!enc) return SPARKATTN_E_NO_DEVICE;
-  const cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.N, (cuuint64_t)s.H, (cuuint64_t)s.B};
-  const cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * elt, (cuuint64_t)s.stride_h * elt, (cuuint64_t)s.stride_b * elt};
-  const cuuint32_t box[4] = {(cuuint32_t)(128 / elt), (cuuint32_t)rows, 1u, 1u};
-  const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
-  const CUresult r = enc(map, elt == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
-                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? SPARKATTN_OK : SPARKATTN_E_CUDA;
-}
-
 // items (query blocks, or pairs of 64-token query blocks) per (batch, head), and list entries per item
 static void pipe_geometry(const sparkattn_shape_t& s, int kmax, int* nbq, int* lstride) {
   const int nb = (s.N + s.block - 1) / s.block;
@@ -898,10 +869,10 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   int rc;
   const int elt = fp8 ? 1 : 2;
   const bool pair = s.block == 64;
-  if ((rc = pipe_map(&mq, q, s, elt)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mk, k, s, elt, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mv, v, s, elt, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
-  if ((rc = pipe_map(&mo, out, s)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mq, q, elt, s, kPBLK)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mk, k, elt, s, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mv, v, elt, s, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
+  if ((rc = make_token_map(&mo, out, 2, s, kPBLK)) != SPARKATTN_OK) return rc;
   const int nb = (s.N + s.block - 1) / s.block;
   int nbq, lstride;
   pipe_geometry(s, kmax, &nbq, &lstride);
@@ -925,13 +896,8 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   prm.stride_b = s.stride_b; prm.stride_h = s.stride_h; prm.stride_n = s.stride_n;
   const float sc = s.softmax_scale > 0.0f ? s.softmax_scale : 1.0f / sqrtf((float)s.d);
   prm.scale_log2 = sc * 1.4426950408889634f;
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count < 1)
-      return SPARKATTN_E_CUDA;
-  }
+  const int sm_count = current_sm_count();
+  if (sm_count < 1) return SPARKATTN_E_CUDA;
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
   if (pair) {
     const size_t bits = (size_t)kPairWarps * 2 * ((nb + 31) / 32) * sizeof(uint32_t);

@@ -1,7 +1,7 @@
 // sparkattn_select: pooled block scores + top-k kept-block lists.
 //
-// The paper's selector M_phi (Sec. 2, Sec. 4.1) is left open ("top-k
-// selection, blockwise scores"); the rule implemented here is
+// The paper's selector M_phi (Sec. 2, Sec. 4.1) is left open (it lists kinds of
+// selectors, top-k over per-block scores among them); the rule implemented here is
 //   pooled mean of every token block (fp32, tokens added in ascending order,
 //   one IEEE divide), score(i,j) = fmaf chain over channels, keep the topk
 //   key blocks first under (score descending, index ascending), emit ascending.

@@ -85,8 +85,10 @@ def test_fullsize_fp8_quant_and_fwd():
                                   items=local, scales=tuple(s[0, heads].cpu() for _, s in cs))
     items = [(heads[h], i) for h, i in local]
     rel, mx = _relrms(_gather(out[0], items, w), _ref_rows(ref_out, local, w))
-    print(f"wan14b fp8: {len(items)} work items, relRMS {rel:.3e}, max abs {mx:.3e}")
-    assert rel <= 5e-2
+    got, ref = _gather(out[0], items, w).double(), _ref_rows(ref_out, local, w).double()
+    worst_row = float((((got - ref) ** 2).sum(-1) / (ref ** 2).sum(-1).clamp_min(1e-300)).sqrt().max())
+    print(f"wan14b fp8: {len(items)} work items, relRMS {rel:.3e}, max abs {mx:.3e}, worst row relRMS {worst_row:.3e}")
+    assert rel <= 5e-2 and worst_row <= 1.5e-1
     assert torch.isfinite(out.float()).all()
 
 
@@ -152,3 +154,66 @@ def test_fullsize_paper_block_size_64_bf16_and_fp8():
     rel8, mx8 = _relrms(_gather(out8[0], [(heads[h], i) for h, i in local8], w64), _ref_rows(ref8, local8, w64))
     print(f"wan14b 64x64 fp8: {len(local8)} work items, relRMS {rel8:.3e}, max abs {mx8:.3e}")
     assert rel8 <= 5e-2
+
+
+# ----------------------------------------------------------------------------- sparsity sweep on the 720P shape
+SWEEP_HEADS = [0, 17, 39]
+FP8_ROW_RELRMS = 1.5e-1     # guard beside the aggregate bound: one wrong row must not hide in the average
+
+
+@pytest.fixture(scope="module")
+def wan14b_inputs():
+    w = workloads.WAN_14B_720P
+    q, k, v = workloads.structured_qkv(w, device=DEV)
+    cs = [sa.quant_fp8(t, w.block) for t in (q, k, v)]
+    heads = SWEEP_HEADS
+    host = {"bf16": tuple(t[0, heads].cpu() for t in (q, k, v)),
+            "codes": tuple(c[0, heads].cpu() for c, _ in cs), "scales": tuple(s[0, heads].cpu() for _, s in cs)}
+    yield w, (q, k, v), cs, host
+    del q, k, v, cs
+    torch.cuda.empty_cache()
+
+
+def _row_relrms(got, ref):
+    got, ref = got.double(), ref.double()
+    return (((got - ref) ** 2).sum(-1) / (ref ** 2).sum(-1).clamp_min(1e-300)).sqrt()
+
+
+@pytest.mark.parametrize("sparsity", [0.0, 0.5, 0.75, 0.9, 0.97])
+def test_sparsity_sweep_points_bf16_and_fp8(wan14b_inputs, sparsity):
+    """Every point of the sparsity sweep the benchmark reports (0 / 50 / 75 / 90 / 97 % on the 40-head
+    75,600-token shape), bf16 and FP8, through the calls and launch configuration the benchmark times:
+    selection in full on three heads against the oracle (bit-exact), then the forward on the whole tensors
+    with a sample of work items (first block, ragged last block, two seeded random blocks per head) recomputed
+    by the fp64 oracle.  The lists run from 18 to 591 tiles per query block."""
+    w0, (q, k, v), cs, host = wan14b_inputs
+    w = w0.with_sparsity(sparsity)
+    heads = SWEEP_HEADS
+    idx, cnt = sa.select(q, k, w.block, w.topk)
+    qh, kh, vh = host["bf16"]
+    ref_idx, ref_cnt = oracle.select(qh, kh, w.block, w.topk)
+    assert torch.equal(idx[0, heads].cpu(), ref_idx), "kept-block lists differ from the oracle"
+    assert torch.equal(cnt[0, heads].cpu(), ref_cnt)
+    if sparsity == 0.0:
+        assert w.topk == w.nb and torch.equal(ref_idx[0, 5], torch.arange(w.nb, dtype=torch.int32))
+    local = _sample_items(w, range(len(heads)), 2, seed=int(1000 * sparsity) + 3)
+    items = [(heads[h], i) for h, i in local]
+
+    out, lse = sa.fwd(q, k, v, idx, cnt, w.block, return_lse=True, check_status=True)
+    ref_out, ref_lse = oracle.attention(qh, kh, vh, ref_idx, ref_cnt, w.block, items=local)
+    got, ref = _gather(out[0], items, w), _ref_rows(ref_out, local, w)
+    rel, mx = _relrms(got, ref)
+    dl = (_gather(lse[0][..., None], items, w)[:, 0].double() - _ref_rows(ref_lse[..., None], local, w)[:, 0]).abs().max().item()
+    print(f"sweep s={sparsity} bf16: kept {w.topk}, {len(items)} items, relRMS {rel:.3e}, max abs {mx:.3e}, lse {dl:.3e}")
+    assert rel <= 1e-2 and mx <= 3e-2 and dl <= 1e-2
+    assert torch.isfinite(out.float()).all()
+    del out, lse
+
+    out8 = sa.fwd(cs[0][0], cs[1][0], cs[2][0], idx, cnt, w.block, scales=tuple(s for _, s in cs), check_status=True)
+    ref8, _ = oracle.attention(*host["codes"], ref_idx, ref_cnt, w.block, items=local, scales=host["scales"])
+    got8, r8 = _gather(out8[0], items, w), _ref_rows(ref8, local, w)
+    rel8, mx8 = _relrms(got8, r8)
+    rows8 = float(_row_relrms(got8, r8).max())
+    print(f"sweep s={sparsity} fp8: relRMS {rel8:.3e}, max abs {mx8:.3e}, worst row relRMS {rows8:.3e}")
+    assert rel8 <= 5e-2 and rows8 <= FP8_ROW_RELRMS
+    assert torch.isfinite(out8.float()).all()

@@ -2,7 +2,7 @@
 window-restricted selection bit-exact, window-masked block-sparse attention within the bf16 / FP8
 tolerances, rows without any admissible kept key (zero output, lse = -inf), and the benchmark shape on
 sampled work items.  Both forward kernels are covered: d = 128 with 128-token blocks runs the
-persistent pipelined kernel, the other shapes the one-item-per-CTA kernel."""
+persistent pipelined kernel (64-token blocks in pairs), d = 64 the one-item-per-CTA kernel."""
 import math
 
 import pytest
@@ -24,7 +24,7 @@ def _relrms(got, ref):
 @pytest.mark.parametrize("H,d,grid,block,topk,window", [
     (2, 128, (6, 10, 23), 128, 4, 2),      # frames of 230 tokens straddle the 128-token blocks; ragged tail
     (3, 128, (12, 12, 15), 128, 6, 3),     # 180-token frames, 17 blocks per head
-    (2, 128, (5, 9, 11), 64, 5, 1),        # 64-token blocks: the one-item-per-CTA kernel
+    (2, 128, (5, 9, 11), 64, 5, 1),        # 64-token blocks: pairs of query blocks on the persistent kernel
     (2, 64, (4, 8, 20), 64, 4, 2),         # d = 64
 ])
 def test_select_and_fwd_with_window(H, d, grid, block, topk, window):

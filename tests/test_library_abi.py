@@ -205,3 +205,18 @@ def test_padded_brick_entry_points_validate_on_the_host(lib):
     assert lib.sparkattn_gather_tokens(ctypes.byref(s128), fake, ctypes.byref(other), fake, ctypes.c_void_p(0x2000), fake, 256, st) == sa.E_INVALID_ARG
     assert lib.sparkattn_gather_tokens(ctypes.byref(s128), fake, ctypes.byref(s128), fake, fake, fake, 256, st) == sa.E_INVALID_ARG
     assert lib.sparkattn_gather_tokens(ctypes.byref(s128), fake, ctypes.byref(s128), fake, ctypes.c_void_p(0x2000), fake, 16, st) == sa.E_WORKSPACE_TOO_SMALL
+
+
+def test_host_buffer_call_rejects_more_batches_than_head_groups(lib):
+    """The host-buffer path runs at most 16 head groups and a group never spans two batch entries: B = 17
+    must come back as an error at once (it used to loop for ever while sizing the groups)."""
+    fake = ctypes.c_void_p(0x1000)
+    st = ctypes.c_void_p(0)
+    s = _shape(B=17, H=2, N=256, d=64, block=64)
+    r = lib.sparkattn_attention_host(ctypes.byref(s), sa.BF16, fake, fake, fake, 2, fake, ctypes.c_void_p(0), fake, 1 << 40, st)
+    assert r == sa.E_UNSUPPORTED_SHAPE
+    # 16 batch entries of many heads still form 16 groups (one per batch entry): passes the group sizing
+    # and stops at the arena-size check
+    s = _shape(B=16, H=40, N=256, d=64, block=64)
+    r = lib.sparkattn_attention_host(ctypes.byref(s), sa.BF16, fake, fake, fake, 2, fake, ctypes.c_void_p(0), fake, 256, st)
+    assert r == sa.E_WORKSPACE_TOO_SMALL

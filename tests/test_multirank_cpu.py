@@ -37,6 +37,10 @@ def _worker(rank, world, port, q):
         # timing reduction: the slowest rank defines the step time
         ms = bench.max_over_ranks(10.0 + 5.0 * rank, "cpu")
         agg = bench.aggregate_throughput(2.0e12, ms, world)
+        # head-sharded mode of the benchmark: every rank counts the kept FLOPs of its own heads, the job's
+        # throughput is their sum over the slowest rank's time
+        w_mine = w.with_heads(len(mine))
+        strong = bench.sharded_throughput(float(bench.kept_flops(w_mine, idx, cnt)), ms, "cpu")
         if rank == 0:
             heads = sum((g[0] for g in gathered), [])
             full_idx, full_cnt = oracle.select(qq[0], kk[0], w.block, w.topk)
@@ -44,7 +48,9 @@ def _worker(rank, world, port, q):
             ok_part = sorted(heads) == list(range(w.H)) and len(heads) == w.H
             ok_idx = torch.equal(torch.cat([g[1] for g in gathered]), full_idx)
             ok_out = torch.equal(torch.cat([g[2] for g in gathered]), full_out)
-            q.put((ok_part, ok_idx, ok_out, ms, agg))
+            full_flops = bench.kept_flops(w, full_idx, full_cnt)
+            ok_strong = abs(strong - full_flops / (ms * 1e-3) / 1e12) <= 1e-9 * max(1.0, strong)
+            q.put((ok_part, ok_idx, ok_out, ms, agg, ok_strong))
     finally:
         dist.destroy_process_group()
 
@@ -60,8 +66,8 @@ def test_two_ranks_shard_heads_without_exchange():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    ok_part, ok_idx, ok_out, ms, agg = res
-    assert ok_part and ok_idx and ok_out
+    ok_part, ok_idx, ok_out, ms, agg, ok_strong = res
+    assert ok_part and ok_idx and ok_out and ok_strong
     assert ms == 15.0
     assert abs(agg - 2 * 2.0e12 / 15e-3 / 1e12) < 1e-9
 
