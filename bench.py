@@ -459,6 +459,31 @@ def run_ours(args, w):
                "fwd_frac_of_fp8_gemm_measured_in_run": (flops / (ms_f8 * 1e-3) / 1e12 / run_peaks["fp8_gemm_tflops"]
                                                         if run_peaks and run_peaks.get("fp8_gemm_tflops") else None),
                "note": "FP8 peak = measured bf16 peak x 2 (nominal ratio); the FP8 GEMM rate measured in this run is in peaks_in_run"}
+        # fused chain: Q and K are read once for pooling + quantisation (sparkattn_quant_fp8_pooled), scores + top-k
+        # run on the pooled means (sparkattn_select_pooled); against it, the separate calls: select + 3 quant + fwd
+        evp = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+
+        def step8_fused(i):
+            if i >= 0:
+                evp[i][0].record(stream)
+            sa.quant_fp8_pooled(q, w.block, False, ws_sel, codes=codes[0], scales=scales[0])
+            sa.quant_fp8_pooled(k, w.block, True, ws_sel, codes=codes[1], scales=scales[1])
+            sa.quant_fp8(v, w.block, codes=codes[2], scales=scales[2])
+            sa.select_pooled(q, w.block, topk, ws_sel, kept_idx=kept_idx, kept_cnt=kept_cnt)
+            if i >= 0:
+                evp[i][1].record(stream)
+            sa.fwd(codes[0], codes[1], codes[2], kept_idx, kept_cnt, w.block, scales=tuple(scales), out=out,
+                   workspace=ws_fwd)
+
+        ms8f = time_region(step8_fused, K, args.warmup, stream, dist_on) / K
+        if sa.read_status(ws_fwd) != sa.OK or sa.read_status(ws_sel) != sa.OK:
+            raise RuntimeError("device status after the fused fp8 chain")
+        ms_pre = statistics.mean(a.elapsed_time(b) for a, b in evp)
+        fp8["chain_separate_ms_select_quant_fwd"] = ms_sel + ms8
+        fp8["chain_fused_ms_quantpool_topk_fwd"] = ms8f
+        fp8["fused_quantpool_plus_topk_ms"] = ms_pre
+        fp8["separate_select_plus_quant_ms"] = ms_sel + ms_q
+        fp8["fused_launches_per_step"] = 4 + (3 if pipelined else 1)
         # per-token activation quantisation (the paper's fused scale-and-cast kernel), one tensor, outside the step
         tok_scales = torch.empty((w.B, Hl, w.N), dtype=torch.float32, device=dev)
         evt = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]

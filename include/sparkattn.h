@@ -81,10 +81,10 @@ int sparkattn_version(void);
 const char* sparkattn_status_string(int status);
 
 /* Bytes of device workspace a call needs.  which: 0 = sparkattn_select (pass
- * topk), 1 = sparkattn_fwd (pass kmax: for d = 128 the forward keeps
- * range-checked, merged copies of the kept lists of every pair of adjacent
- * query blocks and one scale per head behind the status words, about
- * 4 * B * H * nb * (kmax + 2) bytes for 128- and for 64-token blocks; 256 bytes
+ * topk), 1 = sparkattn_fwd (pass kmax: for d = 128 the forward keeps a
+ * range-checked copy of the kept lists (64-token blocks: the merged lists of
+ * every pair of adjacent query blocks) and one scale per head behind the
+ * status words, about 4 * B * H * nb * (kmax + 1) bytes either way; 256 bytes
  * for d = 64), 2 = sparkattn_gather_tokens (256).  Returns 0 for an invalid
  * shape or, for 0 and 1, a non-positive topk / kmax. */
 size_t sparkattn_workspace_bytes(const sparkattn_shape_t* shape, int32_t which, int32_t topk_or_kmax);
@@ -123,6 +123,30 @@ int sparkattn_select(const sparkattn_shape_t* shape, const void* q_bf16, const v
  */
 int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes, float* scales,
                         uint32_t flags, void* cuda_stream);
+
+/*
+ * Quantisation and block pooling in one pass (Sec. 4.3 fuses scaling and
+ * casting into a single pass over memory; here the selection's block pooling
+ * rides on the same pass, so that in the FP8 configuration Q and K are read
+ * from HBM once for selection and quantisation together).
+ *
+ * sparkattn_quant_fp8_pooled: sparkattn_quant_fp8 (same codes, same scales,
+ *   bit for bit) that also writes the pooled fp32 block means of x -- steps 1
+ *   and 2 of the selection rule above, same order of additions, same divide --
+ *   into a selection workspace.  key_side: 0 = x is the query tensor, 1 = x is
+ *   the key tensor.  select_workspace: the workspace a later
+ *   sparkattn_select_pooled call takes (>= sparkattn_workspace_bytes(shape, 0,
+ *   topk) bytes, 256-byte aligned); only its pooled-means region is written.
+ * sparkattn_select_pooled: steps 3 to 5 of the selection rule on a workspace
+ *   that one query-side and one key-side call above have filled (same shape,
+ *   same stream order); outputs as sparkattn_select.  The three calls together
+ *   give the same lists as sparkattn_select on the same Q and K.
+ * Plain layout only (no causal window, no per-block token counts).
+ */
+int sparkattn_quant_fp8_pooled(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes, float* scales,
+                               int32_t key_side, void* select_workspace, size_t workspace_bytes, void* cuda_stream);
+int sparkattn_select_pooled(const sparkattn_shape_t* shape, int32_t topk, int32_t* kept_idx, int32_t* kept_cnt,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * Per-token FP8 quantisation: the activation-quantisation kernel at the

@@ -38,6 +38,7 @@ EXPORTS = (
     "sparkattn_select_noalloc_status", "sparkattn_comp_workspace_bytes", "sparkattn_comp_state",
     "sparkattn_comp_apply", "sparkattn_select_window", "sparkattn_fwd_window", "sparkattn_brick_count",
     "sparkattn_brick_layout", "sparkattn_gather_tokens", "sparkattn_select_padded", "sparkattn_fwd_padded",
+    "sparkattn_quant_fp8_pooled", "sparkattn_select_pooled",
 )
 
 
@@ -81,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_select.argtypes = [sp, vp, vp, i32, vp, vp, vp, sz, vp]
         L.sparkattn_quant_fp8.restype = ctypes.c_int
         L.sparkattn_quant_fp8.argtypes = [sp, vp, vp, vp, ctypes.c_uint32, vp]
+        L.sparkattn_quant_fp8_pooled.restype = ctypes.c_int
+        L.sparkattn_quant_fp8_pooled.argtypes = [sp, vp, vp, vp, i32, vp, sz, vp]
+        L.sparkattn_select_pooled.restype = ctypes.c_int
+        L.sparkattn_select_pooled.argtypes = [sp, i32, vp, vp, vp, sz, vp]
         L.sparkattn_quant_fp8_per_token.restype = ctypes.c_int
         L.sparkattn_quant_fp8_per_token.argtypes = [sp, vp, vp, vp, vp]
         L.sparkattn_fwd.restype = ctypes.c_int
@@ -233,6 +238,42 @@ def quant_fp8(x: torch.Tensor, block: int, *, codes: Optional[torch.Tensor] = No
     rc = lib().sparkattn_quant_fp8(ctypes.byref(shape), _ptr(x), _ptr(codes), _ptr(scales), 0, _stream_ptr(stream))
     _check(rc, "sparkattn_quant_fp8")
     return codes, scales
+
+
+def quant_fp8_pooled(x: torch.Tensor, block: int, key_side: bool, select_workspace: torch.Tensor, *,
+                     codes: Optional[torch.Tensor] = None, scales: Optional[torch.Tensor] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_quant_fp8_pooled``: :func:`quant_fp8` that also leaves the pooled block means of ``x`` (the query
+    tensor, or the key tensor with ``key_side``) in ``select_workspace`` for :func:`select_pooled`."""
+    shape = make_shape(x, block)
+    B, H, N, _ = x.shape
+    nb = (N + block - 1) // block
+    if codes is None:
+        codes = torch.empty_strided(x.shape, x.stride(), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty((B, H, nb), dtype=torch.float32, device=x.device)
+    rc = lib().sparkattn_quant_fp8_pooled(ctypes.byref(shape), _ptr(x), _ptr(codes), _ptr(scales), 1 if key_side else 0,
+                                          _ptr(select_workspace), select_workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_quant_fp8_pooled")
+    return codes, scales
+
+
+def select_pooled(ref: torch.Tensor, block: int, topk: int, workspace: torch.Tensor, *,
+                  kept_idx: Optional[torch.Tensor] = None, kept_cnt: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """``sparkattn_select_pooled``: scores + top-k on the pooled means two :func:`quant_fp8_pooled` calls left in
+    ``workspace``; ``ref`` is any [B,H,N,d] tensor of the problem (for the shape)."""
+    shape = make_shape(ref, block)
+    B, H, N, _ = ref.shape
+    nb = (N + block - 1) // block
+    if kept_idx is None:
+        kept_idx = torch.empty((B, H, nb, max(topk, 1)), dtype=torch.int32, device=ref.device)
+    if kept_cnt is None:
+        kept_cnt = torch.empty((B, H, nb), dtype=torch.int32, device=ref.device)
+    rc = lib().sparkattn_select_pooled(ctypes.byref(shape), topk, _ptr(kept_idx), _ptr(kept_cnt), _ptr(workspace),
+                                       workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_select_pooled")
+    return kept_idx, kept_cnt
 
 
 def quant_fp8_per_token(x: torch.Tensor, *, codes: Optional[torch.Tensor] = None,

@@ -111,6 +111,33 @@ int sparkattn_quant_fp8(const sparkattn_shape_t* shape, const void* x_bf16, uint
   return launch_quant_fp8(*shape, x_bf16, codes, scales, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int sparkattn_quant_fp8_pooled(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes, float* scales,
+                               int32_t key_side, void* select_workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!x_bf16 || !codes || !scales || !select_workspace || (key_side != 0 && key_side != 1)) return SPARKATTN_E_INVALID_ARG;
+  if (num_blocks(shape) > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (!aligned16(x_bf16) || !aligned16(codes) || !aligned256(select_workspace)) return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < select_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  return launch_quant_fp8_pooled(*shape, x_bf16, codes, scales, select_pooled_ptr(*shape, select_workspace, key_side != 0),
+                                 key_side != 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int sparkattn_select_pooled(const sparkattn_shape_t* shape, int32_t topk, int32_t* kept_idx, int32_t* kept_cnt,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!kept_idx || !workspace) return SPARKATTN_E_INVALID_ARG;
+  const int nb = num_blocks(shape);
+  if (topk < 1 || topk > nb) return SPARKATTN_E_INVALID_ARG;
+  if (nb > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (!aligned256(workspace)) return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < select_workspace_bytes(*shape)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  return launch_select_pooled(*shape, topk, kept_idx, kept_cnt, workspace, stream);
+}
+
 int sparkattn_quant_fp8_per_token(const sparkattn_shape_t* shape, const void* x_bf16, uint8_t* codes,
                                   float* scales, void* cuda_stream) {
   int rc = check_shape(shape);

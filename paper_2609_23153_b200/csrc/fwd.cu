@@ -496,7 +496,7 @@ int launch_fwd(const sparkattn_shape_t& s, int dtype, const void* q, const void*
   if (fwd_pipe_supported(s))
     return launch_fwd_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
                            block_valid, out, lse, workspace, stream);
-  // d = 128 always runs the persistent kernels; a sequence too long for their list pre-pass is not served
+  // d = 128 always runs the persistent kernel; a sequence too long for its list pre-pass is not served
   if (s.d != 64 || s.block != 64 || fp8 || block_valid != nullptr) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   const int elt = fp8 ? 1 : 2;
   CUtensorMap mq, mk, mv;

@@ -238,6 +238,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   uint64_t* bar_tok = bars + 23;       // [2] 128 arrivals: warpgroup g has published its reference maxima
   uint64_t* bar_lsum = bars + 25;      // 128 arrivals: the non-closing warpgroup has published its row sums
   uint64_t* bar_lsum_ack = bars + 26;  // 128 arrivals: they have been read
+  uint64_t* bar_wg = bars + 27;        // [2] 128 arrivals: line-up of softmax warpgroup g (a named barrier would not be bounded)
   float* s_mref = reinterpret_cast<float*>(bars + 32);           // [2][128]
   float2* s_lsum = reinterpret_cast<float2*>(s_mref + 2 * 128);  // [128] (partial row sum, reference it is relative to)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_lsum + 128);
@@ -262,6 +263,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1);
     }
     mbar_init(bar_o_free, 128); mbar_init(bar_lsum, 128); mbar_init(bar_lsum_ack, 128);
+    mbar_init(bar_wg + 0, 128); mbar_init(bar_wg + 1, 128);
     int dead = (*reinterpret_cast<volatile int32_t*>(p.status) == SPARKATTN_E_DEVICE_TIMEOUT) ? 1 : 0;
     if ((smem_u32(smem) & 1023u) != 0u) {       // the swizzled tiles need a 1024-byte aligned base
       report_status(p.status, SPARKATTN_E_MISALIGNED, (int)(smem_u32(smem) & 1023u));
@@ -487,6 +489,16 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     int nonempty = 0;                                 // non-empty items finished so far
     bool ok = true;
     int io = 0;
+    int wg_syncs = 0;                                 // line-ups of this warpgroup so far (barrier phase)
+    // Line-up of the warpgroup's 128 threads, bounded like every other wait: a warp that has given up (its own
+    // wait expired, or it saw the abort flag) never arrives, and the others then leave through the abort flag
+    // instead of sitting in a hardware barrier for ever.
+    auto wg_line_up = [&](int wait_id) {
+      mbar_arrive(bar_wg + g);
+      const bool r = mbar_wait(bar_wg + g, wg_syncs & 1, s_abort, p.status, wait_id);
+      ++wg_syncs;
+      return __all_sync(0xffffffffu, r) != 0;
+    };
     for (int item = first_item; ok && item < p.items; item += item_step, ++io) {
       const int qslot = io & 1;
       const int cnt = __ldg(p.clean_cnt + item);
@@ -775,13 +787,15 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // next item, with a phase parity counted in items; that is only sound if no thread of this
         // warpgroup runs ahead while the phase its own warpgroup completes is still open (items of one
         // or two tiles make that possible).  So the warpgroup lines up after arriving.
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");
+        ok = wg_line_up(13);
+        if (!ok) break;
       } else {
         ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum, nonempty & 1, s_abort, p.status, 8));
         if (!ok) break;
         const float2 other = s_lsum[row];
         mbar_arrive(bar_lsum_ack);
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");     // see the note at the hand-over above
+        ok = wg_line_up(14);                                            // see the note at the hand-over above
+        if (!ok) break;
         if (other.x != 0.0f) l += other.x * fast_exp2(other.y - m_used);
         ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + (t_last & 1), (t_last >> 1) & 1, s_abort, p.status, 9));
         if (!ok) break;
@@ -812,7 +826,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         mbar_arrive(bar_o_free);
         if (row_valid && p.lse) p.lse[(int64_t)bh * p.N + q_row] = (m_used + log2f(l)) * 0.6931471805599453f;
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");
+        ok = wg_line_up(15);
+        if (!ok) break;
         if (row == 0) {
           pipe_tma_store_4d(&tmap_o, slot, 0, qb * kPBLK, h, b);
           pipe_tma_store_4d(&tmap_o, slot + kTile / 2, 64, qb * kPBLK, h, b);

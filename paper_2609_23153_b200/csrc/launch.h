@@ -14,6 +14,10 @@ namespace sparkattn {
 int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
                      cudaStream_t stream);
 
+// quantisation + the selection's pooled block means in one pass (pooled: see select_pooled_ptr)
+int launch_quant_fp8_pooled(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales, float* pooled,
+                            bool key_side, cudaStream_t stream);
+
 int launch_quant_fp8_per_token(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
                                cudaStream_t stream);
 
@@ -24,6 +28,11 @@ size_t select_workspace_bytes(const sparkattn_shape_t& s);
 // block_valid: real tokens per block when bricks are padded to whole blocks (device int32 [nb]), else NULL
 int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int frame_tokens, int window,
                   const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt, void* workspace, cudaStream_t stream);
+
+// pooled means inside a selection workspace (query side / key side), and scores + top-k on means already there
+float* select_pooled_ptr(const sparkattn_shape_t& s, void* workspace, bool key_side);
+int launch_select_pooled(const sparkattn_shape_t& s, int topk, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                         cudaStream_t stream);
 
 // fwd.cu
 constexpr int kFwdMaxKept = 2048;  // longest kept list (kmax) the forward kernel stages in shared memory

@@ -16,10 +16,17 @@ namespace sparkattn {
 
 constexpr int kQuantThreads = 256;
 
-template <int D, int BLK>
+// POOL: the same pass also produces the block's pooled mean for the selection (Sec. 4.3 fuses scaling and
+// casting into one pass over memory; with the pooling in it as well, Q and K are read from HBM once for
+// selection and quantisation together).  The selection's pooled sum is a chain of fp32 additions over the
+// block's tokens in ascending order, one chain per channel, so it cannot be spread over the threads that hold
+// the rows: the block is parked in shared memory on the way and thread c walks channel c through it while the
+// other warps encode.  pooled: fp32 [B*H][nb][D] (query side) or transposed [B*H][D][nbp] (key side).
+template <int D, int BLK, bool POOL>
 __global__ void __launch_bounds__(kQuantThreads, 3)
 quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ scales,
-                 int H, int N, int nb, int64_t stride_b, int64_t stride_h, int64_t stride_n) {
+                 int H, int N, int nb, int64_t stride_b, int64_t stride_h, int64_t stride_n,
+                 float* __restrict__ pooled, int pooled_transposed, int nbp) {
   constexpr int kChunksPerRow = D / 8;                      // 16-byte chunks per token row
   constexpr int kChunks = BLK * kChunksPerRow;              // chunks per token block
   constexpr int kPerThread = kChunks / kQuantThreads;       // 8 for (128,128), 2 for (64,64)
@@ -43,6 +50,12 @@ quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ code
     } else {
       v[i] = make_uint4(0u, 0u, 0u, 0u);
     }
+  }
+  __shared__ __align__(16) __nv_bfloat16 s_tile[POOL ? BLK * D : 8];
+  if constexpr (POOL) {
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i)
+      reinterpret_cast<uint4*>(s_tile)[threadIdx.x + i * kQuantThreads] = v[i];     // [row][channel], conflict-free
   }
 #pragma unroll
   for (int i = 0; i < kPerThread; ++i) {
@@ -83,6 +96,26 @@ quant_fp8_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ code
       w[j] = lo | (hi << 16);
     }
     *reinterpret_cast<uint2*>(codes + base + (int64_t)(row0 + r) * stride_n + cc * 8) = make_uint2(w[0], w[1]);
+  }
+  if constexpr (POOL) {
+    // (the __syncthreads of the absmax reduction made the tile visible)
+    if (threadIdx.x < D) {
+      const int c = threadIdx.x;
+      float sum = 0.0f;
+      constexpr int U = 8;     // rows fetched ahead of the addition chain
+      int r = 0;
+      for (; r + U <= nvalid; r += U) {
+        float xr[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) xr[u] = __bfloat162float(s_tile[(r + u) * D + c]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) sum = __fadd_rn(sum, xr[u]);
+      }
+      for (; r < nvalid; ++r) sum = __fadd_rn(sum, __bfloat162float(s_tile[r * D + c]));
+      const float mean = __fdiv_rn(sum, (float)nvalid);
+      if (pooled_transposed) pooled[((int64_t)bh * D + c) * nbp + blk] = mean;
+      else pooled[((int64_t)bh * nb + blk) * D + c] = mean;
+    }
   }
 }
 
@@ -184,25 +217,38 @@ int launch_quant_fp8_per_token(const sparkattn_shape_t& s, const void* x, uint8_
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
-int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
-                     cudaStream_t stream) {
+template <bool POOL>
+static int launch_quant_fp8_t(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales, float* pooled,
+                              int pooled_transposed, cudaStream_t stream) {
   const int nb = (s.N + s.block - 1) / s.block;
+  const int nbp = (nb + 31) / 32 * 32;
   const long long ctas = (long long)s.B * s.H * nb;
   if (ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
   if (s.d == 128 && s.block == 128) {
-    quant_fp8_kernel<128, 128><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
-        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
+    quant_fp8_kernel<128, 128, POOL><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n, pooled, pooled_transposed, nbp);
   } else if (s.d == 128 && s.block == 64) {
-    quant_fp8_kernel<128, 64><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
-        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
+    quant_fp8_kernel<128, 64, POOL><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n, pooled, pooled_transposed, nbp);
   } else if (s.d == 64 && s.block == 64) {
-    quant_fp8_kernel<64, 64><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
-        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n);
+    quant_fp8_kernel<64, 64, POOL><<<(unsigned)ctas, kQuantThreads, 0, stream>>>(
+        xb, codes, scales, s.H, s.N, nb, s.stride_b, s.stride_h, s.stride_n, pooled, pooled_transposed, nbp);
   } else {
     return SPARKATTN_E_UNSUPPORTED_SHAPE;
   }
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
+int launch_quant_fp8(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales,
+                     cudaStream_t stream) {
+  return launch_quant_fp8_t<false>(s, x, codes, scales, nullptr, 0, stream);
+}
+
+// pooled: the selection workspace's pooled-Q or pooled-K region (select.cu lays it out)
+int launch_quant_fp8_pooled(const sparkattn_shape_t& s, const void* x, uint8_t* codes, float* scales, float* pooled,
+                            bool key_side, cudaStream_t stream) {
+  return launch_quant_fp8_t<true>(s, x, codes, scales, pooled, key_side ? 1 : 0, stream);
 }
 
 }  // namespace sparkattn

@@ -396,38 +396,66 @@ static int launch_topk(const float* pq, const float* pkT, int32_t* kept_idx, int
   return SPARKATTN_OK;
 }
 
+// Where the pooled means live in a selection workspace: pooled Q [B*H][nb][d] right behind the header, pooled K
+// transposed [B*H][d][nbp] behind it.
+float* select_pooled_ptr(const sparkattn_shape_t& s, void* workspace, bool key_side) {
+  const int nb = (s.N + s.block - 1) / s.block;
+  float* pq = reinterpret_cast<float*>(static_cast<char*>(workspace) + kWorkspaceHeaderBytes);
+  return key_side ? pq + (int64_t)s.B * s.H * nb * s.d : pq;
+}
+
+// scores + top-k on pooled means that are already in the workspace
+static int launch_topk_any(const sparkattn_shape_t& s, int topk, int frame_tokens, int window, int32_t* kept_idx,
+                           int32_t* kept_cnt, void* workspace, cudaStream_t stream) {
+  const int nb = (s.N + s.block - 1) / s.block;
+  const int nbp = round_up(nb, 32);
+  const int64_t bh = (int64_t)s.B * s.H;
+  const float* pq = select_pooled_ptr(s, workspace, false);
+  const float* pkT = select_pooled_ptr(s, workspace, true);
+  // 16 query blocks per CTA while two CTAs' score rows fit one SM's shared memory and the grid still
+  // fills the device several times over (small problems are bound by the latency of one CTA), else 8
+  constexpr int kNumSMs = 148;   // B200; another count only moves the point where the CTAs get smaller
+  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u && bh * ((nb + 15) / 16) >= 6 * kNumSMs;
+  if (s.d == 128)
+    return rows16 ? launch_topk<128, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
+                  : launch_topk<128, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
+  if (s.d == 64)
+    return rows16 ? launch_topk<64, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
+                  : launch_topk<64, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
+  return SPARKATTN_E_UNSUPPORTED_SHAPE;
+}
+
+int launch_select_pooled(const sparkattn_shape_t& s, int topk, int32_t* kept_idx, int32_t* kept_cnt, void* workspace,
+                         cudaStream_t stream) {
+  const int nb = (s.N + s.block - 1) / s.block;
+  if (nb > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  const int rc = launch_topk_any(s, topk, 0, 0, kept_idx, kept_cnt, workspace, stream);
+  if (rc != SPARKATTN_OK) return rc;
+  return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
+}
+
 int launch_select(const sparkattn_shape_t& s, const void* q, const void* k, int topk, int frame_tokens, int window,
                   const int32_t* block_valid, int32_t* kept_idx, int32_t* kept_cnt, void* workspace, cudaStream_t stream) {
   const int nb = (s.N + s.block - 1) / s.block;
   const int nbp = round_up(nb, 32);
   if (nb > kSelectMaxBlocks) return SPARKATTN_E_UNSUPPORTED_SHAPE;
-  const int64_t bh = (int64_t)s.B * s.H;
-  const int64_t n_items = bh * nb;
-  float* pq = reinterpret_cast<float*>(static_cast<char*>(workspace) + kWorkspaceHeaderBytes);
-  float* pkT = pq + n_items * s.d;
+  const int64_t n_items = (int64_t)s.B * s.H * nb;
+  float* pq = select_pooled_ptr(s, workspace, false);
+  float* pkT = select_pooled_ptr(s, workspace, true);
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
-
   const int64_t pool_ctas = (2 * n_items + kPoolThreads / 32 - 1) / (kPoolThreads / 32);
   if (pool_ctas > 0x7fffffffLL) return SPARKATTN_E_UNSUPPORTED_SHAPE;
-  // 16 query blocks per CTA while two CTAs' score rows fit one SM's shared memory and the grid still
-  // fills the device several times over (small problems are bound by the latency of one CTA), else 8
-  constexpr int kNumSMs = 148;   // B200; another count only moves the point where the CTAs get smaller
-  const bool rows16 = (size_t)16 * nbp * sizeof(uint32_t) <= 100u * 1024u && bh * ((nb + 15) / 16) >= 6 * kNumSMs;
-  int rc;
   if (s.d == 128) {
     pool_kernel<128><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items, block_valid);
-    rc = rows16 ? launch_topk<128, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
-                : launch_topk<128, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
   } else if (s.d == 64) {
     pool_kernel<64><<<(unsigned)pool_ctas, kPoolThreads, 0, stream>>>(
         qb, kb, pq, pkT, s.H, s.N, s.block, nb, nbp, s.stride_b, s.stride_h, s.stride_n, n_items, block_valid);
-    rc = rows16 ? launch_topk<64, 16>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream)
-                : launch_topk<64, 8>(pq, pkT, kept_idx, kept_cnt, nb, nbp, topk, bh, s.N, s.block, frame_tokens, window, stream);
   } else {
     return SPARKATTN_E_UNSUPPORTED_SHAPE;
   }
+  const int rc = launch_topk_any(s, topk, frame_tokens, window, kept_idx, kept_cnt, workspace, stream);
   if (rc != SPARKATTN_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }

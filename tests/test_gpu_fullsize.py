@@ -92,6 +92,25 @@ def test_fullsize_fp8_quant_and_fwd():
     assert torch.isfinite(out.float()).all()
 
 
+def test_fullsize_fused_quant_pool_select_matches_separate_calls(wan14b_inputs):
+    """The 40-head 75,600-token shape through the fused chain the benchmark's FP8 leg times (quantise + pool Q,
+    quantise + pool K, scores + top-k on the pooled means): codes, scales and kept lists identical to the
+    separate calls, which the other tests compare with the oracle."""
+    w, (q, k, v), cs, host = wan14b_inputs
+    ws = sa.alloc_workspace(sa.make_shape(q, w.block), 0, w.topk, DEV)
+    cq, sq = sa.quant_fp8_pooled(q, w.block, False, ws)
+    ck, sk = sa.quant_fp8_pooled(k, w.block, True, ws)
+    idx, cnt = sa.select_pooled(q, w.block, w.topk, ws)
+    assert sa.read_status(ws) == sa.OK
+    ridx, rcnt = sa.select(q, k, w.block, w.topk)
+    assert torch.equal(idx, ridx) and torch.equal(cnt, rcnt)
+    assert torch.equal(cq, cs[0][0]) and torch.equal(ck, cs[1][0])
+    assert torch.equal(sq.view(torch.int32), cs[0][1].view(torch.int32)) and torch.equal(sk.view(torch.int32), cs[1][1].view(torch.int32))
+    heads = SWEEP_HEADS
+    ref_idx, _ = oracle.select(*host["bf16"][:2], w.block, w.topk)
+    assert torch.equal(idx[0, heads].cpu(), ref_idx)
+
+
 def test_host_buffer_call_matches_device_call():
     w = workloads.WAN_1P3B_480P.with_heads(2)
     q, k, v = workloads.structured_qkv(w)

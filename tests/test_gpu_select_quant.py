@@ -178,3 +178,59 @@ def test_per_token_quant_strided_and_fullsize_sample():
     for h in (0, 11):
         rc, rs = oracle.quant_fp8_per_token(q[0, h:h + 1].cpu())
         assert torch.equal(codes[0, h:h + 1].cpu(), rc) and torch.equal(scales[0, h:h + 1].cpu().view(torch.int32), rs.view(torch.int32))
+
+
+def _pooled_from_workspace(ws, H, nb, d):
+    """Pooled Q [H, nb, d] and pooled K [H, nb, d] out of a selection workspace (B = 1): pooled Q sits right
+    behind the 256-byte header, pooled K transposed [H, d, nbp] (nbp = nb rounded up to 32) behind it."""
+    nbp = (nb + 31) // 32 * 32
+    f = ws[256:].view(torch.float32).cpu()
+    pq = f[: H * nb * d].reshape(H, nb, d)
+    pk = f[H * nb * d: H * nb * d + H * d * nbp].reshape(H, d, nbp)[:, :, :nb].transpose(1, 2).contiguous()
+    return pq, pk
+
+
+@pytest.mark.parametrize("w", _small_cases(), ids=lambda w: f"{w.name}-N{w.N}-d{w.d}")
+def test_quant_with_pooling_and_select_from_pooled_match_oracle(w):
+    """One pass over Q and one over K give codes, scales AND the selection's pooled means (same order of
+    additions as the selection's own pooling: bit-exact against oracle.pool); scores + top-k on those means
+    give the oracle's lists."""
+    q, k, _ = workloads.structured_qkv(w)
+    qd, kd = q.to(DEV), k.to(DEV)
+    ws = sa.alloc_workspace(sa.make_shape(qd, w.block), 0, w.topk, DEV)
+    ws.fill_(0x5A)                                           # stale contents must not matter
+    cq, sq = sa.quant_fp8_pooled(qd, w.block, False, ws)
+    ck, sk = sa.quant_fp8_pooled(kd, w.block, True, ws)
+    for (codes, scales), x in (((cq, sq), q), ((ck, sk), k)):
+        rc, rs = oracle.quant_fp8(x[0], w.block)
+        assert torch.equal(codes[0].cpu(), rc)
+        assert torch.equal(scales[0].cpu().view(torch.int32), rs.view(torch.int32))
+    torch.cuda.synchronize()
+    pq, pk = _pooled_from_workspace(ws, w.H, w.nb, w.d)
+    assert torch.equal(pq.view(torch.int32), oracle.pool(q[0], w.block).view(torch.int32))
+    assert torch.equal(pk.view(torch.int32), oracle.pool(k[0], w.block).view(torch.int32))
+    for topk in sorted({1, w.topk, w.nb}):
+        idx, cnt = sa.select_pooled(qd, w.block, topk, ws)
+        ref_idx, ref_cnt = oracle.select(q[0], k[0], w.block, topk)
+        assert sa.read_status(ws) == sa.OK
+        assert torch.equal(idx[0].cpu(), ref_idx) and torch.equal(cnt[0].cpu(), ref_cnt)
+
+
+def test_quant_with_pooling_strided_batch_equals_separate_calls():
+    """[B, N, H, d] buffers viewed as [B, H, N, d], two batch entries: the fused pass must reproduce the separate
+    sparkattn_quant_fp8 / sparkattn_select calls bit for bit."""
+    H, d, block, topk = 3, 128, 128, 2
+    g = torch.Generator().manual_seed(21)
+    q = torch.randn((2, 700, H, d), generator=g).to(torch.bfloat16).to(DEV).permute(0, 2, 1, 3)
+    k = torch.randn((2, 700, H, d), generator=g).to(torch.bfloat16).to(DEV).permute(0, 2, 1, 3)
+    ws = sa.alloc_workspace(sa.make_shape(q, block), 0, topk, DEV)
+    cq, sq = sa.quant_fp8_pooled(q, block, False, ws)
+    ck, sk = sa.quant_fp8_pooled(k, block, True, ws)
+    idx, cnt = sa.select_pooled(q, block, topk, ws)
+    rq, rsq = sa.quant_fp8(q, block)
+    rk, rsk = sa.quant_fp8(k, block)
+    ridx, rcnt = sa.select(q, k, block, topk)
+    assert cq.stride() == q.stride()
+    assert torch.equal(cq, rq) and torch.equal(ck, rk)
+    assert torch.equal(sq.view(torch.int32), rsq.view(torch.int32)) and torch.equal(sk.view(torch.int32), rsk.view(torch.int32))
+    assert torch.equal(idx, ridx) and torch.equal(cnt, rcnt)

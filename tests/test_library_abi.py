@@ -147,6 +147,22 @@ def test_argument_errors_are_caught_on_the_host(lib):
     assert lib.sparkattn_comp_workspace_bytes(ctypes.byref(s128), grid) > 256
 
 
+def test_fused_quant_pool_entry_points_validate_on_the_host(lib):
+    s = _shape()
+    fake = ctypes.c_void_p(0x1000)
+    null = ctypes.c_void_p(0)
+    st = ctypes.c_void_p(0)
+    need = sa.workspace_bytes(s, 0, 4)
+    assert lib.sparkattn_quant_fp8_pooled(ctypes.byref(s), fake, fake, fake, 2, fake, need, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_quant_fp8_pooled(ctypes.byref(s), fake, fake, fake, 0, null, need, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_quant_fp8_pooled(ctypes.byref(s), fake, fake, fake, 1, fake, need - 1, st) == sa.E_WORKSPACE_TOO_SMALL
+    assert lib.sparkattn_quant_fp8_pooled(ctypes.byref(s), fake, fake, fake, 1, ctypes.c_void_p(0x1010), need, st) == sa.E_MISALIGNED
+    assert lib.sparkattn_select_pooled(ctypes.byref(s), 0, fake, null, fake, need, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_select_pooled(ctypes.byref(s), 33, fake, null, fake, need, st) == sa.E_INVALID_ARG
+    assert lib.sparkattn_select_pooled(ctypes.byref(s), 4, fake, null, fake, 16, st) == sa.E_WORKSPACE_TOO_SMALL
+    assert lib.sparkattn_select_pooled(ctypes.byref(_shape(d=96)), 4, fake, null, fake, need, st) == sa.E_UNSUPPORTED_SHAPE
+
+
 def test_binding_checks_layout():
     q = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16)
     with pytest.raises(ValueError):
