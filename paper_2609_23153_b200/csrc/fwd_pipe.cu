@@ -47,7 +47,7 @@ constexpr float kPipeLazyLog2 = 8.0f;        // bf16: P may exceed 1 by up to 2^
 constexpr float kPipeFp8LazyLog2 = 4.0f, kPipeFp8PScaleLog2 = 4.0f;
 constexpr int kTile = 32768;                               // bytes of one 128 x 128 bf16 tile (two 64-column slabs)
 constexpr int kOffQ = 0, kOffK = 2 * kTile, kOffV = 4 * kTile, kOffMisc = 7 * kTile;
-constexpr int kPipeSmem = kOffMisc + 256 /*barriers*/ + 2 * 128 * 4 /*reference maxima*/ + 128 * 8 /*row sums*/ + 64;
+constexpr int kPipeSmem = kOffMisc + 512 /*barriers*/ + 2 * 128 * 4 /*reference maxima*/ + 128 * 8 /*row sums*/ + 64;
 
 struct PipeParams {
   const int32_t* clean_cnt;    // [items] valid kept blocks per item
@@ -226,10 +226,14 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffMisc);
   uint64_t* bar_q_full = bars + 0;     // [2]
   uint64_t* bar_q_free = bars + 2;     // [2] the item's output store has read the slot (or the item was empty)
-  uint64_t* bar_k_full = bars + 4;     // [2]
-  uint64_t* bar_k_free = bars + 6;     // [2] S MMAs that read the slot are complete
-  uint64_t* bar_v_full = bars + 8;     // [3]
-  uint64_t* bar_v_free = bars + 11;    // [3] PV MMAs that read the slot are complete
+  // An input tile is 128 rows x 128 channels: two 64-channel slabs of 16 KB in bf16, one slab in FP8, where the
+  // same bytes hold rings twice as deep (the Q slots keep their 32 KB: the item's output is staged there).
+  constexpr int kSlot = FP8 ? kTile / 2 : kTile;
+  constexpr int RK = FP8 ? 4 : 2, RV = FP8 ? 6 : 3;
+  uint64_t* bar_k_full = bars + 32;           // [RK]
+  uint64_t* bar_k_free = bar_k_full + RK;     // [RK] S MMAs that read the slot are complete
+  uint64_t* bar_v_full = bar_k_free + RK;     // [RV]
+  uint64_t* bar_v_free = bar_v_full + RV;     // [RV] PV MMAs that read the slot are complete
   uint64_t* bar_s_full = bars + 14;    // [2] S of a tile complete in S buffer (tile & 1)
   uint64_t* bar_s_free = bars + 16;    // [2] 128 arrivals: the warpgroup holds that S row in registers
   uint64_t* bar_p_full = bars + 18;    // [2] 128 arrivals: P written to P buffer (tile & 1)
@@ -238,15 +242,12 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   uint64_t* bar_tok = bars + 23;       // [2] 128 arrivals: warpgroup g has published its reference maxima
   uint64_t* bar_lsum = bars + 25;      // 128 arrivals: the non-closing warpgroup has published its row sums
   uint64_t* bar_lsum_ack = bars + 26;  // 128 arrivals: they have been read
-  uint64_t* bar_wg = bars + 27;        // [2] 128 arrivals: line-up of softmax warpgroup g (a named barrier would not be bounded)
-  float* s_mref = reinterpret_cast<float*>(bars + 32);           // [2][128]
+  float* s_mref = reinterpret_cast<float*>(bars + 64);           // [2][128]
   float2* s_lsum = reinterpret_cast<float2*>(s_mref + 2 * 128);  // [128] (partial row sum, reference it is relative to)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_lsum + 128);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // An input tile is 128 rows x 128 channels: two 64-channel slabs of 16 KB in bf16, one slab in FP8
-  // (the slots keep their 32 KB stride).
   constexpr int kTileTx = FP8 ? kTile / 2 : kTile;
   constexpr int kEnt = PAIR ? 2 : 1;              // list entries per tile
   constexpr int kKeyBlk = PAIR ? 64 : 128;        // tokens per key block
@@ -254,16 +255,13 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_q_full + i, 1); mbar_init(bar_q_free + i, 1);
-      mbar_init(bar_k_full + i, 1); mbar_init(bar_k_free + i, 1);
       mbar_init(bar_tok + i, 128);
       mbar_init(bar_s_full + i, 1); mbar_init(bar_s_free + i, 128);
       mbar_init(bar_p_full + i, 128); mbar_init(bar_pv_done + i, 1);
     }
-    for (int i = 0; i < 3; ++i) {
-      mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1);
-    }
+    for (int i = 0; i < RK; ++i) { mbar_init(bar_k_full + i, 1); mbar_init(bar_k_free + i, 1); }
+    for (int i = 0; i < RV; ++i) { mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1); }
     mbar_init(bar_o_free, 128); mbar_init(bar_lsum, 128); mbar_init(bar_lsum_ack, 128);
-    mbar_init(bar_wg + 0, 128); mbar_init(bar_wg + 1, 128);
     int dead = (*reinterpret_cast<volatile int32_t*>(p.status) == SPARKATTN_E_DEVICE_TIMEOUT) ? 1 : 0;
     if ((smem_u32(smem) & 1023u) != 0u) {       // the swizzled tiles need a 1024-byte aligned base
       report_status(p.status, SPARKATTN_E_MISALIGNED, (int)(smem_u32(smem) & 1023u));
@@ -292,109 +290,76 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   if (warp < 4) reg_dec<kPipeCtrlRegs>();
   if (dead) {
     // fall through to the teardown
-  } else if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (one thread)
-    // A K cursor (which also loads Q at the start of an item) and a V cursor walk the same tile
-    // stream; each step tests the barriers both may need back to back and then issues what is
-    // ready.  List entries and item counts are fetched one step ahead of their use.
+  } else if (warp == 0 || warp == 3) {
+    // ------------------------------------------------------------ TMA producers: warp 0 Q + the K ring, warp 3 the V ring
+    // One thread each, walking the CTA's tile stream across item boundaries.  A producer only ever waits for
+    // one thing, the release of the slot it fills next, so it sleeps in that barrier wait (a loop polling
+    // several barriers with a back-off reacts to a freed slot up to a microsecond late, which is exposed
+    // latency on a two-slot ring).  List entries and item counts are fetched one step ahead of their use.
     if (lane == 0) {
-      struct Cursor {
-        int ord, item, n, cnt, t;       // item ordinal, item, tile within the item, valid tiles, global tile counter
-        int kb, kb2, cnt_next, kb_next_item, kb2_next_item; // prefetched: this tile's block(s), next item's count and first block(s)
-        bool open;
-      };
-      auto prefetch_item = [&](Cursor& c) {
-        const int nxt = c.item + item_step;
-        c.cnt_next = nxt < p.items ? __ldg(p.clean_cnt + nxt) : 0;
-        c.kb_next_item = nxt < p.items ? __ldg(p.clean_list + (int64_t)nxt * p.lstride) : 0;
-        c.kb2_next_item = (PAIR && nxt < p.items) ? __ldg(p.clean_list + (int64_t)nxt * p.lstride + 1) : 0;
-      };
-      auto init = [&](Cursor& c) {
-        c.ord = 0; c.item = first_item; c.n = 0; c.t = 0; c.open = false;
-        c.cnt = c.item < p.items ? __ldg(p.clean_cnt + c.item) : 0;
-        c.kb = c.item < p.items ? __ldg(p.clean_list + (int64_t)c.item * p.lstride) : 0;
-        c.kb2 = (PAIR && c.item < p.items) ? __ldg(p.clean_list + (int64_t)c.item * p.lstride + 1) : 0;
-        prefetch_item(c);
-      };
-      auto next_item = [&](Cursor& c) {
-        c.item += item_step; ++c.ord; c.n = 0; c.open = false;
-        c.cnt = c.cnt_next; c.kb = c.kb_next_item; c.kb2 = c.kb2_next_item;
-        if (c.item < p.items) prefetch_item(c);
-      };
-      auto next_tile = [&](Cursor& c) {
-        ++c.n; ++c.t;
-        if (c.n < c.cnt) {             // used one step later
-          c.kb = __ldg(p.clean_list + (int64_t)c.item * p.lstride + c.n * kEnt);
-          if constexpr (PAIR) c.kb2 = __ldg(p.clean_list + (int64_t)c.item * p.lstride + c.n * kEnt + 1);
-        }
-      };
-      // one K or V tile: 128 key rows of one block, or 64 + 64 rows of the tile's two 64-token blocks
-      auto load_kv = [&](unsigned char* slot, const CUtensorMap* map, uint64_t* bar, const Cursor& c) {
-        const int bh = c.item / p.nbq;
-        const int hh = bh % p.H, bb = bh / p.H;
-        mbar_expect_tx(bar, kTileTx);
-        if constexpr (PAIR) {
-          const int r0 = (c.kb & 0x3fffffff) * 64, r1 = (c.kb2 & 0x3fffffff) * 64;
-          tma_load_4d(slot, map, bar, 0, r0, hh, bb);
-          tma_load_4d(slot + 8192, map, bar, 0, r1, hh, bb);
-          if constexpr (!FP8) {
-            tma_load_4d(slot + kTile / 2, map, bar, 64, r0, hh, bb);
-            tma_load_4d(slot + kTile / 2 + 8192, map, bar, 64, r1, hh, bb);
-          }
-        } else {
-          tma_load_4d(slot, map, bar, 0, c.kb * kPBLK, hh, bb);
-          if constexpr (!FP8) tma_load_4d(slot + kTile / 2, map, bar, 64, c.kb * kPBLK, hh, bb);
-        }
-      };
-      Cursor kc, vc;
-      init(kc);
-      init(vc);
+      const bool is_v = warp == 3;
+      unsigned char* ring = is_v ? sV : sK;
+      const CUtensorMap* map = is_v ? &tmap_v : &tmap_k;
+      uint64_t* bar_full = is_v ? bar_v_full : bar_k_full;
+      uint64_t* bar_free = is_v ? bar_v_free : bar_k_free;
+      const int R = is_v ? RV : RK;
+      int ord = 0, t = 0;                               // items seen, tiles loaded so far
+      int item = first_item;
+      int cnt = item < p.items ? __ldg(p.clean_cnt + item) : 0;
+      int kb = item < p.items ? __ldg(p.clean_list + (int64_t)item * p.lstride) : 0;
+      int kb2 = (PAIR && item < p.items) ? __ldg(p.clean_list + (int64_t)item * p.lstride + 1) : 0;
       bool ok = true;
-      PipeIdle guard;
-      guard.reset();
-      while (ok && (kc.item < p.items || vc.item < p.items)) {
-        bool progressed = false;
-        const int qslot = kc.ord & 1, kslot = kc.t & 1, vslot = vc.t % 3;
-        const bool qf = kc.ord < 2 ? true : mbar_test(bar_q_free + qslot, ((kc.ord >> 1) - 1) & 1);
-        const bool kf = kc.t < 2 ? true : mbar_test(bar_k_free + kslot, ((kc.t >> 1) - 1) & 1);
-        const bool vf = vc.t < 3 ? true : mbar_test(bar_v_free + vslot, ((vc.t / 3) - 1) & 1);
-        if (kc.item < p.items) {
-          if (!kc.open) {
-            if (qf) {
-              if (kc.cnt > 0) {
-                const int qb = kc.item % p.nbq, bh = kc.item / p.nbq;
-                mbar_expect_tx(bar_q_full + qslot, kTileTx);
-                tma_load_4d(sQ + qslot * kTile, &tmap_q, bar_q_full + qslot, 0, qb * kPBLK, bh % p.H, bh / p.H);
-                if constexpr (!FP8)
-                  tma_load_4d(sQ + qslot * kTile + kTile / 2, &tmap_q, bar_q_full + qslot, 64, qb * kPBLK, bh % p.H, bh / p.H);
-                kc.open = true;
-              } else {
-                mbar_arrive(bar_q_full + qslot);      // empty item: nothing to load, consumers still step through it
-                next_item(kc);
-              }
-              progressed = true;
+      while (ok && item < p.items) {
+        // the next item's count and first entries, needed when this item is done
+        const int nxt = item + item_step;
+        const int cnt_next = nxt < p.items ? __ldg(p.clean_cnt + nxt) : 0;
+        const int kb_next = nxt < p.items ? __ldg(p.clean_list + (int64_t)nxt * p.lstride) : 0;
+        const int kb2_next = (PAIR && nxt < p.items) ? __ldg(p.clean_list + (int64_t)nxt * p.lstride + 1) : 0;
+        const int bh = item / p.nbq;
+        const int hh = bh % p.H, bb = bh / p.H;
+        if (!is_v) {
+          const int qslot = ord & 1;
+          if (cnt > 0) {
+            if (ord >= 2) ok = mbar_wait(bar_q_free + qslot, ((ord >> 1) - 1) & 1, s_abort, p.status, 1);
+            if (!ok) break;
+            const int qb = item % p.nbq;
+            mbar_expect_tx(bar_q_full + qslot, kTileTx);
+            tma_load_4d(sQ + qslot * kTile, &tmap_q, bar_q_full + qslot, 0, qb * kPBLK, hh, bb);
+            if constexpr (!FP8) tma_load_4d(sQ + qslot * kTile + kTile / 2, &tmap_q, bar_q_full + qslot, 64, qb * kPBLK, hh, bb);
+          } else {
+            mbar_arrive(bar_q_full + qslot);            // empty item: nothing to load, consumers still step through it
+          }
+        }
+        for (int n = 0; ok && n < cnt; ++n, ++t) {
+          const int slot = t % R;
+          // the entries of the tile after this one (used one step later)
+          int kb_n = 0, kb2_n = 0;
+          if (n + 1 < cnt) {
+            kb_n = __ldg(p.clean_list + (int64_t)item * p.lstride + (n + 1) * kEnt);
+            if constexpr (PAIR) kb2_n = __ldg(p.clean_list + (int64_t)item * p.lstride + (n + 1) * kEnt + 1);
+          }
+          if (t >= R) ok = mbar_wait(bar_free + slot, ((t / R) - 1) & 1, s_abort, p.status, is_v ? 16 : 1);
+          if (!ok) break;
+          unsigned char* dst = ring + slot * kSlot;
+          uint64_t* bar = bar_full + slot;
+          mbar_expect_tx(bar, kTileTx);
+          // one K or V tile: 128 key rows of one block, or 64 + 64 rows of the tile's two 64-token blocks
+          if constexpr (PAIR) {
+            const int r0 = (kb & 0x3fffffff) * 64, r1 = (kb2 & 0x3fffffff) * 64;
+            tma_load_4d(dst, map, bar, 0, r0, hh, bb);
+            tma_load_4d(dst + 8192, map, bar, 0, r1, hh, bb);
+            if constexpr (!FP8) {
+              tma_load_4d(dst + kTile / 2, map, bar, 64, r0, hh, bb);
+              tma_load_4d(dst + kTile / 2 + 8192, map, bar, 64, r1, hh, bb);
             }
-          } else if (kc.n >= kc.cnt) {
-            next_item(kc);
-            progressed = true;
-          } else if (kf) {
-            load_kv(sK + kslot * kTile, &tmap_k, bar_k_full + kslot, kc);
-            next_tile(kc);
-            progressed = true;
+          } else {
+            tma_load_4d(dst, map, bar, 0, kb * kPBLK, hh, bb);
+            if constexpr (!FP8) tma_load_4d(dst + kTile / 2, map, bar, 64, kb * kPBLK, hh, bb);
           }
+          kb = kb_n; kb2 = kb2_n;
         }
-        if (vc.item < p.items) {
-          if (vc.n >= vc.cnt) {
-            // the V cursor never passes the K cursor's item
-            if (vc.ord < kc.ord) { next_item(vc); progressed = true; }
-          } else if (vc.t < kc.t && vf) {
-            load_kv(sV + vslot * kTile, &tmap_v, bar_v_full + vslot, vc);
-            next_tile(vc);
-            progressed = true;
-          }
-        }
-        if (progressed) guard.reset();
-        else ok = guard.idle(s_abort, p.status, 1);
+        item = nxt; ++ord;
+        cnt = cnt_next; kb = kb_next; kb2 = kb2_next;
       }
     }
   } else if (warp == 1) {
@@ -411,16 +376,29 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           s_item += item_step; ++si; s_n = 0; s_cnt = -1;
           continue;
         }
-        // polled back to back: a poll is a shared-memory round trip
-        const int sbuf = s_t & 1, kslot = s_t & 1, qslot = si & 1;
+        const int sbuf = s_t & 1, kslot = s_t % RK, qslot = si & 1;
+        const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ + qslot * kTile), 16);
+        const uint64_t dK = make_smem_desc_sw128(smem_u32(sK + kslot * kSlot), 16);
+        const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32), k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
+#ifndef PIPE_POLLING_ISSUE
+        // The product needs all three (its S buffer free, K landed, Q landed), so the thread sleeps in one barrier
+        // wait after the other instead of polling them with a back-off: the K tile, which is waited for longest,
+        // comes first; the others have normally happened by then.
+        ok = mbar_wait(bar_k_full + kslot, (s_t / RK) & 1, s_abort, p.status, 2);
+        if (ok && s_n == 0) ok = mbar_wait(bar_q_full + qslot, (si >> 1) & 1, s_abort, p.status, 17);
+        if (ok && s_t >= 2) ok = mbar_wait(bar_s_free + sbuf, ((s_t >> 1) - 1) & 1, s_abort, p.status, 18);   // row of tile s_t - 2 is in registers
+        if (!ok) break;
+        {
+#else
         const bool pd = s_t < 2 ? true : mbar_test(bar_s_free + sbuf, ((s_t >> 1) - 1) & 1);   // S buffer free: row of tile s_t - 2 is in registers
-        const bool kf = mbar_test(bar_k_full + kslot, (s_t >> 1) & 1);
+        const bool kf = mbar_test(bar_k_full + kslot, (s_t / RK) & 1);
         const bool qf = s_n > 0 ? true : mbar_test(bar_q_full + qslot, (si >> 1) & 1);
-        if (pd && kf && qf) {
+        if (!(pd && kf && qf)) {
+          ok = guard.idle(s_abort, p.status, 2);
+        } else {
+          guard.reset();
+#endif
           tc_fence_after();
-          const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ + qslot * kTile), 16);
-          const uint64_t dK = make_smem_desc_sw128(smem_u32(sK + kslot * kTile), 16);
-          const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32), k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
           // 32 bytes of the channel dimension per MMA: 16 bf16 (8 MMAs over two slabs) or 32 E4M3 (4 MMAs)
 #pragma unroll
           for (int sl = 0; sl < (FP8 ? 1 : 2); ++sl)
@@ -431,9 +409,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           tc_commit(bar_s_full + sbuf);
           tc_commit(bar_k_free + kslot);
           ++s_n; ++s_t;
-          guard.reset();
-        } else {
-          ok = guard.idle(s_abort, p.status, 2);
         }
       }
     }
@@ -455,15 +430,28 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           p_item += item_step; p_n = 0; p_cnt = -1;
           continue;
         }
-        const int pbuf = p_t & 1, vslot = p_t % 3;
+        const int pbuf = p_t & 1, vslot = p_t % RV;
+        const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + vslot * kSlot), kTile / 2);
+        const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
+#ifndef PIPE_POLLING_ISSUE
+        // (see the S issuer) the V tile and the previous item's closer first, P, which arrives last, last
+        ok = mbar_wait(bar_v_full + vslot, (p_t / RV) & 1, s_abort, p.status, 10);
+        // first tile of an item only: O of the previous item must have been read by its closer
+        if (ok && p_n == 0 && p_nonempty > 0) ok = mbar_wait(bar_o_free, (p_nonempty - 1) & 1, s_abort, p.status, 19);
+        if (ok) ok = mbar_wait(bar_p_full + pbuf, (p_t >> 1) & 1, s_abort, p.status, 20);
+        if (!ok) break;
+        {
+#else
         const bool pf = mbar_test(bar_p_full + pbuf, (p_t >> 1) & 1);
-        const bool vf = mbar_test(bar_v_full + vslot, (p_t / 3) & 1);
+        const bool vf = mbar_test(bar_v_full + vslot, (p_t / RV) & 1);
         // first tile of an item only: O of the previous item must have been read by its closer
         const bool of = (p_n > 0 || p_nonempty == 0) ? true : mbar_test(bar_o_free, (p_nonempty - 1) & 1);
-        if (pf && vf && of) {
+        if (!(pf && vf && of)) {
+          ok = guard.idle(s_abort, p.status, 10);
+        } else {
+          guard.reset();
+#endif
           tc_fence_after();
-          const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + vslot * kTile), kTile / 2);
-          const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
 #pragma unroll
           for (int kk = 0; kk < kPvSteps; ++kk)
             mma_ts<FP8>(tmem_O, tmem_P + pbuf * 64 + kk * 8, make_desc(v_lo + ((kk * (128 / kPvSteps) * 128) >> 4), v_hi),
@@ -471,9 +459,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           tc_commit(bar_pv_done + pbuf);
           tc_commit(bar_v_free + vslot);
           ++p_n; ++p_t;
-          guard.reset();
-        } else {
-          ok = guard.idle(s_abort, p.status, 10);
         }
       }
     }
@@ -489,15 +474,14 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     int nonempty = 0;                                 // non-empty items finished so far
     bool ok = true;
     int io = 0;
-    int wg_syncs = 0;                                 // line-ups of this warpgroup so far (barrier phase)
-    // Line-up of the warpgroup's 128 threads, bounded like every other wait: a warp that has given up (its own
-    // wait expired, or it saw the abort flag) never arrives, and the others then leave through the abort flag
-    // instead of sitting in a hardware barrier for ever.
-    auto wg_line_up = [&](int wait_id) {
-      mbar_arrive(bar_wg + g);
-      const bool r = mbar_wait(bar_wg + g, wg_syncs & 1, s_abort, p.status, wait_id);
-      ++wg_syncs;
-      return __all_sync(0xffffffffu, r) != 0;
+    // Line-up of the warpgroup's 128 threads on a named barrier.  A hardware barrier has no time limit, so it
+    // is fenced by the abort flag: no warp enters it once the flag is up, and a warp that leaves its loop
+    // early arrives once on its way out, which releases the warps that were already inside (every other warp
+    // either is inside or will see the flag and arrive as well: the 128 arrivals always come together).
+    auto wg_line_up = [&](int) {
+      if (*s_abort) return false;
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");
+      return true;
     };
     for (int item = first_item; ok && item < p.items; item += item_step, ++io) {
       const int qslot = io & 1;
@@ -839,6 +823,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       t += cnt;
       ++nonempty;
     }
+    if (!ok) asm volatile("bar.arrive %0, 128;" ::"r"(1 + g) : "memory");   // see wg_line_up
     if (row == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
