@@ -17,14 +17,17 @@
 //                    warpgroup keeps its own partial row sum relative to the last reference it
 //                    saw; the warpgroup of the item's last tile combines them, normalises O into
 //                    the item's (now dead) Q slot and stores it with one TMA copy.
-//   warp 0           TMA producer: Q (2 slots), K ring (2), V ring (3), across item boundaries.
-//   warp 1           S issuer, polling: S = Q K^T of the next tile whose K has landed and whose S
-//                    buffer is free (PV of the tile three back complete).
-//   warp 2           PV issuer, polling: O += P V of the oldest tile whose P is written.
+//   warp 0           TMA producer (one thread): Q (2 slots) and the K ring (2 slots; FP8: 4).
+//   warp 3           TMA producer (one thread): the V ring (3 slots; FP8: 6).  Each producer sleeps in
+//                    the wait for the slot it fills next (one thread polling all rings with a
+//                    back-off answered a freed slot up to a microsecond late).
+//   warp 1           S issuer: S = Q K^T of the next tile once its K has landed and its S buffer is
+//                    free (the warpgroup holds the row of the tile two back in registers).
+//   warp 2           PV issuer: O += P V of the oldest tile once its P is written.
 //                    Two issuing warps on two schedulers: an issuing thread shares its scheduler
 //                    with two softmax warps that are almost always ready and only gets an issue
 //                    slot when they stall, so its instruction count per tile is what matters.
-//   warp 3           idle (completes the first warpgroup for the register hand-over).
+//                    Both sleep in their barrier waits (everything a product needs is needed).
 // Work items (batch, head, query block) go to CTA c as c, c + grid, ... in head-major order, so
 // the CTAs running together read K/V of one head from L2.  Kept lists are range-checked and
 // compacted by a small pre-pass into the workspace; every role reads the clean lists from there.
@@ -193,26 +196,6 @@ __device__ __forceinline__ void pipe_tma_store_4d(const void* tmap, const void* 
       : "memory");
 }
 
-struct PipeIdle {
-  uint64_t t0;
-  uint32_t polls;
-  __device__ __forceinline__ void reset() { polls = 0; }
-  // Nothing was ready: yield the issue slots to the softmax warps of this scheduler for a moment.
-  __device__ __forceinline__ bool idle(volatile int* abort_flag, int32_t* status, int wait_id) {
-    if (polls == 0) t0 = global_timer_ns();
-    __nanosleep(32);
-    if ((++polls & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        report_status(status, SPARKATTN_E_DEVICE_TIMEOUT, wait_id);
-        return false;
-      }
-    }
-    return true;
-  }
-};
-
 // PAIR: 64-token blocks; a work item is a pair of query blocks, a tile two key blocks (see pair_lists_kernel).
 template <bool FP8, bool WINDOW, bool PAIR>
 __global__ void __launch_bounds__(kPipeThreads, 1)
@@ -222,14 +205,14 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sQ = smem + kOffQ;
   unsigned char* sK = smem + kOffK;
-  unsigned char* sV = smem + kOffV;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kOffMisc);
   uint64_t* bar_q_full = bars + 0;     // [2]
   uint64_t* bar_q_free = bars + 2;     // [2] the item's output store has read the slot (or the item was empty)
   // An input tile is 128 rows x 128 channels: two 64-channel slabs of 16 KB in bf16, one slab in FP8, where the
   // same bytes hold rings twice as deep (the Q slots keep their 32 KB: the item's output is staged there).
   constexpr int kSlot = FP8 ? kTile / 2 : kTile;
-  constexpr int RK = FP8 ? 4 : 2, RV = FP8 ? 6 : 3;
+  constexpr int RK = FP8 ? 4 : 2, RV = FP8 ? 6 : 3;    // (K 3 / V 2 measures the same)
+  unsigned char* sV = sK + RK * kSlot;         // the V ring follows the K ring (5 x 32 KB between them)
   uint64_t* bar_k_full = bars + 32;           // [RK]
   uint64_t* bar_k_free = bar_k_full + RK;     // [RK] S MMAs that read the slot are complete
   uint64_t* bar_v_full = bar_k_free + RK;     // [RV]
@@ -368,8 +351,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       constexpr uint32_t idesc_qk = make_idesc(FP8 ? 0u : 1u, 128, kPBLK, false);
       int si = 0, s_item = first_item, s_n = 0, s_cnt = -1, s_t = 0;
       bool ok = true;
-      PipeIdle guard;
-      guard.reset();
       while (ok && s_item < p.items) {
         if (s_cnt < 0) s_cnt = __ldg(p.clean_cnt + s_item);
         if (s_n >= s_cnt) {
@@ -380,7 +361,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint64_t dQ = make_smem_desc_sw128(smem_u32(sQ + qslot * kTile), 16);
         const uint64_t dK = make_smem_desc_sw128(smem_u32(sK + kslot * kSlot), 16);
         const uint32_t q_lo = (uint32_t)dQ, q_hi = (uint32_t)(dQ >> 32), k_lo = (uint32_t)dK, k_hi = (uint32_t)(dK >> 32);
-#ifndef PIPE_POLLING_ISSUE
         // The product needs all three (its S buffer free, K landed, Q landed), so the thread sleeps in one barrier
         // wait after the other instead of polling them with a back-off: the K tile, which is waited for longest,
         // comes first; the others have normally happened by then.
@@ -389,15 +369,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (ok && s_t >= 2) ok = mbar_wait(bar_s_free + sbuf, ((s_t >> 1) - 1) & 1, s_abort, p.status, 18);   // row of tile s_t - 2 is in registers
         if (!ok) break;
         {
-#else
-        const bool pd = s_t < 2 ? true : mbar_test(bar_s_free + sbuf, ((s_t >> 1) - 1) & 1);   // S buffer free: row of tile s_t - 2 is in registers
-        const bool kf = mbar_test(bar_k_full + kslot, (s_t / RK) & 1);
-        const bool qf = s_n > 0 ? true : mbar_test(bar_q_full + qslot, (si >> 1) & 1);
-        if (!(pd && kf && qf)) {
-          ok = guard.idle(s_abort, p.status, 2);
-        } else {
-          guard.reset();
-#endif
           tc_fence_after();
           // 32 bytes of the channel dimension per MMA: 16 bf16 (8 MMAs over two slabs) or 32 E4M3 (4 MMAs)
 #pragma unroll
@@ -421,8 +392,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       constexpr int kPvSteps = FP8 ? 4 : 8;          // 32 bytes of P per row per MMA: 16 bf16 or 32 E4M3 keys
       int p_item = first_item, p_n = 0, p_cnt = -1, p_t = 0, p_nonempty = 0;
       bool ok = true;
-      PipeIdle guard;
-      guard.reset();
       while (ok && p_item < p.items) {
         if (p_cnt < 0) p_cnt = __ldg(p.clean_cnt + p_item);
         if (p_n >= p_cnt) {
@@ -433,7 +402,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int pbuf = p_t & 1, vslot = p_t % RV;
         const uint64_t dV = make_smem_desc_sw128(smem_u32(sV + vslot * kSlot), kTile / 2);
         const uint32_t v_lo = (uint32_t)dV, v_hi = (uint32_t)(dV >> 32);
-#ifndef PIPE_POLLING_ISSUE
         // (see the S issuer) the V tile and the previous item's closer first, P, which arrives last, last
         ok = mbar_wait(bar_v_full + vslot, (p_t / RV) & 1, s_abort, p.status, 10);
         // first tile of an item only: O of the previous item must have been read by its closer
@@ -441,16 +409,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (ok) ok = mbar_wait(bar_p_full + pbuf, (p_t >> 1) & 1, s_abort, p.status, 20);
         if (!ok) break;
         {
-#else
-        const bool pf = mbar_test(bar_p_full + pbuf, (p_t >> 1) & 1);
-        const bool vf = mbar_test(bar_v_full + vslot, (p_t / RV) & 1);
-        // first tile of an item only: O of the previous item must have been read by its closer
-        const bool of = (p_n > 0 || p_nonempty == 0) ? true : mbar_test(bar_o_free, (p_nonempty - 1) & 1);
-        if (!(pf && vf && of)) {
-          ok = guard.idle(s_abort, p.status, 10);
-        } else {
-          guard.reset();
-#endif
           tc_fence_after();
 #pragma unroll
           for (int kk = 0; kk < kPvSteps; ++kk)
