@@ -49,7 +49,7 @@ constexpr float kPipeLazyLog2 = 8.0f;        // bf16: P may exceed 1 by up to 2^
 // at most 2^8 = 256 < 448, the E4M3 maximum; values below 2^-13 of the row maximum flush to zero.
 constexpr float kPipeFp8LazyLog2 = 4.0f, kPipeFp8PScaleLog2 = 4.0f;
 constexpr int kTile = 32768;                               // bytes of one 128 x 128 bf16 tile (two 64-column slabs)
-constexpr int kOffQ = 0, kOffK = 2 * kTile, kOffV = 4 * kTile, kOffMisc = 7 * kTile;
+constexpr int kOffQ = 0, kOffK = 2 * kTile, kOffMisc = 7 * kTile;     // Q slots | K ring, V ring (5 x 32 KB) | barriers ...
 constexpr int kPipeSmem = kOffMisc + 512 /*barriers*/ + 2 * 128 * 4 /*reference maxima*/ + 128 * 8 /*row sums*/ + 64;
 
 struct PipeParams {
