@@ -55,7 +55,7 @@ UNIT = "TFLOP/s"
 BRICKS = {"wan14b": (3, 5, 8), "wan1p3b": (3, 5, 4)}
 # DRAM bytes (read + write) of one bf16 forward launch on the default workload (wan14b, 97 %): the dram__bytes_read.sum +
 # dram__bytes_write.sum of a one-pass ncu capture of that launch (a profiler figure: it cannot be taken inside a timed run)
-FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2580123136 + 761104384}
+FWD_DRAM_TRAFFIC_BYTES = {"wan14b": 2462988800 + 760898304}
 
 
 def load_peaks():
