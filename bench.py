@@ -486,12 +486,13 @@ def run_ours(args, w):
         fp8["fused_launches_per_step"] = 4 + (3 if pipelined else 1)
         # per-token activation quantisation (the paper's fused scale-and-cast kernel), one tensor, outside the step
         tok_scales = torch.empty((w.B, Hl, w.N), dtype=torch.float32, device=dev)
+        tok_codes = torch.empty(q.shape, dtype=torch.uint8, device=dev)    # (its own buffer: codes[] feed the later FP8 legs)
         evt = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
 
         def step_tok(i):
             if i >= 0:
                 evt[i][0].record(stream)
-            sa.quant_fp8_per_token(v if i % 2 else k, codes=codes[0], scales=tok_scales)
+            sa.quant_fp8_per_token(v if i % 2 else k, codes=tok_codes, scales=tok_scales)
             if i >= 0:
                 evt[i][1].record(stream)
 
@@ -501,7 +502,7 @@ def run_ours(args, w):
         fp8["quant_per_token_ms"] = ms_tok
         fp8["quant_per_token_GBps"] = tbytes / (ms_tok * 1e-3) / 1e9
         fp8["quant_per_token_frac_of_hbm_peak"] = tbytes / (ms_tok * 1e-3) / 1e9 / peaks["hbm"]
-        del tok_scales
+        del tok_scales, tok_codes
 
     # ---- compensation branch + gate fusion (d = 128 only): state pass over K, V, then the fused apply pass
     comp = None
@@ -593,31 +594,6 @@ def run_ours(args, w):
         b.record(stream); torch.cuda.synchronize()
         return a.elapsed_time(b) / reps
 
-    # ---- sustained leg: about two seconds of back-to-back forward launches per dtype (a DiT runs this kernel for
-    # seconds, under the power cap), against the sustained GEMM peak; SM clock sampled during the region
-    sustained = None
-    if not args.no_sustained:
-        sustained = {}
-        legs = [("bf16", lambda: sa.fwd(q, k, v, kept_idx, kept_cnt, w.block, out=out, workspace=ws_fwd), ms_fwd)]
-        if codes is not None:
-            legs.append(("fp8", lambda: sa.fwd(codes[0], codes[1], codes[2], kept_idx, kept_cnt, w.block, scales=tuple(scales),
-                                               out=out, workspace=ws_fwd), fp8["fwd_ms"]))
-        for name, fn, ms_burst in legs:
-            reps = max(20, int(args.sustained_seconds * 1e3 / ms_burst))
-            with ClockSampler(local) as c2:
-                ms = max_over_ranks(timed_launches(fn, reps, warm=3), dev)
-            tf = flops / (ms * 1e-3) / 1e12
-            ck = c2.summary()
-            denom = peaks["bf16_sustained"] * (2.0 if name == "fp8" else 1.0)
-            sustained[name] = {"ms": ms, "launches": reps, "TFLOPs": tf, "peak_sustained": denom,
-                               "frac_sustained": tf / denom, "clocks": ck,
-                               "ms_x_sm_mhz": ms * ck["sm_mhz"] if ck.get("sm_mhz") else None}
-        if sa.read_status(ws_fwd) != sa.OK:
-            raise RuntimeError("device status after the sustained leg")
-        roofline["frac_sustained"] = sustained["bf16"]["frac_sustained"]
-        roofline["sustained"] = {"ms_per_launch": sustained["bf16"]["ms"], "achieved": sustained["bf16"]["TFLOPs"],
-                                 "peak": peaks["bf16_sustained"], "clocks": sustained["bf16"]["clocks"]}
-
     # ---- sparsity sweep: forward only (lists from sparkattn_select at every level), bf16 and FP8
     sweep = None
     if not args.no_sweep:
@@ -639,7 +615,6 @@ def run_ours(args, w):
             if sa.read_status(ws_fwd) != sa.OK:
                 raise RuntimeError(f"device status in the sweep at sparsity {s}")
             del ki, kc
-    del codes, scales
 
     # ---- second workload (the 480P shape at 90 %): select + forward, bf16 and FP8, same calls
     second = None
@@ -669,6 +644,34 @@ def run_ours(args, w):
                       "step_ms_select_plus_fwd_bf16": ms_s2 + ms_f2, "launches_timed_each": K,
                       "l2": "Q, K, V of this shape (3 x 101 MB) exceed the 126 MB L2 together; no explicit flush"}
             del q2, k2, v2, out2, cs2, ws_s2, ws_f2, ki2, kc2
+
+    # (after the sweep and the second workload: it leaves the board at the power cap)
+    # ---- sustained leg: about two seconds of back-to-back forward launches per dtype (a DiT runs this kernel for
+    # seconds, under the power cap), against the sustained GEMM peak; SM clock sampled during the region
+    sustained = None
+    if not args.no_sustained:
+        sustained = {}
+        legs = [("bf16", lambda: sa.fwd(q, k, v, kept_idx, kept_cnt, w.block, out=out, workspace=ws_fwd), ms_fwd)]
+        if codes is not None:
+            legs.append(("fp8", lambda: sa.fwd(codes[0], codes[1], codes[2], kept_idx, kept_cnt, w.block, scales=tuple(scales),
+                                               out=out, workspace=ws_fwd), fp8["fwd_ms"]))
+        for name, fn, ms_burst in legs:
+            reps = max(20, int(args.sustained_seconds * 1e3 / ms_burst))
+            with ClockSampler(local) as c2:
+                ms = max_over_ranks(timed_launches(fn, reps, warm=3), dev)
+            tf = flops / (ms * 1e-3) / 1e12
+            ck = c2.summary()
+            denom = peaks["bf16_sustained"] * (2.0 if name == "fp8" else 1.0)
+            sustained[name] = {"ms": ms, "launches": reps, "TFLOPs": tf, "peak_sustained": denom,
+                               "frac_sustained": tf / denom, "clocks": ck,
+                               "ms_x_sm_mhz": ms * ck["sm_mhz"] if ck.get("sm_mhz") else None}
+        if sa.read_status(ws_fwd) != sa.OK:
+            raise RuntimeError("device status after the sustained leg")
+        roofline["frac_sustained"] = sustained["bf16"]["frac_sustained"]
+        roofline["sustained"] = {"ms_per_launch": sustained["bf16"]["ms"], "achieved": sustained["bf16"]["TFLOPs"],
+                                 "peak": peaks["bf16_sustained"], "clocks": sustained["bf16"]["clocks"]}
+
+    del codes, scales
 
     # ---- end to end through the host-buffer C-ABI call (H2D of Q,K,V and D2H of O inside the timed region)
     e2e = None
