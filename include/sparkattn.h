@@ -337,6 +337,37 @@ int sparkattn_comp_apply(const sparkattn_shape_t* shape, const void* q_bf16, con
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Sparse forward and gate fusion in one kernel (Sec. 4.1: the module's output
+ * O = O_s + g * r * O_lr, with O_s the block-sparse attention output).
+ *
+ * Equivalent to sparkattn_fwd (bf16) followed by sparkattn_comp_apply with
+ * o_sparse = that call's output, without the round trip of O_s and the second
+ * read of Q through device memory: the warpgroup that finishes a query block
+ * keeps the normalised, bf16-rounded O_s rows in registers, forms
+ * q~ = R_r(p) silu(P_q q) from the Q tile still in shared memory, y = q~^T C
+ * on the tensor cores, and writes O_s + g * r * y / rms(y).  Every step is
+ * taken in the arithmetic and order of the two separate calls, so the output
+ * equals theirs bit for bit.  The state C comes from sparkattn_comp_state.
+ *
+ * Requires bf16 operands, d = 128, block = 128, rank = 64; no window mask and
+ * no padded-brick layout (SPARKATTN_E_UNSUPPORTED_SHAPE otherwise).
+ *
+ * q, k, v           : in,  bf16 [B,H,N,d] with the strides of `shape`
+ * kept_idx, kept_cnt, kmax, lse : as in sparkattn_fwd (lse is that of O_s)
+ * pq, grid_host, rope_axis_host, rope_freq_host, state, gate, eps : as in sparkattn_comp_apply
+ * out_bf16          : out, bf16 [B,H,N,d], strides of `shape`
+ * workspace         : >= sparkattn_fwd_gated_workspace_bytes(shape, kmax, grid_host) bytes
+ *                     (0 = unsupported arguments), 256-byte aligned; first word = device status
+ * Errors as in sparkattn_fwd and sparkattn_comp_apply; on an error the output is undefined.
+ */
+size_t sparkattn_fwd_gated_workspace_bytes(const sparkattn_shape_t* shape, int32_t kmax, const int32_t* grid_host);
+int sparkattn_fwd_gated(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, const void* v_bf16,
+                        const int32_t* kept_idx, const int32_t* kept_cnt, int32_t kmax, const void* pq_bf16,
+                        int32_t rank, const int32_t* grid_host, const int32_t* rope_axis_host,
+                        const float* rope_freq_host, const float* state, const float* gate, float eps, void* out_bf16,
+                        float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Block selection without any allocation (the paper has no counterpart: this
  * is a packaging variant of sparkattn_select, same rule, same outputs).
  *

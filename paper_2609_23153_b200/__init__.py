@@ -38,7 +38,7 @@ EXPORTS = (
     "sparkattn_select_noalloc_status", "sparkattn_comp_workspace_bytes", "sparkattn_comp_state",
     "sparkattn_comp_apply", "sparkattn_select_window", "sparkattn_fwd_window", "sparkattn_brick_count",
     "sparkattn_brick_layout", "sparkattn_gather_tokens", "sparkattn_select_padded", "sparkattn_fwd_padded",
-    "sparkattn_quant_fp8_pooled", "sparkattn_select_pooled",
+    "sparkattn_quant_fp8_pooled", "sparkattn_select_pooled", "sparkattn_fwd_gated_workspace_bytes", "sparkattn_fwd_gated",
 )
 
 
@@ -121,6 +121,11 @@ def lib() -> ctypes.CDLL:
         L.sparkattn_comp_state.argtypes = [sp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
         L.sparkattn_comp_apply.restype = ctypes.c_int
         L.sparkattn_comp_apply.argtypes = [sp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
+        L.sparkattn_fwd_gated_workspace_bytes.restype = sz
+        L.sparkattn_fwd_gated_workspace_bytes.argtypes = [sp, i32, vp]
+        L.sparkattn_fwd_gated.restype = ctypes.c_int
+        L.sparkattn_fwd_gated.argtypes = [sp, vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp, vp, vp, ctypes.c_float, vp,
+                                          vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -463,3 +468,43 @@ def comp_apply(q: torch.Tensor, pq: torch.Tensor, state: torch.Tensor, gate: tor
     if check_status:
         _check(read_status(workspace, stream), "sparkattn_comp_apply (device status)")
     return out
+
+
+def fwd_gated_workspace_bytes(shape: Shape, kmax: int, grid) -> int:
+    g = (ctypes.c_int32 * 3)(*[int(x) for x in grid])
+    return int(lib().sparkattn_fwd_gated_workspace_bytes(ctypes.byref(shape), kmax, g))
+
+
+def fwd_gated(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, kept_idx: torch.Tensor,
+              kept_cnt: Optional[torch.Tensor], pq: torch.Tensor, state: torch.Tensor, gate: torch.Tensor,
+              grid, axis: torch.Tensor, freq: torch.Tensor, *, eps: float = 1e-6, softmax_scale: float = 0.0,
+              out: Optional[torch.Tensor] = None, return_lse: bool = False, workspace: Optional[torch.Tensor] = None,
+              stream: Optional[torch.cuda.Stream] = None, check_status: bool = False):
+    """``sparkattn_fwd_gated``: the bf16 forward over 128-token blocks whose epilogue adds the gated
+    compensation term.  Arguments as in ``fwd`` and ``comp_apply``; returns the module output bf16
+    [B,H,N,d] (and the lse of the sparse branch, fp32 [B,H,N])."""
+    _same_layout(q, k, v)
+    shape = make_shape(q, 128, softmax_scale)
+    B, H, N, d = q.shape
+    rank = pq.shape[1]
+    kmax = kept_idx.shape[-1]
+    g, a, f = _rope_host(grid, axis, freq)
+    if not pq.is_contiguous() or pq.shape != (H, rank, d):
+        raise ValueError("pq must be contiguous [H, rank, d]")
+    if not state.is_contiguous() or state.shape != (B, H, rank, d) or state.dtype != torch.float32:
+        raise ValueError("state must be contiguous fp32 [B, H, rank, d]")
+    if not gate.is_contiguous() or gate.shape != (B, H, N) or gate.dtype != torch.float32:
+        raise ValueError("gate must be contiguous fp32 [B, H, N]")
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if return_lse else None
+    if workspace is None:
+        workspace = torch.empty(max(fwd_gated_workspace_bytes(shape, kmax, grid), 256), dtype=torch.uint8,
+                                device=q.device)
+    rc = lib().sparkattn_fwd_gated(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(kept_idx), _ptr(kept_cnt), kmax,
+                                   _ptr(pq), rank, g, _ptr(a), _ptr(f), _ptr(state), _ptr(gate), ctypes.c_float(eps),
+                                   _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "sparkattn_fwd_gated")
+    if check_status:
+        _check(read_status(workspace, stream), "sparkattn_fwd_gated (device status)")
+    return (out, lse) if return_lse else out

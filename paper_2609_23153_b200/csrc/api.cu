@@ -247,6 +247,37 @@ int sparkattn_comp_apply(const sparkattn_shape_t* shape, const void* q_bf16, con
                            o_sparse_bf16, out_bf16, eps, workspace, static_cast<cudaStream_t>(cuda_stream));
 }
 
+size_t sparkattn_fwd_gated_workspace_bytes(const sparkattn_shape_t* shape, int32_t kmax, const int32_t* grid_host) {
+  if (check_shape(shape) != SPARKATTN_OK || !fwd_pipe_gated_supported(*shape) || !grid_host) return 0;
+  if (kmax < 1 || kmax > num_blocks(shape) || kmax > kFwdMaxKept) return 0;
+  if (grid_host[0] < 1 || grid_host[1] < 1 || grid_host[2] < 1 ||
+      (long long)grid_host[0] * grid_host[1] * grid_host[2] != (long long)shape->N)
+    return 0;
+  return fwd_pipe_gated_workspace_bytes(*shape, kmax, grid_host);
+}
+
+int sparkattn_fwd_gated(const sparkattn_shape_t* shape, const void* q_bf16, const void* k_bf16, const void* v_bf16,
+                        const int32_t* kept_idx, const int32_t* kept_cnt, int32_t kmax, const void* pq_bf16,
+                        int32_t rank, const int32_t* grid_host, const int32_t* rope_axis_host,
+                        const float* rope_freq_host, const float* state, const float* gate, float eps, void* out_bf16,
+                        float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  int rc = check_comp(shape, rank, grid_host, rope_axis_host, rope_freq_host);
+  if (rc != SPARKATTN_OK) return rc;
+  if (!fwd_pipe_gated_supported(*shape)) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (!q_bf16 || !k_bf16 || !v_bf16 || !kept_idx || !pq_bf16 || !state || !gate || !out_bf16 || !workspace)
+    return SPARKATTN_E_INVALID_ARG;
+  if (kmax < 1 || kmax > num_blocks(shape)) return SPARKATTN_E_INVALID_ARG;
+  if (kmax > kFwdMaxKept) return SPARKATTN_E_UNSUPPORTED_SHAPE;
+  if (!(eps > 0.0f) || isinf(eps)) return SPARKATTN_E_INVALID_ARG;
+  if (!aligned16(q_bf16) || !aligned16(k_bf16) || !aligned16(v_bf16) || !aligned16(pq_bf16) || !aligned16(state) ||
+      !aligned16(out_bf16) || !aligned256(workspace))
+    return SPARKATTN_E_MISALIGNED;
+  if (workspace_bytes < fwd_pipe_gated_workspace_bytes(*shape, kmax, grid_host)) return SPARKATTN_E_WORKSPACE_TOO_SMALL;
+  return launch_fwd_pipe_gated(*shape, q_bf16, k_bf16, v_bf16, kept_idx, kept_cnt, kmax, pq_bf16, grid_host,
+                               rope_axis_host, rope_freq_host, state, gate, eps, out_bf16, lse, workspace,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
 namespace {
 // bricks padded to whole blocks: every block is whole, so N is a multiple of the block size
 int check_padded(const sparkattn_shape_t* shape, const int32_t* block_valid) {

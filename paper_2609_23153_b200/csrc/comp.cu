@@ -23,6 +23,7 @@
 
 #include "common.cuh"
 #include "launch.h"
+#include "rope.cuh"
 #include "tmap.h"
 
 namespace sparkattn {
@@ -36,12 +37,6 @@ constexpr int kRank = 64;
 constexpr int kCD = 128;              // head dimension handled by this file
 constexpr int kTileTok = 128;
 constexpr int kNumSMs = 148;          // chunking target (B200); any other count only changes the balance
-
-struct RopeTable {
-  int32_t axis[kRank / 2];            // 0 = t, 1 = y, 2 = x
-  float freq[kRank / 2];
-  int32_t T, Hg, Wg;
-};
 
 struct CompParams {
   RopeTable rope;
@@ -76,12 +71,6 @@ __global__ void rope_table_kernel(const RopeTable rope, float2* __restrict__ tab
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-
-__device__ __forceinline__ float fast_rcp(float x) {
-  float y;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
 }
 
 // One token row of T (64 fp32 columns at `taddr`) -> silu -> rank-truncated rotary rotation of the
@@ -643,7 +632,11 @@ static int comp_chunks(const sparkattn_shape_t& s) {
   return best;
 }
 
-static size_t rope_table_bytes(const int32_t* grid) {
+void launch_rope_table(const RopeTable& rope, float2* table, cudaStream_t stream) {
+  rope_table_kernel<<<(unsigned)(rope.T + rope.Hg + rope.Wg), kRank / 2, 0, stream>>>(rope, table);
+}
+
+size_t rope_table_bytes(const int32_t* grid) {
   return ((size_t)(kRank / 2) * ((size_t)grid[0] + grid[1] + grid[2]) * sizeof(float2) + 255) / 256 * 256;
 }
 

@@ -37,6 +37,7 @@
 
 #include "common.cuh"
 #include "launch.h"
+#include "rope.cuh"
 #include "tmap.h"
 
 namespace sparkattn {
@@ -69,6 +70,12 @@ struct PipeParams {
   const int32_t* blk_valid;    // [nb] real tokens per block (bricks padded to whole blocks), or NULL
   int64_t stride_b, stride_h, stride_n;
   float scale_log2;
+  // fused gate epilogue (GATE instantiation only; Sec. 4.1: O = O_s + g * r * RMSNorm(q~ C))
+  RopeTable rope;
+  const float2* rope_table;    // [T + Hg + Wg][rank/2] (cos, sin)
+  const float* state;          // [B*H][rank][d] fp32
+  const float* gate;           // [B*H][N]
+  float eps;
 };
 
 // one warp per item: drop (and report) kept indices outside [0, nb), clamp the count, own block first
@@ -197,11 +204,16 @@ __device__ __forceinline__ void pipe_tma_store_4d(const void* tmap, const void* 
 }
 
 // PAIR: 64-token blocks; a work item is a pair of query blocks, a tile two key blocks (see pair_lists_kernel).
-template <bool FP8, bool WINDOW, bool PAIR>
+// GATE (bf16, 128-token blocks, no window): the closing warpgroup of an item also computes the low-rank branch
+// of its 128 query rows and writes O = O_s + g * r * RMSNorm(q~ C) instead of O_s: the item's Q tile is still in
+// shared memory and its normalised output row in registers, so the separate pass that would read Q and O_s
+// again and write O falls away.  The V ring gives up one slot for P_q and C of the current head.
+template <bool FP8, bool WINDOW, bool PAIR, bool GATE = false>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
-                const PipeParams p) {
+                const __grid_constant__ CUtensorMap tmap_p, const PipeParams p) {
+  static_assert(!GATE || (!FP8 && !WINDOW && !PAIR), "the fused gate epilogue exists for plain bf16 only");
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sQ = smem + kOffQ;
   unsigned char* sK = smem + kOffK;
@@ -211,12 +223,17 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   // An input tile is 128 rows x 128 channels: two 64-channel slabs of 16 KB in bf16, one slab in FP8, where the
   // same bytes hold rings twice as deep (the Q slots keep their 32 KB: the item's output is staged there).
   constexpr int kSlot = FP8 ? kTile / 2 : kTile;
-  constexpr int RK = FP8 ? 4 : 2, RV = FP8 ? 6 : 3;    // (K 3 / V 2 measures the same)
+  constexpr int RK = FP8 ? 4 : 2, RV = GATE ? 2 : (FP8 ? 6 : 3);    // (K 3 / V 2 measures the same)
   unsigned char* sV = sK + RK * kSlot;         // the V ring follows the K ring (5 x 32 KB between them)
+  unsigned char* sP = sV + RV * kSlot;         // GATE: P_q of the current head (2 slabs of 8 KB), then C as bf16 (2 x 8 KB)
+  unsigned char* sC = sP + 16384;
   uint64_t* bar_k_full = bars + 32;           // [RK]
   uint64_t* bar_k_free = bar_k_full + RK;     // [RK] S MMAs that read the slot are complete
   uint64_t* bar_v_full = bar_k_free + RK;     // [RV]
   uint64_t* bar_v_free = bar_v_full + RV;     // [RV] PV MMAs that read the slot are complete
+  uint64_t* bar_gt = bars + 54;               // GATE [2]: the projection Q P_q^T of warpgroup g's closing is complete
+  uint64_t* bar_gy = bars + 56;               // GATE [2]: y = q~ C is complete
+  uint64_t* bar_pq = bars + 58;               // GATE [2]: P_q of a new head has landed
   uint64_t* bar_s_full = bars + 14;    // [2] S of a tile complete in S buffer (tile & 1)
   uint64_t* bar_s_free = bars + 16;    // [2] 128 arrivals: the warpgroup holds that S row in registers
   uint64_t* bar_p_full = bars + 18;    // [2] 128 arrivals: P written to P buffer (tile & 1)
@@ -229,6 +246,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   float2* s_lsum = reinterpret_cast<float2*>(s_mref + 2 * 128);  // [128] (partial row sum, reference it is relative to)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(s_lsum + 128);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  volatile int* s_gate_bh = s_abort + 1;      // GATE: (batch, head) whose P_q and C are in shared memory
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int kTileTx = FP8 ? kTile / 2 : kTile;
@@ -242,6 +260,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       mbar_init(bar_s_full + i, 1); mbar_init(bar_s_free + i, 128);
       mbar_init(bar_p_full + i, 128); mbar_init(bar_pv_done + i, 1);
     }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_gt + i, 1); mbar_init(bar_gy + i, 1); mbar_init(bar_pq + i, 1); }
+    *s_gate_bh = -1;
     for (int i = 0; i < RK; ++i) { mbar_init(bar_k_full + i, 1); mbar_init(bar_k_free + i, 1); }
     for (int i = 0; i < RV; ++i) { mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1); }
     mbar_init(bar_o_free, 128); mbar_init(bar_lsum, 128); mbar_init(bar_lsum_ack, 128);
@@ -256,6 +276,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   if (warp == 0) {
     if (lane == 0) {
       tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); tma_prefetch_desc(&tmap_o);
+      if constexpr (GATE) tma_prefetch_desc(&tmap_p);
     }
     __syncwarp();
     tmem_alloc(s_tmem, 512);
@@ -432,6 +453,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     int nonempty = 0;                                 // non-empty items finished so far
     bool ok = true;
     int io = 0;
+    int closings = 0, gate_loads = 0;                 // GATE: items this warpgroup has closed, heads it has staged (barrier phases)
     // Line-up of the warpgroup's 128 threads on a named barrier.  A hardware barrier has no time limit, so it
     // is fenced by the abort flag: no warp enters it once the flag is up, and a warp that leaves its loop
     // early arrives once on its way out, which releases the warps that were already inside (every other warp
@@ -746,6 +768,154 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         float inv = l > 0.0f ? 1.0f / l : 0.0f;           // no admissible key at all: zero row, lse = -inf
         if constexpr (FP8) inv *= v_max * 0.0625f;        // undo the 2^4 / max s_v folded into P
         unsigned char* slot = sQ + qslot * kTile;
+        if constexpr (GATE) {
+          // ---- O_s row, normalised and rounded to bf16, stays in registers; the sum of its squares for r_i
+          uint32_t opk[kPD / 2];
+          float so = 0.0f;
+#pragma unroll
+          for (int ch = 0; ch < kPD / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_O + lane_off + ch * 32, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[2 * j]) * inv, __uint_as_float(r[2 * j + 1]) * inv);
+              opk[ch * 16 + j] = *reinterpret_cast<const uint32_t*>(&h2);
+              const float2 f = __bfloat1622float2(h2);
+              so = fmaf(f.x, f.x, fmaf(f.y, f.y, so));
+            }
+          }
+          // ---- P_q and C of this (batch, head), if another head's are in shared memory (the product that read them
+          // last is complete: its warpgroup released O only after reading y)
+          if (*s_gate_bh != bh) {
+            const int a = row >> 1, half = row & 1;      // thread j converts row a, columns [64 half, +64) of the fp32 state
+            const float* src = p.state + ((int64_t)bh * kCompRank + a) * kPD + half * 64;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const float4 lo = __ldg(reinterpret_cast<const float4*>(src + 8 * c));
+              const float4 hi = __ldg(reinterpret_cast<const float4*>(src + 8 * c + 4));
+              const __nv_bfloat162 h0 = __floats2bfloat162_rn(lo.x, lo.y), h1 = __floats2bfloat162_rn(lo.z, lo.w);
+              const __nv_bfloat162 h2 = __floats2bfloat162_rn(hi.x, hi.y), h3 = __floats2bfloat162_rn(hi.z, hi.w);
+              *reinterpret_cast<uint4*>(sC + half * 8192 + a * 128 + ((c ^ (a & 7)) << 4)) =
+                  make_uint4(*reinterpret_cast<const uint32_t*>(&h0), *reinterpret_cast<const uint32_t*>(&h1),
+                             *reinterpret_cast<const uint32_t*>(&h2), *reinterpret_cast<const uint32_t*>(&h3));
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (row == 0) {
+              mbar_expect_tx(bar_pq + g, 16384);
+              tma_load_4d(sP, &tmap_p, bar_pq + g, 0, 0, h, 0);
+              tma_load_4d(sP + 8192, &tmap_p, bar_pq + g, 64, 0, h, 0);
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_pq + g, gate_loads & 1, s_abort, p.status, 21));
+            ++gate_loads;
+            if (ok) ok = wg_line_up(22);
+            if (!ok) break;
+            if (row == 0) *s_gate_bh = bh;
+          }
+          // ---- T = Q P_q^T into this warpgroup's P buffer (64 fp32 columns; its last P has been consumed)
+          const uint32_t tT = tmem_P + g * 64;
+          if (row == 0) {
+            tc_fence_after();
+            const uint64_t dX = make_smem_desc_sw128(smem_u32(slot), 16), dP = make_smem_desc_sw128(smem_u32(sP), 16);
+            const uint32_t x_lo = (uint32_t)dX, x_hi = (uint32_t)(dX >> 32), p_lo = (uint32_t)dP, p_hi = (uint32_t)(dP >> 32);
+            constexpr uint32_t idesc_t = make_idesc(1u, 128, kCompRank, false);
+#pragma unroll
+            for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk)
+                mma_ss<false>(tT, make_desc(x_lo + ((sl * 16384 + kk * 32) >> 4), x_hi),
+                              make_desc(p_lo + ((sl * 8192 + kk * 32) >> 4), p_hi), idesc_t, (sl | kk) != 0 ? 1u : 0u);
+            tc_commit(bar_gt + g);
+          }
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_gt + g, closings & 1, s_abort, p.status, 23));
+          if (!ok) break;
+          tc_fence_after();
+          // ---- q~ = R(p) silu(T) as bf16 over the first 32 columns of T (a thread only touches its own row)
+          {
+            const int token = min(q_row, p.N - 1);
+            const int x = token % p.rope.Wg, yy = token / p.rope.Wg;
+            const int y = yy % p.rope.Hg, tt = yy / p.rope.Hg;
+            const float2* row_t = p.rope_table + tt * (kCompRank / 2);
+            const float2* row_y = p.rope_table + (p.rope.T + y) * (kCompRank / 2);
+            const float2* row_x = p.rope_table + (p.rope.T + p.rope.Hg + x) * (kCompRank / 2);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t r[32];
+              tmem_ld32(tT + lane_off + half * 32, r);
+              float2 cs[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int m = half * 16 + j;
+                const int ax = p.rope.axis[m];
+                cs[j] = __ldg((ax == 0 ? row_t : (ax == 1 ? row_y : row_x)) + m);
+              }
+              tc_wait_ld();
+              uint32_t w[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float u0 = __uint_as_float(r[2 * j]), u1 = __uint_as_float(r[2 * j + 1]);
+                const float2 e = unpack_f32x2(fadd2(pack_f32x2(fast_exp2(u0 * -1.4426950408889634f), fast_exp2(u1 * -1.4426950408889634f)),
+                                                    pack_f32x2(1.0f, 1.0f)));
+                const float z0 = u0 * fast_rcp(e.x), z1 = u1 * fast_rcp(e.y);
+                const float o0 = fmaf(z0, cs[j].x, -z1 * cs[j].y);
+                const float o1 = fmaf(z0, cs[j].y, z1 * cs[j].x);
+                const __nv_bfloat162 h2 = __floats2bfloat162_rn(o0, o1);
+                w[j] = *reinterpret_cast<const uint32_t*>(&h2);
+              }
+              tmem_st16(tT + lane_off + half * 16, w);
+            }
+          }
+          tc_wait_st();
+          tc_fence_before();
+          ok = wg_line_up(24);
+          if (!ok) break;
+          // ---- y = q~ C over the O columns (O_s is in registers): A = q~ from TMEM, B = C, d contiguous
+          if (row == 0) {
+            tc_fence_after();
+            const uint64_t dC = make_smem_desc_sw128(smem_u32(sC), 8192);
+            const uint32_t c_lo = (uint32_t)dC, c_hi = (uint32_t)(dC >> 32);
+            constexpr uint32_t idesc_y = make_idesc(1u, 128, kPD, true);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              mma_ts<false>(tmem_O, tT + kk * 8, make_desc(c_lo + ((kk * 2048) >> 4), c_hi), idesc_y, kk != 0 ? 1u : 0u);
+            tc_commit(bar_gy + g);
+          }
+          const float gte = row_valid ? __ldg(p.gate + (int64_t)bh * p.N + q_row) : 0.0f;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_gy + g, closings & 1, s_abort, p.status, 25));
+          ++closings;
+          if (!ok) break;
+          tc_fence_after();
+          // ---- two passes over y: its mean square, then O = O_s + g * r * y / rms(y) into the Q slot
+          float ss = 0.0f;
+#pragma unroll
+          for (int ch = 0; ch < kPD / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_O + lane_off + ch * 32, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ss = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ss);
+          }
+          const float coef = gte * sqrtf(so * (1.0f / kPD)) * rsqrtf(ss * (1.0f / kPD) + p.eps);
+#pragma unroll
+          for (int ch = 0; ch < kPD / 32; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(tmem_O + lane_off + ch * 32, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+              uint32_t ww[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&opk[ch * 16 + cc * 4 + j]));
+                const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(coef, __uint_as_float(r[8 * cc + 2 * j]), f.x),
+                                                                fmaf(coef, __uint_as_float(r[8 * cc + 2 * j + 1]), f.y));
+                ww[j] = *reinterpret_cast<const uint32_t*>(&o2);
+              }
+              *reinterpret_cast<uint4*>(slot + (ch >> 1) * (kTile / 2) + row * 128 + ((((ch & 1) * 4 + cc) ^ (row & 7)) << 4)) =
+                  make_uint4(ww[0], ww[1], ww[2], ww[3]);
+            }
+          }
+        } else {
 #pragma unroll 1
         for (int ch = 0; ch < kPD / 32; ++ch) {
           uint32_t r[32];
@@ -763,6 +933,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             *reinterpret_cast<uint4*>(slot + (ch >> 1) * (kTile / 2) + row * 128 + ((((ch & 1) * 4 + cc) ^ (row & 7)) << 4)) =
                 make_uint4(ww[0], ww[1], ww[2], ww[3]);
           }
+        }
         }
         tc_fence_before();
         mbar_arrive(bar_o_free);
@@ -819,11 +990,51 @@ size_t fwd_pipe_workspace_bytes(const sparkattn_shape_t& s, int kmax) {
          (size_t)s.B * s.H * 4;
 }
 
+bool fwd_pipe_gated_supported(const sparkattn_shape_t& s) { return s.d == 128 && s.block == 128; }
+
+// ... | rotary table of the fused compensation epilogue
+size_t fwd_pipe_gated_workspace_bytes(const sparkattn_shape_t& s, int kmax, const int32_t* grid) {
+  return (fwd_pipe_workspace_bytes(s, kmax) + 255) / 256 * 256 + rope_table_bytes(grid);
+}
+
+// the compensation branch's operands of the fused epilogue (device pointers except grid / axis / freq)
+struct PipeGateArgs {
+  const void* pq;
+  const int32_t* grid;
+  const int32_t* axis;
+  const float* freq;
+  const float* state;
+  const float* gate;
+  float eps;
+};
+
+static int launch_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
+                       const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                       const int32_t* kept_cnt, int kmax, int frame_tokens, int window, const int32_t* block_valid,
+                       void* out, float* lse, void* workspace, const PipeGateArgs* ga, cudaStream_t stream);
+
 int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
                     const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
                     const int32_t* kept_cnt, int kmax, int frame_tokens, int window, const int32_t* block_valid,
                     void* out, float* lse, void* workspace, cudaStream_t stream) {
-  CUtensorMap mq, mk, mv, mo;
+  return launch_pipe(s, fp8, q, k, v, q_scale, k_scale, v_scale, kept_idx, kept_cnt, kmax, frame_tokens, window,
+                     block_valid, out, lse, workspace, nullptr, stream);
+}
+
+int launch_fwd_pipe_gated(const sparkattn_shape_t& s, const void* q, const void* k, const void* v,
+                          const int32_t* kept_idx, const int32_t* kept_cnt, int kmax, const void* pq,
+                          const int32_t* grid, const int32_t* axis, const float* freq, const float* state,
+                          const float* gate, float eps, void* out, float* lse, void* workspace, cudaStream_t stream) {
+  const PipeGateArgs ga{pq, grid, axis, freq, state, gate, eps};
+  return launch_pipe(s, false, q, k, v, nullptr, nullptr, nullptr, kept_idx, kept_cnt, kmax, 0, 0, nullptr, out, lse,
+                     workspace, &ga, stream);
+}
+
+static int launch_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const void* k, const void* v,
+                       const float* q_scale, const float* k_scale, const float* v_scale, const int32_t* kept_idx,
+                       const int32_t* kept_cnt, int kmax, int frame_tokens, int window, const int32_t* block_valid,
+                       void* out, float* lse, void* workspace, const PipeGateArgs* ga, cudaStream_t stream) {
+  CUtensorMap mq, mk, mv, mo, mp;
   int rc;
   const int elt = fp8 ? 1 : 2;
   const bool pair = s.block == 64;
@@ -831,6 +1042,12 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   if ((rc = make_token_map(&mk, k, elt, s, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
   if ((rc = make_token_map(&mv, v, elt, s, pair ? 64 : kPBLK)) != SPARKATTN_OK) return rc;
   if ((rc = make_token_map(&mo, out, 2, s, kPBLK)) != SPARKATTN_OK) return rc;
+  mp = mo;                                           // never read without the fused epilogue
+  if (ga) {
+    const uint64_t dims[4] = {(uint64_t)kPD, (uint64_t)kCompRank, (uint64_t)s.H, 1};
+    const uint64_t strides[3] = {(uint64_t)kPD, (uint64_t)kCompRank * kPD, (uint64_t)s.H * kCompRank * kPD};
+    if ((rc = make_slab_map(&mp, ga->pq, 2, dims, strides, kCompRank)) != SPARKATTN_OK) return rc;
+  }
   const int nb = (s.N + s.block - 1) / s.block;
   int nbq, lstride;
   pipe_geometry(s, kmax, &nbq, &lstride);
@@ -841,7 +1058,7 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   int32_t* clean_list = reinterpret_cast<int32_t*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256);
   float* v_max = reinterpret_cast<float*>(base + kWorkspaceHeaderBytes + ((size_t)items * 4 + 255) / 256 * 256 +
                                           ((size_t)items * lstride * 4 + 255) / 256 * 256);
-  PipeParams prm;
+  PipeParams prm{};
   prm.clean_cnt = clean_cnt;
   prm.clean_list = clean_list;
   prm.q_scale = q_scale; prm.k_scale = k_scale; prm.v_scale = v_scale; prm.v_max = v_max;
@@ -857,6 +1074,14 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
   const int sm_count = current_sm_count();
   if (sm_count < 1) return SPARKATTN_E_CUDA;
   if (cudaMemsetAsync(workspace, 0, kWorkspaceHeaderBytes, stream) != cudaSuccess) return SPARKATTN_E_CUDA;
+  if (ga) {
+    for (int m = 0; m < kCompRank / 2; ++m) { prm.rope.axis[m] = ga->axis[m]; prm.rope.freq[m] = ga->freq[m]; }
+    prm.rope.T = ga->grid[0]; prm.rope.Hg = ga->grid[1]; prm.rope.Wg = ga->grid[2];
+    float2* table = reinterpret_cast<float2*>(base + (fwd_pipe_workspace_bytes(s, kmax) + 255) / 256 * 256);
+    launch_rope_table(prm.rope, table, stream);
+    prm.rope_table = table;
+    prm.state = ga->state; prm.gate = ga->gate; prm.eps = ga->eps;
+  }
   if (pair) {
     const size_t bits = (size_t)kPairWarps * 2 * ((nb + 31) / 32) * sizeof(uint32_t);
     pair_lists_kernel<<<(unsigned)((items + kPairWarps - 1) / kPairWarps), kPairWarps * 32, bits, stream>>>(
@@ -871,10 +1096,11 @@ int launch_fwd_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, const v
                           : (win ? fwd_pipe_kernel<false, true, true> : fwd_pipe_kernel<false, false, true>))
                    : (fp8 ? (win ? fwd_pipe_kernel<true, true, false> : fwd_pipe_kernel<true, false, false>)
                           : (win ? fwd_pipe_kernel<false, true, false> : fwd_pipe_kernel<false, false, false>));
+  if (ga) kern = fwd_pipe_kernel<false, false, false, true>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
-  kern<<<grid, kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, prm);
+  kern<<<grid, kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, mp, prm);
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 

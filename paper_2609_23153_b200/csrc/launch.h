@@ -60,6 +60,15 @@ int launch_comp_apply(const sparkattn_shape_t& s, const void* q, const void* pq,
                       const int32_t* axis, const float* freq, const float* state, const float* gate,
                       const void* o_sparse, void* out, float eps, void* workspace, cudaStream_t stream);
 
+// fwd_pipe.cu: forward whose epilogue adds the gated compensation term (bf16, d = 128, 128-token blocks);
+// workspace = that of the plain forward, rounded up to 256 bytes, then the rotary table
+bool fwd_pipe_gated_supported(const sparkattn_shape_t& s);
+size_t fwd_pipe_gated_workspace_bytes(const sparkattn_shape_t& s, int kmax, const int32_t* grid);
+int launch_fwd_pipe_gated(const sparkattn_shape_t& s, const void* q, const void* k, const void* v,
+                          const int32_t* kept_idx, const int32_t* kept_cnt, int kmax, const void* pq,
+                          const int32_t* grid, const int32_t* axis, const float* freq, const float* state,
+                          const float* gate, float eps, void* out, float* lse, void* workspace, cudaStream_t stream);
+
 // reorder.cu: tokens stored brick by brick, every brick padded to a whole block
 int launch_brick_layout(const int32_t* grid, const int32_t* brick, int block, int32_t* gather, int32_t* block_valid,
                         int32_t* scatter, cudaStream_t stream);
