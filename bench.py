@@ -504,6 +504,19 @@ def run_ours(args, w):
         fp8["quant_per_token_frac_of_hbm_peak"] = tbytes / (ms_tok * 1e-3) / 1e9 / peaks["hbm"]
         del tok_scales, tok_codes
 
+    def timed_launches(fn, reps, warm=1, idle_s=0.0):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        if idle_s > 0:
+            time.sleep(idle_s)       # let the board come back from the power cap of whatever ran before
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream); torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
     # ---- compensation branch + gate fusion (d = 128 only): state pass over K, V, then the fused apply pass
     comp = None
     if not args.no_comp and w.d == 128:
@@ -537,6 +550,24 @@ def run_ours(args, w):
                 "apply_ms": ms_a, "apply_GBps": abytes / (ms_a * 1e-3) / 1e9,
                 "apply_frac_of_hbm_peak": abytes / (ms_a * 1e-3) / 1e9 / peaks["hbm"],
                 "launches_per_step": 3}
+        # the same module output from one call: the forward whose epilogue adds the gated term (bf16, 128-token blocks),
+        # against the forward followed by the apply pass, each timed alone after an idle second
+        if w.block == 128 and not args.block:
+            ws_g = torch.empty(sa.fwd_gated_workspace_bytes(shape, kept_idx.shape[-1], w.grid), dtype=torch.uint8, device=dev)
+            gated = lambda: sa.fwd_gated(q, k, v, kept_idx, kept_cnt, pq, state, gate, w.grid, axis, freq, out=fused,
+                                         workspace=ws_g)
+
+            def two_calls():
+                sa.fwd(q, k, v, kept_idx, kept_cnt, w.block, out=out, workspace=ws_fwd)
+                sa.comp_apply(q, pq, state, gate, out, w.grid, axis, freq, out=fused, workspace=ws_c)
+
+            ms_two = timed_launches(two_calls, K, warm=3, idle_s=1.0)
+            ms_one = timed_launches(gated, K, warm=3, idle_s=1.0)
+            if sa.read_status(ws_g) != sa.OK:
+                raise RuntimeError("device status after the gated forward")
+            comp["fwd_then_apply_ms"] = ms_two
+            comp["fwd_gated_ms"] = ms_one
+            del ws_g
         del fused, state, ws_c, pq, pk, gate
 
     # ---- brick token order (d = 128, 128-token blocks): gather into bricks padded to whole blocks, selection and
@@ -580,19 +611,6 @@ def run_ours(args, w):
                   "select_ms": statistics.mean(a.elapsed_time(b) for a, b in evs_b),
                   "fwd_ms": statistics.mean(a.elapsed_time(b) for a, b in evf_b)}
         del qb_, kb_, vb_, out_b, ws_sb, ws_fb
-
-    def timed_launches(fn, reps, warm=1, idle_s=0.0):
-        for _ in range(warm):
-            fn()
-        torch.cuda.synchronize()
-        if idle_s > 0:
-            time.sleep(idle_s)       # let the board come back from the power cap of whatever ran before
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(reps):
-            fn()
-        b.record(stream); torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps
 
     # ---- sparsity sweep: forward only (lists from sparkattn_select at every level), bf16 and FP8
     sweep = None
