@@ -236,3 +236,37 @@ def test_host_buffer_call_rejects_more_batches_than_head_groups(lib):
     s = _shape(B=16, H=40, N=256, d=64, block=64)
     r = lib.sparkattn_attention_host(ctypes.byref(s), sa.BF16, fake, fake, fake, 2, fake, ctypes.c_void_p(0), fake, 256, st)
     assert r == sa.E_WORKSPACE_TOO_SMALL
+
+
+def test_gated_forward_validates_on_the_host(lib):
+    """sparkattn_fwd_gated: every argument check happens before the device is touched."""
+    s = _shape(N=2048, d=128, block=128)
+    fake = ctypes.c_void_p(0x1000)
+    null = ctypes.c_void_p(0)
+    st = ctypes.c_void_p(0)
+    grid = (ctypes.c_int32 * 3)(2, 32, 32)
+    axis = (ctypes.c_int32 * 32)(*([0] * 10 + [1] * 11 + [2] * 11))
+    freq = (ctypes.c_float * 32)(*[0.01 * (m + 1) for m in range(32)])
+    eps = ctypes.c_float(1e-6)
+    need = lib.sparkattn_fwd_gated_workspace_bytes(ctypes.byref(s), 4, grid)
+    assert need > sa.workspace_bytes(s, 1, 4)          # the plain forward's workspace plus the rotary table
+
+    def call(shape=s, q=fake, kmax=4, rank=64, g=grid, ax=axis, e=eps, ws=fake, nbytes=need, state=fake):
+        return lib.sparkattn_fwd_gated(ctypes.byref(shape), q, fake, fake, fake, null, kmax, fake, rank, g, ax, freq, state,
+                                       fake, e, fake, null, ws, nbytes, st)
+
+    assert call(q=null) == sa.E_INVALID_ARG
+    assert call(state=null) == sa.E_INVALID_ARG
+    assert call(kmax=0) == sa.E_INVALID_ARG
+    assert call(kmax=17) == sa.E_INVALID_ARG                          # more than the 16 key blocks
+    assert call(e=ctypes.c_float(0.0)) == sa.E_INVALID_ARG
+    assert call(g=(ctypes.c_int32 * 3)(2, 32, 31)) == sa.E_INVALID_ARG     # grid does not multiply to N
+    assert call(ax=(ctypes.c_int32 * 32)(*([3] * 32))) == sa.E_INVALID_ARG
+    assert call(rank=32) == sa.E_UNSUPPORTED_SHAPE
+    assert call(shape=_shape(N=2048, d=128, block=64)) == sa.E_UNSUPPORTED_SHAPE
+    assert call(shape=_shape(N=2048, d=64, block=128)) == sa.E_UNSUPPORTED_SHAPE
+    assert call(q=ctypes.c_void_p(0x1008)) == sa.E_MISALIGNED
+    assert call(ws=ctypes.c_void_p(0x1010)) == sa.E_MISALIGNED
+    assert call(nbytes=need - 1) == sa.E_WORKSPACE_TOO_SMALL
+    assert lib.sparkattn_fwd_gated_workspace_bytes(ctypes.byref(_shape(N=2048, d=128, block=64)), 4, grid) == 0
+    assert lib.sparkattn_fwd_gated_workspace_bytes(ctypes.byref(s), 4, (ctypes.c_int32 * 3)(2, 32, 31)) == 0
