@@ -1,6 +1,6 @@
-"""Pins for the causal frame window of the oracle (WIN-0: the paper's one-line extension "compensated
-sparse attention can be restricted to a causal window", read as: key j counts for query i iff its
-frame j // F lies in (i // F - W, i // F]).  Independent formulations: library softmax over explicitly
+"""Pins for the causal frame window of the oracle (WIN-0: Sec. 1 mentions, without a formula, that the
+method extends to auto-regressive generation by limiting attention to a causal window; read as: key j
+counts for query i iff its frame j // F lies in (i // F - W, i // F]).  Independent formulations: library softmax over explicitly
 masked logits, per-frame dense attention, brute-force candidate enumeration."""
 import math
 
