@@ -53,8 +53,12 @@
 
 namespace sparkattn {
 
-constexpr int kPipeThreads = 384;
+constexpr int kPipeThreads = 384;                           // GATE variant: 4 control warps + 2 softmax warpgroups
 constexpr int kPipeSoftmaxRegs = 216, kPipeCtrlRegs = 64;   // 2*128*216 + 128*64 <= 384*168
+// bf16 with short kept lists (EPI): a third warpgroup (warps 12-15) closes the items, see below
+constexpr int kEpiThreads = 512;
+constexpr int kEpiMaxKept = 32;                             // longest kept list the launcher gives to that variant
+constexpr int kEpiSoftmaxRegs = 216, kEpiCtrlRegs = 40, kEpiCloseRegs = 40;   // 2*128*216 + 128*40 + 128*40 = 512*128
 constexpr int kPD = 128, kPBLK = 128;
 constexpr float kPipeLazyLog2 = 8.0f;        // bf16: P may exceed 1 by up to 2^8 before O is rescaled
 // FP8: P is pre-scaled by 2^4 * (s_v[j] / max s_v) and may grow by another 2^4 before O is rescaled:
@@ -219,8 +223,8 @@ __device__ __forceinline__ void pipe_tma_store_4d(const void* tmap, const void* 
 // of its 128 query rows and writes O = O_s + g * r * RMSNorm(q~ C) instead of O_s: the item's Q tile is still in
 // shared memory and its normalised output row in registers, so the separate pass that would read Q and O_s
 // again and write O falls away.  The V ring gives up one slot for P_q and C of the current head.
-template <bool FP8, bool WINDOW, bool PAIR, bool GATE = false>
-__global__ void __launch_bounds__(kPipeThreads, 1)
+template <bool FP8, bool WINDOW, bool PAIR, bool GATE = false, bool EPI = false>
+__global__ void __launch_bounds__(EPI ? kEpiThreads : kPipeThreads, 1)
 fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
                 const __grid_constant__ CUtensorMap tmap_p, const PipeParams p) {
@@ -242,6 +246,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   uint64_t* bar_k_free = bar_k_full + RK;     // [RK] S MMAs that read the slot are complete
   uint64_t* bar_v_full = bar_k_free + RK;     // [RV]
   uint64_t* bar_v_free = bar_v_full + RV;     // [RV] PV MMAs that read the slot are complete
+  uint64_t* bar_cl = bars + 54;               // EPI [2], 128 arrivals: the sums of the warpgroup of the item's last tile are in Q slot i
   uint64_t* bar_gt = bars + 54;               // GATE [2]: the projection Q P_q^T of warpgroup g's closing is complete
   uint64_t* bar_gy = bars + 56;               // GATE [2]: y = q~ C is complete
   uint64_t* bar_pq = bars + 58;               // GATE [2]: P_q of a new head has landed
@@ -271,7 +276,11 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       mbar_init(bar_s_full + i, 1); mbar_init(bar_s_free + i, 128);
       mbar_init(bar_p_full + i, 128); mbar_init(bar_pv_done + i, 1);
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_gt + i, 1); mbar_init(bar_gy + i, 1); mbar_init(bar_pq + i, 1); }
+    if constexpr (GATE) {
+      for (int i = 0; i < 2; ++i) { mbar_init(bar_gt + i, 1); mbar_init(bar_gy + i, 1); mbar_init(bar_pq + i, 1); }
+    } else if constexpr (EPI) {
+      mbar_init(bar_cl, 128); mbar_init(bar_cl + 1, 128);
+    }
     *s_gate_bh = -1;
     for (int i = 0; i < RK; ++i) { mbar_init(bar_k_full + i, 1); mbar_init(bar_k_free + i, 1); }
     for (int i = 0; i < RV; ++i) { mbar_init(bar_v_full + i, 1); mbar_init(bar_v_free + i, 1); }
@@ -302,7 +311,13 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   const bool dead = *s_abort != 0;
   const int first_item = blockIdx.x, item_step = gridDim.x;
 
-  if (warp < 4) reg_dec<kPipeCtrlRegs>();
+  static_assert(!EPI || (!GATE && !FP8), "the closing warpgroup exists for the plain bf16 variants");
+  if constexpr (EPI) {
+    if (warp < 4) reg_dec<kEpiCtrlRegs>();
+    else if (warp >= 12) reg_dec<kEpiCloseRegs>();
+  } else {
+    if (warp < 4) reg_dec<kPipeCtrlRegs>();
+  }
   if (dead) {
     // fall through to the teardown
   } else if (warp == 0 || warp == 3) {
@@ -452,9 +467,9 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp >= 4 && warp < 12) {
     // ----------------------------------------------------------------- softmax
-    reg_inc<kPipeSoftmaxRegs>();
+    if constexpr (EPI) reg_inc<kEpiSoftmaxRegs>(); else reg_inc<kPipeSoftmaxRegs>();
     const int g = (warp >> 2) - 1;                    // warpgroup: takes the tiles with (global tile counter & 1) == g
     const int row = threadIdx.x & 127;                // query row inside the block = TMEM lane
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -474,11 +489,11 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       asm volatile("bar.sync %0, 128;" ::"r"(1 + g) : "memory");
       return true;
     };
-    // bf16, 128-token blocks: the thread that stores an item's output does not wait until the copy has read the
-    // Q slot (about 1300 clocks, on the path to the closing warpgroup's next tile); it releases the slot after
-    // its next tile, or, should the item after the next come first (its Q goes into this very slot), before that.
-    // (The FP8 and paired instantiations measured slower with the extra test per tile and wait at once.)
-    constexpr bool kDeferStoreWait = !FP8 && !PAIR;
+    // GATE (a softmax warpgroup closes the item, lists are short): the thread that stores an item's output does not wait
+    // until the copy has read the Q slot (about 1300 clocks, on the path to the closing warpgroup's next tile);
+    // it releases the slot after its next tile, or, should the item after the next come first (its Q goes into
+    // this very slot), before that.
+    constexpr bool kDeferStoreWait = GATE;            // (elsewhere the extra test per tile costs more than the wait: lists are long, or FP8)
     int store_slot = -1, store_io = 0;                // row 0: Q slot whose output store is in flight, and its item
     auto store_flush = [&]() {
       asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -767,7 +782,23 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
       // ------------------------------------------------------------ end of the item
       const int t_last = t + cnt - 1;
-      if ((t_last & 1) != g) {
+      if constexpr (EPI) {
+        // The closing warpgroup (warps 12-15) finishes the item; the softmax warpgroups only leave it their
+        // partial row sums and the reference they are relative to, and go on to the next item's tiles: the
+        // warpgroup of the item's last tile in the first KB of the item's Q slot (it has read the last S, so every
+        // S product of the item is complete and Q is dead), the other one in s_lsum.
+        if ((t_last & 1) != g) {
+          if (nonempty > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum_ack, (nonempty - 1) & 1, s_abort, p.status, 7));
+            if (!ok) break;
+          }
+          s_lsum[row] = make_float2(l, m_used);
+          mbar_arrive(bar_lsum);
+        } else {
+          reinterpret_cast<float2*>(sQ + qslot * kTile)[row] = make_float2(l, m_used);
+          mbar_arrive(bar_cl + qslot);
+        }
+      } else if ((t_last & 1) != g) {
         // not the closer: hand the partial row sum over (after the previous hand-over was read)
         if (nonempty > 0) {
           ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum_ack, (nonempty - 1) & 1, s_abort, p.status, 7));
@@ -988,6 +1019,89 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (row == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
+  else if (EPI && warp >= 12) {
+    // ----------------------------------------------------------------- closing warpgroup (EPI variants)
+    // Walks the CTA's items in order.  For each: the two partial row sums, the last PV, then the normalised O
+    // row as bf16 into the item's Q slot, O back to the PV issuer, lse, one TMA store, the Q slot back to the
+    // producer.  Nothing here is on the softmax warpgroups' path.
+    const int row = threadIdx.x & 127;
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    auto line_up = [&]() {
+      if (*s_abort) return false;
+      asm volatile("bar.sync 3, 128;" ::: "memory");
+      return true;
+    };
+    int t = 0, nonempty = 0, io = 0;
+    int slot_use[2] = {0, 0};                         // non-empty items that have used Q slot i
+    bool ok = true;
+    for (int item = first_item; ok && item < p.items; item += item_step, ++io) {
+      const int cnt = __ldg(p.clean_cnt + item);
+      if (cnt == 0) continue;                          // warpgroup 0 writes the zero rows of an empty list
+      const int qslot = io & 1;
+      const int qb = item % p.nbq, bh = item / p.nbq;
+      const int h = bh % p.H, b = bh / p.H;
+      const int q_row = qb * kPBLK + row;
+      const bool row_valid = q_row < p.N;
+      const int t_last = t + cnt - 1;
+      unsigned char* slot = sQ + qslot * kTile;
+      float v_max = 1.0f;
+      if constexpr (FP8) v_max = __ldg(p.v_max + bh);
+      // the slot's barrier completes once per non-empty item that uses the slot; this item's Q could only be
+      // loaded after the previous user's output had left, so the wait is never more than one phase behind
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_cl + qslot, slot_use[qslot] & 1, s_abort, p.status, 8));
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_lsum, nonempty & 1, s_abort, p.status, 27));
+      if (!ok) break;
+      const float2 mine = reinterpret_cast<const float2*>(slot)[row];
+      const float2 other = s_lsum[row];
+      mbar_arrive(bar_lsum_ack);
+      ++slot_use[qslot];
+      float l = mine.x;
+      const float m_used = mine.y;
+      if (other.x != 0.0f) l += other.x * fast_exp2(other.y - m_used);
+      ok = line_up();                                  // every row's sums are read before O rows overwrite them
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pv_done + (t_last & 1), (t_last >> 1) & 1, s_abort, p.status, 9));
+      if (!ok) break;
+      tc_fence_after();
+      float inv = l > 0.0f ? 1.0f / l : 0.0f;          // no admissible key at all: zero row, lse = -inf
+      if constexpr (FP8) inv *= v_max * 0.0625f;       // undo the 2^4 / max s_v folded into P
+#pragma unroll 1
+      for (int ch = 0; ch < kPD / 32; ++ch) {
+        uint32_t r[32];
+        tmem_ld32(tmem_O + lane_off + ch * 32, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t ww[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[8 * cc + 2 * j]) * inv,
+                                                            __uint_as_float(r[8 * cc + 2 * j + 1]) * inv);
+            ww[j] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          *reinterpret_cast<uint4*>(slot + (ch >> 1) * (kTile / 2) + row * 128 + ((((ch & 1) * 4 + cc) ^ (row & 7)) << 4)) =
+              make_uint4(ww[0], ww[1], ww[2], ww[3]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_o_free);
+      if (row_valid && p.lse) p.lse[(int64_t)bh * p.N + q_row] = (m_used + log2f(l)) * 0.6931471805599453f;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      ok = line_up();
+      if (!ok) break;
+      if (row == 0) {
+        pipe_tma_store_4d(&tmap_o, slot, 0, qb * kPBLK, h, b);
+        pipe_tma_store_4d(&tmap_o, slot + kTile / 2, 64, qb * kPBLK, h, b);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        mbar_arrive(bar_q_free + qslot);
+      }
+      t += cnt;
+      ++nonempty;
+    }
+    if (!ok) asm volatile("bar.arrive 3, 128;" ::: "memory");
+    if (row == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
@@ -1128,11 +1242,17 @@ static int launch_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, cons
                           : (win ? fwd_pipe_kernel<false, true, true> : fwd_pipe_kernel<false, false, true>))
                    : (fp8 ? (win ? fwd_pipe_kernel<true, true, false> : fwd_pipe_kernel<true, false, false>)
                           : (win ? fwd_pipe_kernel<false, true, false> : fwd_pipe_kernel<false, false, false>));
+  // bf16 with short lists: the variant with a closing warpgroup (it takes the item boundary off the softmax
+  // warpgroups, 2 % at 18 tiles per item, but its main loop is 3 % slower: it stops paying near 30 tiles per item)
+  const bool epi = !fp8 && !ga && kmax <= kEpiMaxKept;
+  if (epi)
+    kern = pair ? (win ? fwd_pipe_kernel<false, true, true, false, true> : fwd_pipe_kernel<false, false, true, false, true>)
+                : (win ? fwd_pipe_kernel<false, true, false, false, true> : fwd_pipe_kernel<false, false, false, false, true>);
   if (ga) kern = fwd_pipe_kernel<false, false, false, true>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;
   const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
-  kern<<<grid, kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, mp, prm);
+  kern<<<grid, epi ? kEpiThreads : kPipeThreads, kPipeSmem, stream>>>(mq, mk, mv, mo, mp, prm);
   return cudaGetLastError() == cudaSuccess ? SPARKATTN_OK : SPARKATTN_E_CUDA;
 }
 
