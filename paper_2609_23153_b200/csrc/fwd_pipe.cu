@@ -33,16 +33,25 @@
 // compacted by a small pre-pass into the workspace; every role reads the clean lists from there.
 // Every wait is bounded; nothing here waits on another CTA.
 //
-// GATE variant (sparkattn_fwd_gated; bf16, 128-token blocks): the closing warpgroup adds the gated
-// low-rank term of Sec. 4.1 before the store.  Once the last PV of the item is complete it issues
-// T = Q P_q^T (Q still in its slot) into its own P buffer, turns T into q~ = R(p) silu(T) as bf16 in
+// EPI variant (bf16, kept lists of at most kEpiMaxKept blocks): 512 threads, warps 12-15 are a closing
+// warpgroup.  At the end of an item the softmax warpgroups only leave their partial row sums (the
+// warpgroup of the last tile in the first KB of the item's dead Q slot, the other one in s_lsum) and go
+// on to the next item's tiles; the closing warpgroup waits for the last PV, reads O, normalises it into
+// the Q slot, hands O back to the PV issuer, writes lse and stores the tile.  That takes the wait for the
+// last PV, the O read and the store off the warpgroup whose next tile the pipeline needs (-2 % at 18
+// tiles per item); with four more warps resident the tile loop itself runs 3 % slower, so the launcher
+// keeps the 384-thread kernel for longer lists, and for FP8, which measured slower with it.
+//
+// GATE variant (sparkattn_fwd_gated; bf16, 128-token blocks, 384 threads): the closing softmax warpgroup
+// adds the gated low-rank term of Sec. 4.1 before the store.  Once the last PV of the item is complete it
+// issues T = Q P_q^T (Q still in its slot) into its own P buffer, turns T into q~ = R(p) silu(T) as bf16 in
 // place (rotary factors requested before the wait for T), reads O, issues y = q~ C (q~ from TMEM, C as
 // bf16 in shared memory) over the O columns, and writes O_s + g r y / rms(y) into the Q slot.  P_q
 // (16 KB) and C (16 KB) of the current (batch, head) take the place of the third V slot.  Arithmetic
 // and order are those of comp.cu's apply pass, so the result equals the two separate calls bit for
 // bit.  Measured (720p shape, 97 % sparsity): the closing grows from ~1300 to ~7200 clocks per item
 // (two dependent tensor-core round trips, 128 special-function operations per row, three passes over
-// TMEM), during which the pipeline drains, so the fused call only just beats the two calls.
+// TMEM), during which the pipeline drains: the fused call takes as long as the two calls it replaces.
 #include <cuda.h>
 #include <cuda_fp8.h>
 
