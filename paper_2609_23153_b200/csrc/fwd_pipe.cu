@@ -1073,13 +1073,15 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       tc_fence_after();
       float inv = l > 0.0f ? 1.0f / l : 0.0f;          // no admissible key at all: zero row, lse = -inf
       if constexpr (FP8) inv *= v_max * 0.0625f;       // undo the 2^4 / max s_v folded into P
+      // (16 columns at a time: this warpgroup runs on 40 registers, and what it spills goes to an L1 that the
+      // shared-memory carve-out leaves very small)
 #pragma unroll 1
-      for (int ch = 0; ch < kPD / 32; ++ch) {
-        uint32_t r[32];
-        tmem_ld32(tmem_O + lane_off + ch * 32, r);
+      for (int ch = 0; ch < kPD / 16; ++ch) {
+        uint32_t r[16];
+        tmem_ld16(tmem_O + lane_off + ch * 16, r);
         tc_wait_ld();
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cc = 0; cc < 2; ++cc) {
           uint32_t ww[4];
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
@@ -1087,7 +1089,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                                                             __uint_as_float(r[8 * cc + 2 * j + 1]) * inv);
             ww[j] = *reinterpret_cast<const uint32_t*>(&h2);
           }
-          *reinterpret_cast<uint4*>(slot + (ch >> 1) * (kTile / 2) + row * 128 + ((((ch & 1) * 4 + cc) ^ (row & 7)) << 4)) =
+          *reinterpret_cast<uint4*>(slot + (ch >> 2) * (kTile / 2) + row * 128 + ((((ch & 3) * 2 + cc) ^ (row & 7)) << 4)) =
               make_uint4(ww[0], ww[1], ww[2], ww[3]);
         }
       }
