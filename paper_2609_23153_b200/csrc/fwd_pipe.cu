@@ -33,14 +33,15 @@
 // compacted by a small pre-pass into the workspace; every role reads the clean lists from there.
 // Every wait is bounded; nothing here waits on another CTA.
 //
-// EPI variant (bf16, kept lists of at most kEpiMaxKept blocks): 512 threads, warps 12-15 are a closing
+// EPI variant (kept lists of at most kEpiMaxKept blocks): 512 threads, warps 12-15 are a closing
 // warpgroup.  At the end of an item the softmax warpgroups only leave their partial row sums (the
 // warpgroup of the last tile in the first KB of the item's dead Q slot, the other one in s_lsum) and go
 // on to the next item's tiles; the closing warpgroup waits for the last PV, reads O, normalises it into
 // the Q slot, hands O back to the PV issuer, writes lse and stores the tile.  That takes the wait for the
-// last PV, the O read and the store off the warpgroup whose next tile the pipeline needs (-2 % at 18
-// tiles per item); with four more warps resident the tile loop itself runs 3 % slower, so the launcher
-// keeps the 384-thread kernel for longer lists, and for FP8, which measured slower with it.
+// last PV, the O read and the store off the warpgroup whose next tile the pipeline needs (bf16 -2.6 %,
+// FP8 -1 % at 18 tiles per item, 6-8 % at 6); with four more warps resident, and 40 registers for the
+// control warps, the tile loop itself runs 3 % slower, so the launcher keeps the 384-thread kernel for
+// longer lists.
 //
 // GATE variant (sparkattn_fwd_gated; bf16, 128-token blocks, 384 threads): the closing softmax warpgroup
 // adds the gated low-rank term of Sec. 4.1 before the store.  Once the last PV of the item is complete it
@@ -64,7 +65,7 @@ namespace sparkattn {
 
 constexpr int kPipeThreads = 384;                           // GATE variant: 4 control warps + 2 softmax warpgroups
 constexpr int kPipeSoftmaxRegs = 216, kPipeCtrlRegs = 64;   // 2*128*216 + 128*64 <= 384*168
-// bf16 with short kept lists (EPI): a third warpgroup (warps 12-15) closes the items, see below
+// short kept lists (EPI): a third warpgroup (warps 12-15) closes the items, see below
 constexpr int kEpiThreads = 512;
 constexpr int kEpiMaxKept = 32;                             // longest kept list the launcher gives to that variant
 constexpr int kEpiSoftmaxRegs = 216, kEpiCtrlRegs = 40, kEpiCloseRegs = 40;   // 2*128*216 + 128*40 + 128*40 = 512*128
@@ -320,7 +321,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   const bool dead = *s_abort != 0;
   const int first_item = blockIdx.x, item_step = gridDim.x;
 
-  static_assert(!EPI || (!GATE && !FP8), "the closing warpgroup exists for the plain bf16 variants");
+  static_assert(!EPI || !GATE, "the gated variant closes its items in the softmax warpgroups");
   if constexpr (EPI) {
     if (warp < 4) reg_dec<kEpiCtrlRegs>();
     else if (warp >= 12) reg_dec<kEpiCloseRegs>();
@@ -1253,12 +1254,16 @@ static int launch_pipe(const sparkattn_shape_t& s, bool fp8, const void* q, cons
                           : (win ? fwd_pipe_kernel<false, true, true> : fwd_pipe_kernel<false, false, true>))
                    : (fp8 ? (win ? fwd_pipe_kernel<true, true, false> : fwd_pipe_kernel<true, false, false>)
                           : (win ? fwd_pipe_kernel<false, true, false> : fwd_pipe_kernel<false, false, false>));
-  // bf16 with short lists: the variant with a closing warpgroup (it takes the item boundary off the softmax
-  // warpgroups, 2 % at 18 tiles per item, but its main loop is 3 % slower: it stops paying near 30 tiles per item)
-  const bool epi = !fp8 && !ga && kmax <= kEpiMaxKept;
-  if (epi)
+  // short lists: the variant with a closing warpgroup (it takes the item boundary off the softmax warpgroups: 2.6 %
+  // bf16 / 1 % FP8 at 18 tiles per item, 6-8 % at 6; but its tile loop is 3 % slower, and the two are level near 60
+  // tiles per item)
+  const bool epi = !ga && kmax <= kEpiMaxKept;
+  if (epi && !fp8)
     kern = pair ? (win ? fwd_pipe_kernel<false, true, true, false, true> : fwd_pipe_kernel<false, false, true, false, true>)
                 : (win ? fwd_pipe_kernel<false, true, false, false, true> : fwd_pipe_kernel<false, false, false, false, true>);
+  if (epi && fp8)
+    kern = pair ? (win ? fwd_pipe_kernel<true, true, true, false, true> : fwd_pipe_kernel<true, false, true, false, true>)
+                : (win ? fwd_pipe_kernel<true, true, false, false, true> : fwd_pipe_kernel<true, false, false, false, true>);
   if (ga) kern = fwd_pipe_kernel<false, false, false, true>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPipeSmem) != cudaSuccess)
     return SPARKATTN_E_CUDA;

@@ -246,15 +246,15 @@ def test_long_permuted_lists_own_block_anywhere(block, fp8):
     assert (num / den) ** 0.5 <= (5e-2 if fp8 else 1e-2)
 
 
-@pytest.mark.parametrize("block,window", [(128, 0), (64, 0), (128, 2)])
-def test_both_bf16_kernels_agree_bitwise(block, window):
-    """bf16, d = 128: kept lists of at most 32 entries run the kernel with a closing warpgroup, longer list strides
-    the two-warpgroup kernel.  The same lists padded to a stride of 40 (the counts say how many entries are real)
+@pytest.mark.parametrize("block,window,fp8", [(128, 0, False), (64, 0, False), (128, 2, False), (128, 0, True), (64, 0, True)])
+def test_both_kernels_agree_bitwise(block, window, fp8):
+    """d = 128: kept lists of at most 32 entries run the kernel with a closing warpgroup, longer list strides the
+    two-warpgroup kernel.  The same lists padded to a stride of 40 (the counts say how many entries are real)
     must give the same output and lse bit for bit: both kernels take every step in the same arithmetic and order.
     More items than SMs, counts 0 ... kmax, a ragged last block; with a causal window the same through the masked
-    instantiations."""
+    instantiations; bf16 and FP8."""
     grid = (15, 18, 19)                                        # N = 5130: 41 blocks of 128 (last: 10 tokens) / 81 of 64
-    w = _small(71 + block + window, 6, 128, grid, block, 0.0)
+    w = _small(71 + block + window + int(fp8), 6, 128, grid, block, 0.0)
     q, k, v = workloads.structured_qkv(w)
     g = torch.Generator().manual_seed(500 + block + window)
     kmax = 9
@@ -265,13 +265,22 @@ def test_both_bf16_kernels_agree_bitwise(block, window):
     wide[:, :, :kmax] = idx
     qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
     kw = dict(frame_tokens=18 * 19, window=window) if window else {}
+    okw = dict(kw)
+    if fp8:
+        cs = [sa.quant_fp8(t, block) for t in (qd, kd, vd)]
+        qd, kd, vd = (c for c, _ in cs)
+        kw["scales"] = tuple(s for _, s in cs)
+        okw["scales"] = tuple(s[0].cpu() for _, s in cs)
     a, la = sa.fwd(qd, kd, vd, idx[None].to(DEV), cnt[None].to(DEV), w.block, return_lse=True, check_status=True, **kw)
     b, lb = sa.fwd(qd, kd, vd, wide[None].to(DEV), cnt[None].to(DEV), w.block, return_lse=True, check_status=True, **kw)
     assert torch.equal(a.view(torch.int16), b.view(torch.int16))
     assert torch.equal(la.view(torch.int32), lb.view(torch.int32))
     items = [(h, i) for h in (0, w.H - 1) for i in list(range(0, w.nb, 5)) + [w.nb - 1] if cnt[h, i] > 0]
-    okw = dict(frame_tokens=18 * 19, window=window) if window else {}
-    ref_out, ref_lse = oracle.attention(q[0], k[0], v[0], idx, cnt, w.block, items=items, **okw)
+    oq, ok_, ov = (qd[0].cpu(), kd[0].cpu(), vd[0].cpu()) if fp8 else (q[0], k[0], v[0])
+    ref_out, ref_lse = oracle.attention(oq, ok_, ov, idx, cnt, w.block, items=items, **okw)
     # (random lists under a causal window leave some rows without any admissible key: lse = -inf on both sides,
     # which test_gpu_window.py checks; here the output alone is compared with the oracle in that case)
-    _compare_items(b[0], None if window else lb[0], ref_out, ref_lse, items, w.block, w.N, BF16_RELRMS, BF16_MAXABS)
+    if fp8:
+        _compare_items(b[0], lb[0], ref_out, ref_lse, items, w.block, w.N, FP8_RELRMS, None)
+    else:
+        _compare_items(b[0], None if window else lb[0], ref_out, ref_lse, items, w.block, w.N, BF16_RELRMS, BF16_MAXABS)
