@@ -73,11 +73,10 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// One token row of T (64 fp32 columns at `taddr`) -> silu -> rank-truncated rotary rotation of the
-// adjacent pairs -> bf16 -> row `row` of a [128 rows x 128 B] tile with 128-byte swizzle.
-// Done in two halves of 32 columns to bound the live registers.
-__device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile, int row, const RopeTable& rope,
-                                            const float2* __restrict__ table, int token) {
+// The (cos, sin) pairs of one token's rank/2 feature pairs, requested from the position-major table.  Called
+// before the wait for the token tile's projection, so that the table's L2 latency is not on the row's path.
+__device__ __forceinline__ void rope_factors(float2 (&cs)[kRank / 2], const RopeTable& rope,
+                                             const float2* __restrict__ table, int token) {
   const int x = token % rope.Wg;
   const int yy = token / rope.Wg;
   const int y = yy % rope.Hg;
@@ -86,26 +85,31 @@ __device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile,
   const float2* row_y = table + (rope.T + y) * (kRank / 2);
   const float2* row_x = table + (rope.T + rope.Hg + x) * (kRank / 2);
 #pragma unroll
+  for (int m = 0; m < kRank / 2; ++m) {
+    const int ax = rope.axis[m];
+    cs[m] = __ldg((ax == 0 ? row_t : (ax == 1 ? row_y : row_x)) + m);
+  }
+}
+
+// One token row of T (64 fp32 columns at `taddr`) -> silu -> rank-truncated rotary rotation of the
+// adjacent pairs -> bf16 -> row `row` of a [128 rows x 128 B] tile with 128-byte swizzle.
+// Done in two halves of 32 columns to bound the live registers.
+__device__ __forceinline__ void feature_row(uint32_t taddr, unsigned char* tile, int row, const float2 (&cs)[kRank / 2]) {
+#pragma unroll
   for (int half = 0; half < 2; ++half) {
     uint32_t r[32];
     tmem_ld32(taddr + half * 32, r);
-    float2 cs[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const int m = half * 16 + j;
-      const int ax = rope.axis[m];
-      cs[j] = __ldg((ax == 0 ? row_t : (ax == 1 ? row_y : row_x)) + m);
-    }
     tc_wait_ld();
     uint32_t w[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
+      const float2 cj = cs[half * 16 + j];
       const float u0 = __uint_as_float(r[2 * j]), u1 = __uint_as_float(r[2 * j + 1]);
       const float2 e = unpack_f32x2(fadd2(pack_f32x2(fast_exp2(u0 * -1.4426950408889634f), fast_exp2(u1 * -1.4426950408889634f)),
                                           pack_f32x2(1.0f, 1.0f)));
       const float z0 = u0 * fast_rcp(e.x), z1 = u1 * fast_rcp(e.y);
-      const float o0 = fmaf(z0, cs[j].x, -z1 * cs[j].y);
-      const float o1 = fmaf(z0, cs[j].y, z1 * cs[j].x);
+      const float o0 = fmaf(z0, cj.x, -z1 * cj.y);
+      const float o1 = fmaf(z0, cj.y, z1 * cj.x);
       const __nv_bfloat162 h2 = __floats2bfloat162_rn(o0, o1);
       w[j] = *reinterpret_cast<const uint32_t*>(&h2);
     }
@@ -295,6 +299,8 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
     unsigned char* tileF = sF + g * 16384;
     bool ok = true;
     for (int i = g, u = 0; ok && i < ntiles; i += kFeatWGs, ++u) {
+      float2 cs[kRank / 2];
+      rope_factors(cs, p.rope, p.rope_table, min((tile0 + i) * kTileTok + row, p.N - 1));   // rows past N are zero anyway
       ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full + g, u & 1, s_abort, p.status, 56));
       if (!ok) break;
       if (u > 0) {                                        // k~ tile g still read by the previous accumulation?
@@ -302,8 +308,7 @@ comp_state_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_const
         if (!ok) break;
       }
       tc_fence_after();
-      feature_row(tmem + g * 64 + lane_off, tileF, row, p.rope, p.rope_table,
-                  min((tile0 + i) * kTileTok + row, p.N - 1));       // rows past N are zero anyway
+      feature_row(tmem + g * 64 + lane_off, tileF, row, cs);
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar_f_full + g);
@@ -522,16 +527,18 @@ comp_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     for (int i = g, u = 0; ok && i < ntiles; i += kFeatWGs, ++u) {
       const int tile_row = (tile0 + i) * kTileTok;
       const int token = tile_row + row;
+      float2 cs[kRank / 2];
+      rope_factors(cs, p.rope, p.rope_table, min(token, p.N - 1));
+      const float gte = token < p.N ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
       ok = __all_sync(0xffffffffu, mbar_wait(bar_t_full + g, u & 1, s_abort, p.status, 64));
       if (!ok) break;
       tc_fence_after();
       // the previous tile of this warpgroup has passed its Y wait, so the q~ tile is free
-      feature_row(tmem_g, tileF, row, p.rope, p.rope_table, min(token, p.N - 1));
+      feature_row(tmem_g, tileF, row, cs);
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar_f_full + g);
 
-      const float gte = token < p.N ? __ldg(p.gate + (int64_t)bh * p.N + token) : 0.0f;
       // sum of squares of the sparse-branch row (rows past N are zero tiles)
       ok = __all_sync(0xffffffffu, mbar_wait(bar_os_full + g, u & 1, s_abort, p.status, 66));
       if (!ok) break;
